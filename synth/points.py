@@ -1,0 +1,41 @@
+"""Interpolation point sets used by the workloads.
+
+Each set is a list of (numerator, denominator) pairs for the finite points,
+followed by the point at infinity written as (1, 0) (projective coordinates,
+Section 2.4).  Standard sets are the integer points of Table 1 (Section 2.2);
+"nova" sets are the discovered configurations of Table 3 (Section 5.2).  The
+half-integer F(6,3) set is the customary Lavin-Gray choice that the workload
+list names as "standard" for that tile.
+"""
+
+INF = (1, 0)
+
+
+def _sym(*pos):
+    out = [(0, 1)]
+    for (a, b) in pos:
+        out.append((a, b))
+        out.append((-a, b))
+    out.append(INF)
+    return out
+
+
+POINT_SETS = {
+    # Table 1: standard integer points
+    ("std", 2): _sym((1, 1)),
+    ("std", 4): _sym((1, 1), (2, 1)),
+    ("std", 6): _sym((1, 1), (2, 1), (3, 1)),
+    ("std", 8): _sym((1, 1), (2, 1), (3, 1), (4, 1)),
+    # customary F(6,3) set with +-1/2 (named "standard" by the F(6,3) workload)
+    ("half", 6): _sym((1, 1), (2, 1), (1, 2)),
+    # Table 3: discovered points
+    ("nova", 2): _sym((1, 1)),
+    ("nova", 4): _sym((5, 6), (7, 6)),
+    ("nova", 6): _sym((3, 5), (1, 1), (7, 6)),
+    ("nova", 8): _sym((2, 5), (5, 6), (1, 1), (7, 6)),
+}
+
+
+def point_set(kind, m):
+    """Return a fresh list of (num, den) pairs; the last entry is infinity."""
+    return list(POINT_SETS[(kind, m)])

@@ -1,0 +1,156 @@
+"""Pins for the oracle's convolution functions (no GPU).
+
+direct_conv_fp64 is checked against plain nested loops and closed forms;
+winograd_conv_fp64 against the direct result (Theorem A.2: the algorithm is
+exact); the exact-rational Winograd against integer direct convolution with
+zero error; the rounding emulation against cases where every rounding is exact.
+"""
+import numpy as np
+import pytest
+
+from oracle import conv
+from synth import POINT_SETS, point_set, make_conv_inputs
+
+ALL_SETS = sorted(POINT_SETS.keys())
+
+
+def brute_force(x, g):
+    N, H, W, C = x.shape
+    K = g.shape[0]
+    y = np.zeros((N, H, W, K))
+    for n in range(N):
+        for h in range(H):
+            for w in range(W):
+                for k in range(K):
+                    s = 0.0
+                    for a in range(3):
+                        for b in range(3):
+                            hh, ww = h + a - 1, w + b - 1
+                            if 0 <= hh < H and 0 <= ww < W:
+                                for c in range(C):
+                                    s += float(x[n, hh, ww, c]) * float(g[k, a, b, c])
+                    y[n, h, w, k] = s
+    return y
+
+
+def test_direct_matches_nested_loops():
+    x, g = make_conv_inputs(2, 5, 7, 3, 4, "fp32", False, False, seed=11)
+    np.testing.assert_allclose(conv.direct_conv_fp64(x, g), brute_force(x, g), rtol=0, atol=1e-12)
+
+
+def test_direct_closed_forms():
+    x, _ = make_conv_inputs(1, 6, 5, 4, 4, "fp32", False, False, seed=12)
+    g = np.zeros((4, 3, 3, 4))
+    for k in range(4):
+        g[k, 1, 1, k] = 1.0                       # centre delta -> identity
+    assert np.array_equal(conv.direct_conv_fp64(x, g), x.astype(np.float64))
+    g = np.zeros((4, 3, 3, 4))
+    for k in range(4):
+        g[k, 0, 2, k] = 1.0                       # tap (a=0,b=2): y[h,w] = x[h-1,w+1]
+    y = conv.direct_conv_fp64(x, g)
+    assert np.array_equal(y[:, 1:, :-1, :], x[:, :-1, 1:, :].astype(np.float64))
+    assert np.all(y[:, 0, :, :] == 0) and np.all(y[:, :, -1, :] == 0)
+    # no kernel flip: an asymmetric filter and its flip give different results
+    x2, g2 = make_conv_inputs(1, 4, 4, 1, 1, "fp32", False, False, seed=13)
+    assert not np.allclose(conv.direct_conv_fp64(x2, g2), conv.direct_conv_fp64(x2, g2[:, ::-1, ::-1, :]))
+
+
+def test_direct_is_linear():
+    x, g = make_conv_inputs(1, 6, 6, 2, 3, "fp32", False, False, seed=14)
+    x2, g2 = make_conv_inputs(1, 6, 6, 2, 3, "fp32", False, False, seed=15)
+    lhs = conv.direct_conv_fp64(x + 2.0 * x2, g)
+    rhs = conv.direct_conv_fp64(x, g) + 2.0 * conv.direct_conv_fp64(x2, g)
+    np.testing.assert_allclose(lhs, rhs, atol=1e-5)
+
+
+@pytest.mark.parametrize("kind,m", ALL_SETS)
+@pytest.mark.parametrize("H,W", [(13, 11), (8, 8), (3, 17)])
+def test_winograd_fp64_equals_direct(kind, m, H, W):
+    x, g = make_conv_inputs(2, H, W, 5, 3, "fp32", False, False, seed=20 + m)
+    y1 = conv.direct_conv_fp64(x, g)
+    y3 = conv.winograd_conv_fp64(x, g, m, point_set(kind, m))
+    tol = 1e-9 if (kind, m) == ("std", 8) else 1e-11
+    assert conv.rel_l2(y3, y1) < tol
+
+
+@pytest.mark.parametrize("kind,m", [("std", 2), ("nova", 4), ("nova", 6), ("nova", 8), ("std", 8)])
+def test_rational_winograd_is_exactly_direct(kind, m):
+    rng = np.random.default_rng(30 + m)
+    H, W = m + 3, m + 1                              # ragged in both directions
+    x = rng.integers(-5, 6, (1, H, W, 2))
+    g = rng.integers(-5, 6, (2, 3, 3, 2))
+    y = conv.winograd_conv_exact(x, g, m, point_set(kind, m))
+    ref = brute_force(x, g)
+    for h in range(H):
+        for w in range(W):
+            for k in range(2):
+                v = y[0][h][w][k]
+                assert v.denominator == 1 and int(v) == int(ref[0, h, w, k])
+
+
+def test_emulation_is_exact_when_every_rounding_is_exact():
+    """F(2,3) standard tables hold only 0, +-1, +-1/2; with small even-integer
+    filters and small integer inputs every intermediate is an integer below
+    2048, so the fp16 pipeline has no rounding and must equal direct conv."""
+    rng = np.random.default_rng(40)
+    x = rng.integers(0, 4, (2, 7, 9, 8)).astype(np.float16)
+    g = (2 * rng.integers(-1, 2, (8, 3, 3, 8))).astype(np.float16)
+    y = conv.winograd_conv_emulated(x, g, 2, point_set("std", 2), "fp16")
+    assert y.dtype == np.float16
+    assert np.array_equal(y.astype(np.float64), conv.direct_conv_fp64(x, g))
+    y32 = conv.winograd_conv_emulated(x.astype(np.float32), g.astype(np.float32), 2,
+                                      point_set("std", 2), "fp32")
+    assert y32.dtype == np.float32
+    assert np.array_equal(y32.astype(np.float64), conv.direct_conv_fp64(x, g))
+
+
+def test_emulation_rounds_operands_to_fp16():
+    """With 1/3-like values the fp16 pipeline must differ from the fp32 one by
+    about the fp16 unit roundoff, and the fp32 one from fp64 by about fp32's."""
+    x, g = make_conv_inputs(2, 12, 12, 16, 16, "fp16", True, True, seed=41)
+    y1 = conv.direct_conv_fp64(x, g)
+    pts = point_set("std", 4)
+    e16 = conv.rel_l2(conv.winograd_conv_emulated(x, g, 4, pts, "fp16"), y1)
+    e32 = conv.rel_l2(conv.winograd_conv_emulated(x.astype(np.float32), g.astype(np.float32), 4, pts, "fp32"), y1)
+    assert 2e-4 < e16 < 2e-2
+    assert 1e-8 < e32 < 1e-5
+    # coefficient precision is second order next to operand rounding
+    e16c = conv.rel_l2(conv.winograd_conv_emulated(x, g, 4, pts, "fp16", coef="fp32"), y1)
+    assert 0.3 < e16c / e16 < 3
+
+
+def test_fp32_emulation_meets_stated_tolerances():
+    x, g = make_conv_inputs(2, 14, 14, 32, 16, "fp32", True, True, seed=42)
+    y1 = conv.direct_conv_fp64(x, g)
+    for kind, m, tol in [("std", 2, 1e-5), ("std", 4, 1e-5), ("nova", 4, 1e-5), ("nova", 6, 1e-4), ("nova", 8, 2e-4)]:
+        e = conv.rel_l2(conv.winograd_conv_emulated(x, g, m, point_set(kind, m), "fp32"), y1)
+        assert e < tol, (kind, m, e)
+
+
+def test_standard_f8_overflows_fp16_and_nova_does_not():
+    x, g = make_conv_inputs(1, 16, 16, 64, 8, "fp16", True, True, seed=43)
+    y1 = conv.direct_conv_fp64(x, g)
+    e_std = conv.rel_l2(conv.winograd_conv_emulated(x, g, 8, point_set("std", 8), "fp16"), y1)
+    e_nova = conv.rel_l2(conv.winograd_conv_emulated(x, g, 8, point_set("nova", 8), "fp16"), y1)
+    assert not np.isfinite(e_std) or e_std >= 1.0
+    assert np.isfinite(e_nova) and e_nova < 1.0
+
+
+def test_relu_and_pool():
+    x = np.array([-1.0, 2.0, np.inf, -np.inf]).reshape(1, 2, 2, 1)
+    assert np.array_equal(conv.relu(x).ravel(), [0, 2, np.inf, 0])
+    p = conv.maxpool2x2(np.arange(16.0).reshape(1, 4, 4, 1))
+    assert np.array_equal(p.ravel(), [5, 7, 13, 15])
+
+
+def test_filter_transform_matches_pipeline_stage():
+    _, g = make_conv_inputs(1, 4, 4, 8, 8, "fp16", True, True, seed=44)
+    U = conv.filter_transform_emulated(g, 4, point_set("nova", 4), "fp16")
+    assert U.shape == (8, 6, 6, 8) and U.dtype == np.float16
+    # centre-only filter: U[k,p,q,c] = G[p,1] G[q,1] g[k,1,1,c]
+    g0 = np.zeros_like(g)
+    g0[:, 1, 1, :] = 1
+    _, G, _ = conv.coefficient_tables(4, point_set("nova", 4), "fp16")
+    U0 = conv.filter_transform_emulated(g0, 4, point_set("nova", 4), "fp16")
+    want = (G[:, 1][:, None] * G[:, 1][None, :]).astype(np.float16)
+    assert np.array_equal(U0[0, :, :, 0], want)

@@ -1,0 +1,135 @@
+"""Pins for the oracle's exact Toom-Cook construction (no GPU).
+
+The construction is checked against what the paper and the mathematics fix:
+the exact decomposition identity, every condition number the paper prints,
+the textbook F(2,3) matrices, and the 1-D algorithm on random integers.
+"""
+import os
+from fractions import Fraction
+import numpy as np
+import pytest
+
+from oracle import toom_cook as tc
+from synth import POINT_SETS, point_set
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+ALL_SETS = sorted(POINT_SETS.keys())
+
+
+@pytest.mark.parametrize("kind,m", ALL_SETS)
+def test_decomposition_identity_is_exact(kind, m):
+    AT, G, BT = tc.build_matrices(m, 3, point_set(kind, m))
+    assert tc.decomposition_residual(m, 3, AT, G, BT) == []
+
+
+def test_identity_detects_planted_mistakes():
+    m = 4
+    AT, G, BT = tc.build_matrices(m, 3, point_set("nova", m))
+    G2 = [row[:] for row in G]
+    G2[1][2] = -G2[1][2]                                   # wrong sign
+    assert tc.decomposition_residual(m, 3, AT, G2, BT)
+    BT2 = [list(r) for r in zip(*BT)]                      # transposed operand
+    assert tc.decomposition_residual(m, 3, AT, G, BT2)
+    AT2 = [row[:] for row in AT]
+    AT2[m - 1][m + 1] = Fraction(0)                        # dropped infinity term
+    assert tc.decomposition_residual(m, 3, AT2, G, BT)
+
+
+def _golden_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "kappa_paper.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                m, kind, mat, val, unit = line.split()
+                rows.append((int(m), kind, mat, float(val), float(unit)))
+    return rows
+
+
+@pytest.mark.parametrize("m,kind,mat,val,unit", _golden_rows())
+def test_paper_condition_numbers(m, kind, mat, val, unit):
+    pts = point_set(kind, m)
+    AT, G, BT = (tc.to_float(M) for M in tc.build_matrices(m, 3, pts))
+    got = {
+        "V": lambda: tc.kappa2_V(pts),
+        "V2D": lambda: tc.kappa2(np.kron(tc.vandermonde(pts), tc.vandermonde(pts))),
+        "A": lambda: tc.kappa2(AT),
+        "B": lambda: tc.kappa2(BT),
+        "G": lambda: tc.kappa2(G),
+        "maxA": lambda: float(np.abs(AT).max()),
+    }[mat]()
+    # the paper rounds (sometimes truncates) to the printed digit
+    assert abs(got - val) <= 1.0 * unit, (got, val)
+
+
+def test_improvement_ratios_match_abstract():
+    # 415x in 1-D and about 172,484x in 2-D for F(8,3) (abstract)
+    k_std, k_nova = tc.kappa2_V(point_set("std", 8)), tc.kappa2_V(point_set("nova", 8))
+    assert abs(k_std / k_nova - 415) < 1.0
+    assert abs((k_std / k_nova) ** 2 - 172484) / 172484 < 5e-3
+
+
+def _read_textbook():
+    mats, cur = {}, None
+    with open(os.path.join(GOLDEN, "f23_textbook.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            if line in ("AT", "G", "BT"):
+                cur = line
+                mats[cur] = []
+            else:
+                mats[cur].append([Fraction(t) for t in line.split()])
+    return mats
+
+
+def test_f23_rank_one_terms_equal_textbook():
+    AT, G, BT = tc.build_matrices(2, 3, point_set("std", 2))
+    ref = _read_textbook()
+    for p in range(4):
+        for i in range(2):
+            for k in range(3):
+                for j in range(4):
+                    assert AT[i][p] * G[p][k] * BT[p][j] == \
+                        ref["AT"][i][p] * ref["G"][p][k] * ref["BT"][p][j]
+
+
+@pytest.mark.parametrize("kind,m", ALL_SETS)
+def test_one_dimensional_algorithm_on_integers(kind, m):
+    """y = A^T[(G g) (.) (B^T x)] equals y_i = sum_k g_k x_{i+k} exactly (Section 2.1)."""
+    AT, G, BT = tc.build_matrices(m, 3, point_set(kind, m))
+    n = m + 2
+    rng = np.random.default_rng(7 + m)
+    x = [int(v) for v in rng.integers(-9, 10, n)]
+    g = [int(v) for v in rng.integers(-9, 10, 3)]
+    gt = [sum(G[p][k] * g[k] for k in range(3)) for p in range(n)]
+    xt = [sum(BT[p][j] * x[j] for j in range(n)) for p in range(n)]
+    y = [sum(AT[i][p] * gt[p] * xt[p] for p in range(n)) for i in range(m)]
+    assert y == [sum(g[k] * x[i + k] for k in range(3)) for i in range(m)]
+
+
+def test_vandermonde_uses_finite_points_only():
+    V = tc.vandermonde(point_set("std", 4))
+    assert V.shape == (5, 5)
+    assert np.array_equal(V[0], [1, 0, 0, 0, 0])           # alpha = 0, 0^0 = 1
+    assert np.array_equal(V[3], [1, 2, 4, 8, 16])
+
+
+def test_invalid_point_sets_are_rejected():
+    with pytest.raises(ValueError):
+        tc.build_matrices(2, 3, [(0, 1), (1, 1), (1, 1), (1, 0)])     # duplicate
+    with pytest.raises(ValueError):
+        tc.build_matrices(2, 3, [(0, 1), (1, 1), (-1, 1), (2, 1)])    # no infinity
+    with pytest.raises(ValueError):
+        tc.build_matrices(2, 3, [(0, 1), (1, 0), (-1, 1), (1, 0)])    # two infinities
+    with pytest.raises(ValueError):
+        tc.build_matrices(4, 3, point_set("std", 2))                  # wrong count
+
+
+def test_float_tables_are_correctly_rounded():
+    AT, G, BT = tc.build_matrices(4, 3, point_set("nova", 4))
+    a = tc.to_float(G)
+    assert a[1, 0] == float(G[1][0])
+    assert tc.to_float(G, np.float16).dtype == np.float16
+    assert float(tc.to_float(AT, np.float16)[1, 1]) == float(np.float16(5 / 6))
