@@ -1,0 +1,170 @@
+/*
+ * nova.h - C ABI of the B200 (sm_100a) Winograd convolution library.
+ *
+ * 2-D Winograd convolution F(m x m, 3 x 3), m in {2, 4, 6, 8}, driven by an
+ * arbitrary set of interpolation points (possibly fractional) with the point
+ * at infinity, as in Section 2.1 ("Winograd Convolution via Cook-Toom") of
+ * "NOVA: Discovering Well-Conditioned Winograd Transforms through Numerical
+ * Optimization of Vandermonde Arithmetic".
+ *
+ * Fixed semantics: cross-correlation y_i = sum_k g_k x_{i+k} (Section 2.1),
+ * stride 1, zero padding 1, dilation 1, groups 1, tensors NHWC:
+ *   x [N,H,W,C]   g [K,3,3,C]   y [N,H,W,K],  C % 8 == 0 and K % 8 == 0.
+ * The image is cut into ceil(H/m) x ceil(W/m) tiles; tile (th, tw) reads the
+ * n x n patch (n = m + 2) whose top-left corner is (m*th - 1, m*tw - 1) of the
+ * zero-extended image; outputs beyond H x W are dropped.
+ *
+ * Every function returns an int status (0 = NOVA_OK, negative = error) unless
+ * stated otherwise; nothing throws or aborts across this boundary.  Pointers
+ * named *_dev are device pointers, *_host host pointers; the caller owns every
+ * buffer.  Device work is enqueued on `stream` (a cudaStream_t passed as
+ * void*) and is asynchronous.  There is no CPU fallback: without a CUDA device
+ * the device entry points return NOVA_ERR_CUDA.
+ */
+#ifndef NOVA_H_
+#define NOVA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* A point alpha = num/den (den > 0).  den == 0 denotes the point at infinity,
+ * projective (1:0) (Section 2.4, "Symbolic Verification"). */
+typedef struct { int64_t num, den; } nova_rat;
+
+/* Arithmetic mode.  NOVA_FP32: x, g, y and every intermediate are float.
+ * NOVA_FP16_F32ACC: x, g, y are IEEE half; transforms are evaluated in float
+ * and rounded once to half; the transformed-domain product accumulates in
+ * float (Section 5.1 "FP16 Setup"; Appendix "Float16 Precision Analysis"). */
+enum { NOVA_FP32 = 0, NOVA_FP16_F32ACC = 1 };
+
+/* Precision of the transform coefficient tables in NOVA_FP16_F32ACC mode:
+ * rounded to half then widened (the paper's "cast to FP16"), or float. */
+enum { NOVA_COEF_ROUND_TO_MODE = 0, NOVA_COEF_FP32 = 1 };
+
+/* nova_conv2d_fwd flags (bitwise or). */
+enum {
+  NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
+  NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
+  NOVA_GEMM_TCGEN05 = 2 << 8 /* force the tcgen05 tensor-core product kernel */
+};
+
+enum {
+  NOVA_OK = 0,
+  NOVA_ERR_INVALID_ARG = -1,        /* null / misaligned pointer, bad shape, m not in {2,4,6,8}, n != m+r-1 */
+  NOVA_ERR_NO_INFINITY = -2,        /* the point set has no point at infinity */
+  NOVA_ERR_MULTIPLE_INFINITY = -3,  /* more than one, or infinity not last */
+  NOVA_ERR_DUPLICATE_POINT = -4,    /* finite points must be distinct (Theorem A.2) */
+  NOVA_ERR_RATIONAL_OVERFLOW = -5,  /* an exact matrix entry does not fit 127-bit rationals */
+  NOVA_ERR_VERIFY_FAILED = -6,      /* the exact decomposition identity is not zero */
+  NOVA_ERR_UNSUPPORTED = -7,        /* r != 3, or an unsupported mode on this path */
+  NOVA_ERR_CUDA = -8,               /* a CUDA runtime/driver call failed (or no device) */
+  NOVA_ERR_DEVICE_TIMEOUT = -9,     /* a bounded device-side wait expired */
+  NOVA_ERR_WORKSPACE = -10          /* workspace too small or misaligned */
+};
+
+typedef struct nova_plan nova_plan;   /* opaque; immutable after creation */
+typedef void* nova_stream;            /* a cudaStream_t */
+
+/*
+ * Build the transform matrices for F(m, r) from `n` points (n == m + r - 1),
+ * exactly one of which - the last - is infinity.  Algorithm 3 ("Symbolic
+ * Cook-Toom Construction"): Lagrange factors F_i = prod_{j!=i}(a_i - a_j);
+ * A^T[i][p] = a_p^i (infinity column e_{m-1}); G[p][k] = a_p^k / F_p (infinity
+ * row e_{r-1}); B^T[p][:] = ascending coefficients of prod_{j!=p}(t - a_j)
+ * (infinity row: prod_j (t - a_j)).  All entries are computed as exact
+ * rationals, the decomposition identity of Section 2.4 is checked to be
+ * exactly zero, and the tables are then rounded (rational -> double -> float
+ * or half, round to nearest even).  Host only: works without a CUDA device.
+ * On success *out must be released with nova_plan_destroy.
+ */
+int nova_plan_create(int m, int r, const nova_rat* points_host, int n,
+                     int mode, int coef, nova_plan** out);
+void nova_plan_destroy(nova_plan* plan);
+
+/* Copy the fp64 tables, row-major, in the caller's point order:
+ * AT [m*n], G [n*r], BT [n*n].  Any pointer may be null. */
+int nova_plan_get_matrices(const nova_plan* plan, double* AT_host, double* G_host, double* BT_host);
+
+/* The tables as the kernels use them (after rounding to the coefficient
+ * precision), as float, same shapes. */
+int nova_plan_get_device_tables(const nova_plan* plan, float* AT_host, float* G_host, float* BT_host);
+
+/* kappa_2 = sigma_max/sigma_min of the Vandermonde matrix V_ij = a_i^j over the
+ * n-1 finite points only (Section 2.2, "Vandermonde Conditioning"). */
+int nova_plan_kappa(const nova_plan* plan, double* kappa2_V_host);
+
+/* Bytes of the transformed filter U for K filters of C channels. */
+size_t nova_filter_transform_bytes(const nova_plan* plan, int K, int C);
+
+/*
+ * Kernel transform (Section 2.1 step 2, nested in 2-D as in Appendix B.5):
+ * U = G g G^T for every (k, c), evaluated in float and rounded once to the
+ * operand type.  g_dev [K,3,3,C] (half or float per the plan's mode);
+ * U_dev receives a library-defined layout ([n*n][K][C], operand type) of
+ * nova_filter_transform_bytes() bytes, 16-byte aligned.
+ */
+int nova_filter_transform(const nova_plan* plan, const void* g_dev, int K, int C,
+                          void* U_dev, nova_stream stream);
+
+/* Scratch (device global memory) nova_conv2d_fwd wants for this problem; any
+ * size >= nova_conv2d_min_workspace_bytes() works (the batch of tiles is then
+ * processed in more, smaller chunks). */
+size_t nova_conv2d_workspace_bytes(const nova_plan* plan, int N, int H, int W, int C, int K);
+size_t nova_conv2d_min_workspace_bytes(const nova_plan* plan, int N, int H, int W, int C, int K);
+
+/*
+ * Forward convolution (Section 2.1 steps 1, 3, 4; 2-D form
+ * Y = A^T [ (G g G^T) (.) (B^T d B) ] A summed over input channels):
+ * input-tile transform V = B^T d B (float, rounded once to the operand type),
+ * transformed-domain product M[f] = V[f] U[f]^T for each of the n*n
+ * frequencies f (float accumulation; tcgen05 tensor cores in fp16 mode), and
+ * output transform Y = A^T M A (float, rounded once to the storage type).
+ * x_dev [N,H,W,C], y_dev [N,H,W,K] in the storage type, 16-byte aligned;
+ * U_dev from nova_filter_transform with the same plan, K and C.
+ * workspace_dev: 256-byte aligned scratch of workspace_bytes; contents are
+ * undefined afterwards; calls sharing a workspace must be stream-ordered.
+ */
+int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
+                    int N, int H, int W, int C, int K,
+                    void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream);
+
+/*
+ * The same call for host tensors: copies x_host to x_stage_dev, runs
+ * nova_conv2d_fwd, copies the result to y_host, all on `stream`.  The staging
+ * buffers are device memory of the sizes of x and y.  Host buffers should be
+ * page-locked for the copies to be asynchronous.
+ */
+int nova_conv2d_fwd_host(const nova_plan* plan, const void* x_host, const void* U_dev, void* y_host,
+                         int N, int H, int W, int C, int K,
+                         void* x_stage_dev, void* y_stage_dev,
+                         void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream);
+
+/* Number of kernel launches one nova_conv2d_fwd call issues for this problem
+ * and workspace size (negative = error). */
+int nova_conv2d_launch_count(const nova_plan* plan, int N, int H, int W, int C, int K,
+                             size_t workspace_bytes, int flags);
+
+/* 2x2 max pooling, stride 2, NHWC, H and W even, C % 8 == 0 (used between the
+ * blocks of a VGG-style stack; not part of the paper's method).  `mode`
+ * selects half or float elements. */
+int nova_maxpool2x2(const void* x_dev, void* y_dev, int N, int H, int W, int C,
+                    int mode, nova_stream stream);
+
+/*
+ * Device-side health: every wait inside the kernels is bounded; a wait that
+ * expires records NOVA_ERR_DEVICE_TIMEOUT in a plan-owned device word.  This
+ * call synchronises `stream`, reads and clears that word, and returns it (or
+ * NOVA_ERR_CUDA if the stream reports an error).
+ */
+int nova_last_device_status(const nova_plan* plan, nova_stream stream);
+
+const char* nova_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* NOVA_H_ */

@@ -1,0 +1,203 @@
+"""ctypes binding of libnova.so: argument marshalling only."""
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libnova.so")
+
+FP32, FP16_F32ACC = 0, 1
+COEF_ROUND_TO_MODE, COEF_FP32 = 0, 1
+RELU = 1
+GEMM_SIMT = 1 << 8
+GEMM_TCGEN05 = 2 << 8
+
+EXPORTED_SYMBOLS = (
+    "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
+    "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
+    "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
+    "nova_conv2d_fwd_host", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
+    "nova_status_string",
+)
+
+
+class NovaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, status_string(status), status))
+
+
+class _Rat(ctypes.Structure):
+    _fields_ = [("num", ctypes.c_int64), ("den", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libnova.so; there is no fallback when it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("libnova.so is not built; run `python -m paper_2512_18453_b200.build`")
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.nova_plan_create.argtypes = [i, i, ctypes.POINTER(_Rat), i, i, i, ctypes.POINTER(vp)]
+    L.nova_plan_create.restype = i
+    L.nova_plan_destroy.argtypes = [vp]
+    L.nova_plan_destroy.restype = None
+    dp, fp = ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_float)
+    L.nova_plan_get_matrices.argtypes = [vp, dp, dp, dp]
+    L.nova_plan_get_matrices.restype = i
+    L.nova_plan_get_device_tables.argtypes = [vp, fp, fp, fp]
+    L.nova_plan_get_device_tables.restype = i
+    L.nova_plan_kappa.argtypes = [vp, dp]
+    L.nova_plan_kappa.restype = i
+    L.nova_filter_transform_bytes.argtypes = [vp, i, i]
+    L.nova_filter_transform_bytes.restype = sz
+    L.nova_filter_transform.argtypes = [vp, vp, i, i, vp, vp]
+    L.nova_filter_transform.restype = i
+    for name in ("nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes"):
+        getattr(L, name).argtypes = [vp, i, i, i, i, i]
+        getattr(L, name).restype = sz
+    L.nova_conv2d_fwd.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, sz, i, vp]
+    L.nova_conv2d_fwd.restype = i
+    L.nova_conv2d_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, vp, sz, i, vp]
+    L.nova_conv2d_fwd_host.restype = i
+    L.nova_conv2d_launch_count.argtypes = [vp, i, i, i, i, i, sz, i]
+    L.nova_conv2d_launch_count.restype = i
+    L.nova_maxpool2x2.argtypes = [vp, vp, i, i, i, i, i, vp]
+    L.nova_maxpool2x2.restype = i
+    L.nova_last_device_status.argtypes = [vp, vp]
+    L.nova_last_device_status.restype = i
+    L.nova_status_string.argtypes = [i]
+    L.nova_status_string.restype = ctypes.c_char_p
+    _lib = L
+    return L
+
+
+def status_string(status):
+    return lib().nova_status_string(int(status)).decode()
+
+
+def _check(status, where):
+    if status != 0:
+        raise NovaError(status, where)
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _torch_dtype(mode):
+    import torch
+    return torch.float32 if mode == FP32 else torch.float16
+
+
+class Plan:
+    """nova_plan: transform matrices for F(m x m, 3 x 3) from a point set.
+
+    points: list of (num, den); exactly one entry, the last, has den == 0
+    (the point at infinity).
+    """
+
+    def __init__(self, m, points, mode=FP16_F32ACC, coef=COEF_ROUND_TO_MODE, r=3):
+        arr = (_Rat * len(points))(*[_Rat(int(a), int(b)) for a, b in points])
+        h = ctypes.c_void_p()
+        _check(lib().nova_plan_create(m, r, arr, len(points), mode, coef, ctypes.byref(h)), "nova_plan_create")
+        self._h = h
+        self.m, self.r, self.n, self.mode, self.coef = m, r, m + r - 1, mode, coef
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().nova_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- host side
+    def matrices(self):
+        import numpy as np
+        AT = np.empty((self.m, self.n)); G = np.empty((self.n, self.r)); BT = np.empty((self.n, self.n))
+        dp = ctypes.POINTER(ctypes.c_double)
+        _check(lib().nova_plan_get_matrices(self._h, AT.ctypes.data_as(dp), G.ctypes.data_as(dp),
+                                            BT.ctypes.data_as(dp)), "nova_plan_get_matrices")
+        return AT, G, BT
+
+    def device_tables(self):
+        import numpy as np
+        AT = np.empty((self.m, self.n), np.float32); G = np.empty((self.n, self.r), np.float32)
+        BT = np.empty((self.n, self.n), np.float32)
+        fp = ctypes.POINTER(ctypes.c_float)
+        _check(lib().nova_plan_get_device_tables(self._h, AT.ctypes.data_as(fp), G.ctypes.data_as(fp),
+                                                 BT.ctypes.data_as(fp)), "nova_plan_get_device_tables")
+        return AT, G, BT
+
+    def kappa(self):
+        k = ctypes.c_double()
+        _check(lib().nova_plan_kappa(self._h, ctypes.byref(k)), "nova_plan_kappa")
+        return k.value
+
+    # ---- device side (torch tensors carry the memory)
+    def filter_transform_bytes(self, K, C):
+        return lib().nova_filter_transform_bytes(self._h, K, C)
+
+    def filter_transform(self, g):
+        """g [K,3,3,C] on the GPU in the plan's storage dtype -> opaque U tensor."""
+        import torch
+        assert g.is_cuda and g.is_contiguous() and g.dtype == _torch_dtype(self.mode)
+        K, _, _, C = g.shape
+        U = torch.empty(self.n * self.n, K, C, dtype=g.dtype, device=g.device)
+        _check(lib().nova_filter_transform(self._h, g.data_ptr(), K, C, U.data_ptr(), _stream()),
+               "nova_filter_transform")
+        return U
+
+    def workspace_bytes(self, N, H, W, C, K):
+        return lib().nova_conv2d_workspace_bytes(self._h, N, H, W, C, K)
+
+    def min_workspace_bytes(self, N, H, W, C, K):
+        return lib().nova_conv2d_min_workspace_bytes(self._h, N, H, W, C, K)
+
+    def launch_count(self, N, H, W, C, K, workspace_bytes, flags=0):
+        return lib().nova_conv2d_launch_count(self._h, N, H, W, C, K, workspace_bytes, flags)
+
+    def conv2d(self, x, U, y=None, workspace=None, flags=0):
+        """x [N,H,W,C], U from filter_transform -> y [N,H,W,K]."""
+        import torch
+        assert x.is_cuda and x.is_contiguous() and x.dtype == _torch_dtype(self.mode)
+        N, H, W, C = x.shape
+        K = U.shape[1]
+        if y is None:
+            y = torch.empty(N, H, W, K, dtype=x.dtype, device=x.device)
+        if workspace is None:
+            workspace = torch.empty(self.workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device=x.device)
+        _check(lib().nova_conv2d_fwd(self._h, x.data_ptr(), U.data_ptr(), y.data_ptr(), N, H, W, C, K,
+                                     workspace.data_ptr(), workspace.numel(), flags, _stream()),
+               "nova_conv2d_fwd")
+        return y
+
+    def conv2d_host(self, x_host, U, y_host, x_stage, y_stage, workspace, flags=0):
+        """Host tensors in and out (pinned for asynchronous copies)."""
+        N, H, W, C = x_host.shape
+        K = U.shape[1]
+        _check(lib().nova_conv2d_fwd_host(self._h, x_host.data_ptr(), U.data_ptr(), y_host.data_ptr(),
+                                          N, H, W, C, K, x_stage.data_ptr(), y_stage.data_ptr(),
+                                          workspace.data_ptr(), workspace.numel(), flags, _stream()),
+               "nova_conv2d_fwd_host")
+        return y_host
+
+    def device_status(self):
+        return lib().nova_last_device_status(self._h, _stream())
+
+
+def maxpool2x2(x, mode):
+    import torch
+    N, H, W, C = x.shape
+    y = torch.empty(N, H // 2, W // 2, C, dtype=x.dtype, device=x.device)
+    _check(lib().nova_maxpool2x2(x.data_ptr(), y.data_ptr(), N, H, W, C, mode, _stream()), "nova_maxpool2x2")
+    return y

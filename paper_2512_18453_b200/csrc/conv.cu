@@ -1,0 +1,162 @@
+// Host orchestration of the forward convolution and the remaining C ABI.
+//
+// The tiles of a problem are processed in chunks sized so that the transformed
+// input V (operand type) and the transformed-domain product M (float) of one
+// chunk stay resident in the 126 MB L2: input transform -> product -> output
+// transform per chunk, all on the caller's stream, no host synchronisation.
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+
+namespace nova {
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kTargetChunkBytes = (size_t)64 << 20;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Chunking {
+  int pc;            // tiles per chunk
+  int pc_pad;        // row stride of V and M inside the workspace
+  int chunks;
+  size_t v_bytes, m_bytes;
+};
+
+size_t per_tile_bytes(const nova_plan* p, const Geom& g) {
+  return (size_t)g.n * g.n * ((size_t)g.C * elt_bytes(p->mode) + (size_t)g.K * 4);
+}
+
+// Largest chunk (a multiple of 128 tiles when possible) that fits `bytes`.
+bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* c) {
+  const size_t pt = per_tile_bytes(p, g);
+  if (bytes < 2 * kAlign + pt) return false;
+  long long pc = (long long)((bytes - 2 * kAlign) / pt);
+  if (pc >= g.P) pc = g.P;
+  else if (pc >= 128) pc = pc / 128 * 128;
+  else if (pc >= 8) pc = pc / 8 * 8;
+  if (pc < 1) return false;
+  c->pc = (int)pc;
+  c->pc_pad = (int)pc;
+  c->chunks = (int)((g.P + pc - 1) / pc);
+  c->v_bytes = round_up((size_t)g.n * g.n * c->pc_pad * g.C * elt_bytes(p->mode), kAlign);
+  c->m_bytes = round_up((size_t)g.n * g.n * c->pc_pad * g.K * 4, kAlign);
+  return c->v_bytes + c->m_bytes <= bytes;
+}
+
+bool shape_ok(int N, int H, int W, int C, int K) {
+  return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
+}
+bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+bool use_tcgen05(const nova_plan* p, int flags) {
+  if (p->mode == NOVA_FP32) return false;
+  return (flags & NOVA_GEMM_SIMT) == 0;
+}
+
+}  // namespace
+}  // namespace nova
+
+using namespace nova;
+
+extern "C" size_t nova_filter_transform_bytes(const nova_plan* p, int K, int C) {
+  if (!p || K <= 0 || C <= 0) return 0;
+  return (size_t)p->n * p->n * K * C * elt_bytes(p->mode);
+}
+
+extern "C" int nova_filter_transform(const nova_plan* p, const void* g, int K, int C, void* U,
+                                     nova_stream stream) {
+  if (!p || !aligned16(g) || !aligned16(U) || K <= 0 || C <= 0 || (K % 8) || (C % 8))
+    return NOVA_ERR_INVALID_ARG;
+  return launch_filter_transform(p, g, K, C, U, stream) == 0 ? NOVA_OK : NOVA_ERR_CUDA;
+}
+
+extern "C" size_t nova_conv2d_min_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
+  if (!p || !shape_ok(N, H, W, C, K)) return 0;
+  Geom g = make_geom(p, N, H, W, C, K);
+  const long long pc = g.P < 128 ? g.P : 128;
+  return (size_t)pc * per_tile_bytes(p, g) + 4 * kAlign;
+}
+
+extern "C" size_t nova_conv2d_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
+  if (!p || !shape_ok(N, H, W, C, K)) return 0;
+  Geom g = make_geom(p, N, H, W, C, K);
+  const size_t pt = per_tile_bytes(p, g);
+  long long pc = (long long)(kTargetChunkBytes / pt) / 128 * 128;
+  if (pc < 128) pc = 128;
+  if (pc > g.P) pc = g.P;
+  return (size_t)pc * pt + 4 * kAlign;
+}
+
+extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W, int C, int K,
+                                        size_t workspace_bytes, int flags) {
+  (void)flags;
+  if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  Geom g = make_geom(p, N, H, W, C, K);
+  Chunking c;
+  if (!choose_chunking(p, g, workspace_bytes, &c)) return NOVA_ERR_WORKSPACE;
+  return 3 * c.chunks;
+}
+
+extern "C" int nova_conv2d_fwd(const nova_plan* p, const void* x, const void* U, void* y, int N, int H,
+                               int W, int C, int K, void* ws, size_t ws_bytes, int flags,
+                               nova_stream stream) {
+  if (!p || !aligned16(x) || !aligned16(U) || !aligned16(y) || !shape_ok(N, H, W, C, K))
+    return NOVA_ERR_INVALID_ARG;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
+  if ((flags & NOVA_GEMM_TCGEN05) && p->mode == NOVA_FP32) return NOVA_ERR_UNSUPPORTED;
+  Geom g = make_geom(p, N, H, W, C, K);
+  Chunking c;
+  if (!choose_chunking(p, g, ws_bytes, &c)) return NOVA_ERR_WORKSPACE;
+  const bool tc = use_tcgen05(p, flags);
+  if (tc && !p->status_dev) return NOVA_ERR_CUDA;
+  char* Vb = static_cast<char*>(ws);
+  float* Mb = reinterpret_cast<float*>(Vb + c.v_bytes);
+  const int nfreq = g.n * g.n;
+  for (long long p0 = 0; p0 < g.P; p0 += c.pc) {
+    const int pc = (int)((g.P - p0) < c.pc ? (g.P - p0) : c.pc);
+    if (launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream)) return NOVA_ERR_CUDA;
+    const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream)
+                     : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);
+    if (e) return NOVA_ERR_CUDA;
+    if (launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, (flags & NOVA_RELU) ? 1 : 0, stream))
+      return NOVA_ERR_CUDA;
+  }
+  return NOVA_OK;
+}
+
+extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, const void* U, void* y_host,
+                                    int N, int H, int W, int C, int K, void* x_stage, void* y_stage,
+                                    void* ws, size_t ws_bytes, int flags, nova_stream stream) {
+  if (!p || !x_host || !y_host || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t xb = (size_t)N * H * W * C * elt_bytes(p->mode);
+  const size_t yb = (size_t)N * H * W * K * elt_bytes(p->mode);
+  if (cudaMemcpyAsync(x_stage, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return NOVA_ERR_CUDA;
+  const int st = nova_conv2d_fwd(p, x_stage, U, y_stage, N, H, W, C, K, ws, ws_bytes, flags, stream);
+  if (st != NOVA_OK) return st;
+  if (cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return NOVA_ERR_CUDA;
+  return NOVA_OK;
+}
+
+extern "C" int nova_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode,
+                               nova_stream stream) {
+  if (!aligned16(x) || !aligned16(y) || N <= 0 || H <= 0 || W <= 0 || (H & 1) || (W & 1) || C <= 0 || (C % 8))
+    return NOVA_ERR_INVALID_ARG;
+  if (mode != NOVA_FP32 && mode != NOVA_FP16_F32ACC) return NOVA_ERR_INVALID_ARG;
+  return launch_maxpool2x2(x, y, N, H, W, C, mode, stream) == 0 ? NOVA_OK : NOVA_ERR_CUDA;
+}
+
+extern "C" int nova_last_device_status(const nova_plan* p, nova_stream stream) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  if (!p->status_dev) return NOVA_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  int v = 0;
+  if (cudaMemcpyAsync(&v, p->status_dev, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return NOVA_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return NOVA_ERR_CUDA;
+  if (v != 0) {
+    cudaMemsetAsync(p->status_dev, 0, sizeof(int), s);
+    cudaStreamSynchronize(s);
+  }
+  return v;
+}

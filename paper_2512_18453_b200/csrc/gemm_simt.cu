@@ -1,0 +1,88 @@
+// Transformed-domain product on CUDA cores (Section 2.1 step 3, summed over
+// input channels): for every frequency f,
+//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c]   (float accumulation).
+// This is the product kernel of the fp32 mode (a single-pass TF32 tensor-core
+// product cannot meet a 1e-5 tolerance) and a cross-check for the tcgen05
+// kernel in fp16 mode.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+
+namespace nova {
+namespace {
+
+constexpr int BM = 64, BN = 64, BK = 16;
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__half v) { return __half2float(v); }
+
+// 256 threads, each a 4 x 4 block of the 64 x 64 output tile.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __restrict__ Mo,
+                 int pc, int pc_pad, int C, int K) {
+  __shared__ float sV[BK][BM + 4];
+  __shared__ float sU[BK][BN + 4];
+  const int f = blockIdx.z;
+  const int pb = blockIdx.x * BM, kb = blockIdx.y * BN;
+  const T* Vf = V + (size_t)f * pc_pad * C;
+  const T* Uf = U + (size_t)f * K * C;
+  float* Mf = Mo + (size_t)f * pc_pad * K;
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;           // tx -> k, ty -> p
+  const int lr = tid >> 2, lc = (tid & 3) * 4;      // loader: row 0..63, 4 channels at lc
+  float acc[4][4] = {};
+  for (int c0 = 0; c0 < C; c0 += BK) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int c = c0 + lc + e;
+      const int p = pb + lr, k = kb + lr;
+      sV[lc + e][lr] = (p < pc && c < C) ? to_f(Vf[(size_t)p * C + c]) : 0.f;
+      sU[lc + e][lr] = (k < K && c < C) ? to_f(Uf[(size_t)k * C + c]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = sV[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = sU[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int p = pb + ty * 4 + i;
+    if (p >= pc) continue;
+    const int k = kb + tx * 4;
+    if (k + 3 < K) {
+      *reinterpret_cast<float4*>(Mf + (size_t)p * K + k) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (k + j < K) Mf[(size_t)p * K + k + j] = acc[i][j];
+    }
+  }
+}
+
+}  // namespace
+
+int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M, int nfreq, int pc,
+                     int pc_pad, int C, int K, void* stream) {
+  dim3 grid((pc + BM - 1) / BM, (K + BN - 1) / BN, nfreq);
+  if (plan->mode == NOVA_FP32)
+    gemm_simt_kernel<float><<<grid, 256, 0, (cudaStream_t)stream>>>((const float*)V, (const float*)U, M, pc,
+                                                                    pc_pad, C, K);
+  else
+    gemm_simt_kernel<__half><<<grid, 256, 0, (cudaStream_t)stream>>>((const __half*)V, (const __half*)U, M,
+                                                                     pc, pc_pad, C, K);
+  return (int)cudaGetLastError();
+}
+
+}  // namespace nova

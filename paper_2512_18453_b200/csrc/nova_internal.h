@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of libnova.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include "nova.h"
+
+namespace nova {
+
+constexpr int kMaxN = 10;   // n = m + 2 for m = 8
+constexpr int kMaxM = 8;
+constexpr int kR = 3;
+
+// Coefficient tables as the kernels evaluate them.  Passed by value as a
+// __grid_constant__ kernel parameter, i.e. they live in the constant bank and
+// fully unrolled loops read them as constant-memory operands.
+struct Coefs {
+  float BT[kMaxN][kMaxN];
+  float AT[kMaxM][kMaxN];
+  float G[kMaxN][kR];
+};
+
+}  // namespace nova
+
+struct nova_plan {
+  int m, r, n;
+  int mode, coef;
+  nova_rat points[nova::kMaxN];
+  double AT[nova::kMaxM * nova::kMaxN];   // m x n row-major
+  double G[nova::kMaxN * nova::kR];       // n x r
+  double BT[nova::kMaxN * nova::kMaxN];   // n x n
+  double kappa2_V;
+  nova::Coefs coefs;                      // rounded to the coefficient precision
+  int* status_dev;                        // device status word (null without a device)
+  int device;                             // device that owns status_dev
+};
+
+namespace nova {
+
+inline size_t elt_bytes(int mode) { return mode == NOVA_FP32 ? 4 : 2; }
+
+// Tile geometry of one problem.
+struct Geom {
+  int N, H, W, C, K, m, n, Th, Tw;
+  long long P;   // total tiles
+};
+inline Geom make_geom(const nova_plan* p, int N, int H, int W, int C, int K) {
+  Geom g;
+  g.N = N; g.H = H; g.W = W; g.C = C; g.K = K; g.m = p->m; g.n = p->n;
+  g.Th = (H + p->m - 1) / p->m;
+  g.Tw = (W + p->m - 1) / p->m;
+  g.P = (long long)N * g.Th * g.Tw;
+  return g;
+}
+
+// Kernel launchers (defined in the .cu files).  All return a cudaError_t as int.
+int launch_filter_transform(const nova_plan* plan, const void* g, int K, int C, void* U, void* stream);
+int launch_input_transform(const nova_plan* plan, const Geom& g, const void* x, void* V,
+                           long long p0, int pc, int pc_pad, void* stream);
+int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y,
+                            long long p0, int pc, int pc_pad, int relu, void* stream);
+int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,
+                     int nfreq, int pc, int pc_pad, int C, int K, void* stream);
+int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M,
+                        int nfreq, int pc, int pc_pad, int C, int K, int* status_dev, void* stream);
+int launch_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode, void* stream);
+
+}  // namespace nova

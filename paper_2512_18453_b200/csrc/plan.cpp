@@ -1,0 +1,390 @@
+// Host-side plan builder: exact Toom-Cook construction of A^T, G, B^T from a
+// rational point set with the point at infinity (Algorithm 3, "Symbolic
+// Cook-Toom Construction"), the exact decomposition check of Section 2.4,
+// rounding of the tables, and kappa_2 of the Vandermonde matrix (Section 2.2).
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime_api.h>
+
+#include "nova_internal.h"
+
+namespace {
+
+typedef __int128 i128;
+typedef unsigned __int128 u128;
+
+// ---------------------------------------------------------------- rationals
+// Reduced fractions over 128-bit integers; `bad` latches overflow.
+struct Rat {
+  i128 n = 0, d = 1;
+};
+
+i128 iabs(i128 v) { return v < 0 ? -v : v; }
+i128 gcd128(i128 a, i128 b) {
+  a = iabs(a); b = iabs(b);
+  while (b) { i128 t = a % b; a = b; b = t; }
+  return a;
+}
+struct Arith {
+  bool bad = false;
+  i128 mul(i128 a, i128 b) {
+    i128 r;
+    if (__builtin_mul_overflow(a, b, &r)) { bad = true; return 0; }
+    return r;
+  }
+  i128 add(i128 a, i128 b) {
+    i128 r;
+    if (__builtin_add_overflow(a, b, &r)) { bad = true; return 0; }
+    return r;
+  }
+  Rat norm(i128 n, i128 d) {
+    if (d == 0) { bad = true; return Rat(); }
+    if (d < 0) { n = -n; d = -d; }
+    i128 g = gcd128(n, d);
+    if (g > 1) { n /= g; d /= g; }
+    Rat r; r.n = n; r.d = d;
+    return r;
+  }
+  Rat mul(const Rat& a, const Rat& b) {
+    // cross-reduce first to keep the products small
+    i128 g1 = gcd128(a.n, b.d), g2 = gcd128(b.n, a.d);
+    if (g1 == 0) g1 = 1;
+    if (g2 == 0) g2 = 1;
+    return norm(mul(a.n / g1, b.n / g2), mul(a.d / g2, b.d / g1));
+  }
+  Rat div(const Rat& a, const Rat& b) {
+    if (b.n == 0) { bad = true; return Rat(); }
+    Rat inv; inv.n = b.d; inv.d = b.n;
+    if (inv.d < 0) { inv.n = -inv.n; inv.d = -inv.d; }
+    return mul(a, inv);
+  }
+  Rat plus(const Rat& a, const Rat& b) {
+    Rat nb = b; nb.n = -nb.n;
+    return sub(a, nb);
+  }
+  Rat sub(const Rat& a, const Rat& b) {
+    i128 g = gcd128(a.d, b.d);
+    if (g == 0) g = 1;
+    i128 bd = b.d / g, ad = a.d / g;
+    return norm(add(mul(a.n, bd), -mul(b.n, ad)), mul(a.d, bd));
+  }
+};
+
+double rat_to_double(const Rat& r) {
+  const i128 lim = (i128)1 << 53;
+  if (iabs(r.n) < lim && r.d < lim) return (double)(long long)r.n / (double)(long long)r.d;  // one IEEE division: correctly rounded
+  return (double)((long double)r.n / (long double)r.d);
+}
+
+// ------------------------------------------------------- big integers (check)
+// Sign-magnitude, base 2^32, only what the exactness check needs.
+struct Big {
+  bool neg = false;
+  std::vector<uint32_t> w;   // little endian, no leading zeros
+  bool zero() const { return w.empty(); }
+};
+Big big_from(i128 v) {
+  Big b;
+  b.neg = v < 0;
+  u128 u = b.neg ? (u128)(-(v + 1)) + 1 : (u128)v;
+  while (u) { b.w.push_back((uint32_t)u); u >>= 32; }
+  return b;
+}
+void trim(Big& b) {
+  while (!b.w.empty() && b.w.back() == 0) b.w.pop_back();
+  if (b.w.empty()) b.neg = false;
+}
+int cmp_mag(const Big& a, const Big& b) {
+  if (a.w.size() != b.w.size()) return a.w.size() < b.w.size() ? -1 : 1;
+  for (size_t i = a.w.size(); i-- > 0;)
+    if (a.w[i] != b.w[i]) return a.w[i] < b.w[i] ? -1 : 1;
+  return 0;
+}
+Big add_mag(const Big& a, const Big& b) {
+  Big r;
+  uint64_t c = 0;
+  size_t n = std::max(a.w.size(), b.w.size());
+  for (size_t i = 0; i < n; ++i) {
+    uint64_t s = c + (i < a.w.size() ? a.w[i] : 0) + (i < b.w.size() ? b.w[i] : 0);
+    r.w.push_back((uint32_t)s);
+    c = s >> 32;
+  }
+  if (c) r.w.push_back((uint32_t)c);
+  return r;
+}
+Big sub_mag(const Big& a, const Big& b) {   // |a| >= |b|
+  Big r;
+  int64_t c = 0;
+  for (size_t i = 0; i < a.w.size(); ++i) {
+    int64_t s = (int64_t)a.w[i] - (i < b.w.size() ? b.w[i] : 0) + c;
+    c = 0;
+    if (s < 0) { s += ((int64_t)1 << 32); c = -1; }
+    r.w.push_back((uint32_t)s);
+  }
+  trim(r);
+  return r;
+}
+Big big_add(const Big& a, const Big& b) {
+  Big r;
+  if (a.neg == b.neg) { r = add_mag(a, b); r.neg = a.neg; }
+  else {
+    int c = cmp_mag(a, b);
+    if (c == 0) return Big();
+    if (c > 0) { r = sub_mag(a, b); r.neg = a.neg; }
+    else { r = sub_mag(b, a); r.neg = b.neg; }
+  }
+  trim(r);
+  return r;
+}
+Big big_mul(const Big& a, const Big& b) {
+  Big r;
+  if (a.zero() || b.zero()) return r;
+  r.w.assign(a.w.size() + b.w.size(), 0);
+  for (size_t i = 0; i < a.w.size(); ++i) {
+    uint64_t c = 0;
+    for (size_t j = 0; j < b.w.size(); ++j) {
+      uint64_t t = (uint64_t)a.w[i] * b.w[j] + r.w[i + j] + c;
+      r.w[i + j] = (uint32_t)t;
+      c = t >> 32;
+    }
+    size_t k = i + b.w.size();
+    while (c) { uint64_t t = (uint64_t)r.w[k] + c; r.w[k] = (uint32_t)t; c = t >> 32; ++k; }
+  }
+  r.neg = a.neg != b.neg;
+  trim(r);
+  return r;
+}
+
+// ------------------------------------------------------------ half rounding
+// double -> IEEE binary16 (round to nearest even) -> float, on the host.
+float round_through_half(double v) {
+  if (std::isnan(v)) return NAN;
+  double a = std::fabs(v);
+  float sign = std::signbit(v) ? -1.f : 1.f;
+  if (a >= 65520.0) return sign * INFINITY;            // halfway between 65504 and 2^16 rounds to inf
+  if (a == 0.0) return sign * 0.f;
+  int e;
+  std::frexp(a, &e);                                    // a = f * 2^e, f in [0.5, 1)
+  int exp2 = e - 1;                                     // a in [2^exp2, 2^(exp2+1))
+  if (exp2 < -14) exp2 = -14;                           // subnormal spacing 2^-24
+  double ulp = std::ldexp(1.0, exp2 - 10);
+  double q = std::nearbyint(a / ulp);                   // default rounding mode: to nearest even
+  return sign * (float)(q * ulp);
+}
+
+// ---------------------------------------------------------------- kappa_2
+// One-sided Jacobi SVD of a small square matrix; returns sigma_max/sigma_min.
+double cond2(std::vector<double> a, int n) {
+  for (int sweep = 0; sweep < 60; ++sweep) {
+    double off = 0;
+    for (int p = 0; p < n - 1; ++p)
+      for (int q = p + 1; q < n; ++q) {
+        double al = 0, be = 0, ga = 0;
+        for (int i = 0; i < n; ++i) {
+          al += a[i * n + p] * a[i * n + p];
+          be += a[i * n + q] * a[i * n + q];
+          ga += a[i * n + p] * a[i * n + q];
+        }
+        if (ga == 0) continue;
+        off = std::max(off, std::fabs(ga) / std::sqrt(al * be));
+        double zeta = (be - al) / (2 * ga);
+        double t = (zeta >= 0 ? 1.0 : -1.0) / (std::fabs(zeta) + std::sqrt(1 + zeta * zeta));
+        double c = 1 / std::sqrt(1 + t * t), s = c * t;
+        for (int i = 0; i < n; ++i) {
+          double x = a[i * n + p], y = a[i * n + q];
+          a[i * n + p] = c * x - s * y;
+          a[i * n + q] = s * x + c * y;
+        }
+      }
+    if (off < 1e-15) break;
+  }
+  double smax = 0, smin = INFINITY;
+  for (int j = 0; j < n; ++j) {
+    double s = 0;
+    for (int i = 0; i < n; ++i) s += a[i * n + j] * a[i * n + j];
+    s = std::sqrt(s);
+    smax = std::max(smax, s);
+    smin = std::min(smin, s);
+  }
+  return smax / smin;
+}
+
+}  // namespace
+
+extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int mode, int coef,
+                                nova_plan** out) {
+  if (out) *out = nullptr;
+  if (!points || !out) return NOVA_ERR_INVALID_ARG;
+  if (m != 2 && m != 4 && m != 6 && m != 8) return NOVA_ERR_INVALID_ARG;
+  if (r != 3) return NOVA_ERR_UNSUPPORTED;
+  if (n != m + r - 1) return NOVA_ERR_INVALID_ARG;
+  if (mode != NOVA_FP32 && mode != NOVA_FP16_F32ACC) return NOVA_ERR_INVALID_ARG;
+  if (coef != NOVA_COEF_ROUND_TO_MODE && coef != NOVA_COEF_FP32) return NOVA_ERR_INVALID_ARG;
+
+  int n_inf = 0;
+  for (int i = 0; i < n; ++i) {
+    if (points[i].den < 0) return NOVA_ERR_INVALID_ARG;
+    if (points[i].den == 0) ++n_inf;
+  }
+  if (n_inf == 0) return NOVA_ERR_NO_INFINITY;
+  if (n_inf > 1 || points[n - 1].den != 0) return NOVA_ERR_MULTIPLE_INFINITY;
+
+  Arith ar;
+  const int nf = n - 1;
+  Rat al[nova::kMaxN];
+  for (int i = 0; i < nf; ++i) al[i] = ar.norm(points[i].num, points[i].den);
+  for (int i = 0; i < nf; ++i)
+    for (int j = i + 1; j < nf; ++j)
+      if (al[i].n == al[j].n && al[i].d == al[j].d) return NOVA_ERR_DUPLICATE_POINT;
+
+  // Lagrange factors F_i = prod_{j != i} (alpha_i - alpha_j)
+  Rat F[nova::kMaxN];
+  for (int i = 0; i < nf; ++i) {
+    Rat f; f.n = 1; f.d = 1;
+    for (int j = 0; j < nf; ++j)
+      if (j != i) f = ar.mul(f, ar.sub(al[i], al[j]));
+    F[i] = f;
+  }
+  Rat zero, one; one.n = 1;
+  std::vector<Rat> AT(m * n, zero), G(n * r, zero), BT(n * n, zero);
+  for (int p = 0; p < nf; ++p) {
+    Rat pw = one;                                         // alpha_p^i, 0^0 = 1
+    for (int i = 0; i < std::max(m, r); ++i) {
+      if (i < m) AT[i * n + p] = pw;
+      if (i < r) G[p * r + i] = ar.div(pw, F[p]);
+      pw = ar.mul(pw, al[p]);
+    }
+  }
+  AT[(m - 1) * n + (n - 1)] = one;
+  G[(n - 1) * r + (r - 1)] = one;
+  for (int p = 0; p < n; ++p) {                           // row n-1: all finite roots
+    std::vector<Rat> poly(1, one);
+    for (int j = 0; j < nf; ++j) {
+      if (j == p) continue;
+      std::vector<Rat> nx(poly.size() + 1, zero);
+      for (size_t t = 0; t < poly.size(); ++t) {
+        nx[t + 1] = ar.plus(nx[t + 1], poly[t]);          // t * poly
+        nx[t] = ar.sub(nx[t], ar.mul(poly[t], al[j]));    // -= poly[t] * alpha_j
+      }
+      poly.swap(nx);
+    }
+    for (size_t t = 0; t < poly.size(); ++t) BT[p * n + t] = poly[t];
+  }
+  if (ar.bad) return NOVA_ERR_RATIONAL_OVERFLOW;
+
+  // Exact check: sum_p A^T[i][p] G[p][k] B^T[p][j] == [j == i + k]  (Section 2.4)
+  for (int i = 0; i < m; ++i)
+    for (int k = 0; k < r; ++k)
+      for (int j = 0; j < n; ++j) {
+        Big num, den = big_from(1);
+        for (int p = 0; p < n; ++p) {
+          const Rat &a = AT[i * n + p], &g = G[p * r + k], &b = BT[p * n + j];
+          if (a.n == 0 || g.n == 0 || b.n == 0) continue;
+          Big tn = big_mul(big_mul(big_from(a.n), big_from(g.n)), big_from(b.n));
+          Big td = big_mul(big_mul(big_from(a.d), big_from(g.d)), big_from(b.d));
+          num = big_add(big_mul(num, td), big_mul(tn, den));
+          den = big_mul(den, td);
+        }
+        if (j == i + k) { Big md = den; md.neg = !md.neg; num = big_add(num, md); }
+        if (!num.zero()) return NOVA_ERR_VERIFY_FAILED;
+      }
+
+  nova_plan* pl = new (std::nothrow) nova_plan();
+  if (!pl) return NOVA_ERR_INVALID_ARG;
+  std::memset(pl, 0, sizeof(*pl));
+  pl->m = m; pl->r = r; pl->n = n; pl->mode = mode; pl->coef = coef;
+  for (int i = 0; i < n; ++i) pl->points[i] = points[i];
+  for (int i = 0; i < m * n; ++i) pl->AT[i] = rat_to_double(AT[i]);
+  for (int i = 0; i < n * r; ++i) pl->G[i] = rat_to_double(G[i]);
+  for (int i = 0; i < n * n; ++i) pl->BT[i] = rat_to_double(BT[i]);
+
+  const bool through_half = (mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE);
+  auto rnd = [&](double v) { return through_half ? round_through_half(v) : (float)v; };
+  for (int i = 0; i < m; ++i)
+    for (int p = 0; p < n; ++p) pl->coefs.AT[i][p] = rnd(pl->AT[i * n + p]);
+  for (int p = 0; p < n; ++p)
+    for (int k = 0; k < r; ++k) pl->coefs.G[p][k] = rnd(pl->G[p * r + k]);
+  for (int p = 0; p < n; ++p)
+    for (int j = 0; j < n; ++j) pl->coefs.BT[p][j] = rnd(pl->BT[p * n + j]);
+
+  std::vector<double> V(nf * nf);
+  for (int i = 0; i < nf; ++i) {
+    double a = rat_to_double(al[i]), pw = 1.0;
+    for (int j = 0; j < nf; ++j) { V[i * nf + j] = pw; pw *= a; }
+  }
+  pl->kappa2_V = cond2(V, nf);
+
+  // One device status word, if a device is present (host-only use is allowed).
+  pl->status_dev = nullptr;
+  pl->device = -1;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+      int* w = nullptr;
+      if (cudaMalloc((void**)&w, sizeof(int)) == cudaSuccess) {
+        cudaMemset(w, 0, sizeof(int));
+        pl->status_dev = w;
+        pl->device = dev;
+      }
+    }
+  }
+  (void)cudaGetLastError();
+  *out = pl;
+  return NOVA_OK;
+}
+
+extern "C" void nova_plan_destroy(nova_plan* plan) {
+  if (!plan) return;
+  if (plan->status_dev) cudaFree(plan->status_dev);
+  delete plan;
+}
+
+extern "C" int nova_plan_get_matrices(const nova_plan* p, double* AT, double* G, double* BT) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  if (AT) std::memcpy(AT, p->AT, sizeof(double) * p->m * p->n);
+  if (G) std::memcpy(G, p->G, sizeof(double) * p->n * p->r);
+  if (BT) std::memcpy(BT, p->BT, sizeof(double) * p->n * p->n);
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_get_device_tables(const nova_plan* p, float* AT, float* G, float* BT) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  for (int i = 0; i < p->m; ++i)
+    for (int q = 0; q < p->n; ++q)
+      if (AT) AT[i * p->n + q] = p->coefs.AT[i][q];
+  for (int q = 0; q < p->n; ++q)
+    for (int k = 0; k < p->r; ++k)
+      if (G) G[q * p->r + k] = p->coefs.G[q][k];
+  for (int q = 0; q < p->n; ++q)
+    for (int j = 0; j < p->n; ++j)
+      if (BT) BT[q * p->n + j] = p->coefs.BT[q][j];
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_kappa(const nova_plan* p, double* k) {
+  if (!p || !k) return NOVA_ERR_INVALID_ARG;
+  *k = p->kappa2_V;
+  return NOVA_OK;
+}
+
+extern "C" const char* nova_status_string(int s) {
+  switch (s) {
+    case NOVA_OK: return "ok";
+    case NOVA_ERR_INVALID_ARG: return "invalid argument";
+    case NOVA_ERR_NO_INFINITY: return "point set has no point at infinity";
+    case NOVA_ERR_MULTIPLE_INFINITY: return "point at infinity must appear exactly once, last";
+    case NOVA_ERR_DUPLICATE_POINT: return "finite points must be distinct";
+    case NOVA_ERR_RATIONAL_OVERFLOW: return "exact rational arithmetic overflowed 127 bits";
+    case NOVA_ERR_VERIFY_FAILED: return "exact decomposition identity failed";
+    case NOVA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case NOVA_ERR_CUDA: return "CUDA call failed or no device";
+    case NOVA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case NOVA_ERR_WORKSPACE: return "workspace too small or misaligned";
+    default: return "unknown status";
+  }
+}
