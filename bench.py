@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the Winograd convolution hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg3|cfg4|cfg2] [--points nova|half|std] [--workspace-mb M]
+
+One "step" is one nova_conv2d_fwd call (input transform, transformed-domain
+product, output transform) over one synthetic batch of the workload, with the
+filter already transformed (as at inference time; that kernel is timed
+separately and reported as filter_transform_ms).  Prints ONE JSON line.
+With N > 1 (launched under torch.distributed.run) every rank runs its own batch
+(weak scaling, no data-path collective); the time is the max over ranks.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fp16 Winograd conv TFLOP/s (direct-equivalent)"
+UNIT = "TFLOP/s"
+
+
+def read_peaks():
+    """Measured peaks written by the driver, else the documented fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "tflops_burst": float(d["bf16_tflops"]),
+                "tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.samples, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for s in self.samples:
+            parts = [p.strip() for p in s.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                mhz.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nme, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(mhz)}
+
+
+def workload(name):
+    from synth import CONFIGS
+    return CONFIGS[name]
+
+
+def flops(c):
+    n = c.m + 2
+    th, tw = -(-c.H // c.m), -(-c.W // c.m)
+    P = c.N * th * tw
+    direct = 2.0 * c.N * c.H * c.W * c.K * c.C * 9
+    actual = 2.0 * n * n * c.K * c.C * P
+    min_bytes = 2.0 * c.N * c.H * c.W * (c.C + c.K) + 2.0 * n * n * c.K * c.C
+    return direct, actual, min_bytes, P
+
+
+def _host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return int(max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1]))
+    except Exception:
+        return int(os.cpu_count() or 1)
+
+
+def _oracle_sample(c, budget_s):
+    """Inputs for a bounded sample: as many images of the batch as fit `budget_s` seconds."""
+    from oracle import conv
+    from synth import make_conv_inputs
+    x, g = make_conv_inputs(1, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    conv.direct_conv_fp64(x, g)                      # page in BLAS
+    t0 = time.perf_counter()
+    conv.direct_conv_fp64(x, g)
+    t1 = time.perf_counter() - t0
+    n_img = int(max(1, min(c.N, budget_s / max(t1, 1e-4))))
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    return x, g, n_img
+
+
+def time_oracle(c, budget_s=20.0):
+    """The oracle's fp64 direct convolution (as it stands) on a bounded sample of the batch."""
+    from oracle import conv
+    x, g, n_img = _oracle_sample(c, budget_s / 3.0)
+    best = float("inf")
+    for _ in range(3):
+        t0 = time.perf_counter()
+        conv.direct_conv_fp64(x, g)
+        best = min(best, time.perf_counter() - t0)
+    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * 9
+    return {"value": fl / best / 1e12, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
+            "sample": "oracle.conv.direct_conv_fp64 (fp64, numpy) on %d of %d images of %s, best of 3"
+                      % (n_img, c.N, c.name)}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the same workload and metric.
+    Each step is one direct convolution of a bounded sample of the batch."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import conv
+    c = workload(args.workload)
+    x, g, n_img = _oracle_sample(c, min(6.0, 120.0 / (args.steps + args.warmup)))
+    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * 9
+    for _ in range(args.warmup):
+        conv.direct_conv_fp64(x, g)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        conv.direct_conv_fp64(x, g)
+    sec = (time.perf_counter() - t0) / args.steps
+    val = fl / sec / 1e12
+    sample = "oracle.conv.direct_conv_fp64 (fp64, numpy) on %d of %d images of %s per step" % (n_img, c.N, c.name)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s: F(%dx%d,3x3), N=%d C=%d K=%d H=W=%d; %s"
+                               % (c.name, c.m, c.m, c.N, c.C, c.K, c.H, sample)},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": _host_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import paper_2512_18453_b200 as nv
+    from synth import point_set, make_conv_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    c = workload(args.workload)
+    direct, actual, min_bytes, P = flops(c)
+    pts = point_set(args.points, c.m)
+    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC)
+    # each rank gets its own batch (weak scaling): seed offset by rank
+    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed + 100 * rank)
+    g = torch.from_numpy(g_np).cuda()
+    n_sets = 3
+    xs = [torch.from_numpy(x_np).cuda() if i == 0 else torch.from_numpy(np.roll(x_np, i, axis=0)).cuda()
+          for i in range(n_sets)]
+    ys = [torch.empty(c.N, c.H, c.W, c.K, dtype=torch.float16, device="cuda") for _ in range(n_sets)]
+    ws_bytes = plan.workspace_bytes(c.N, c.H, c.W, c.C, c.K) if args.workspace_mb is None \
+        else int(args.workspace_mb * (1 << 20))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    flags = {"auto": 0, "tcgen05": nv.GEMM_TCGEN05, "simt": nv.GEMM_SIMT}[args.gemm]
+    launches = plan.launch_count(c.N, c.H, c.W, c.C, c.K, ws_bytes, flags)
+
+    # S1, once per layer: timed on its own
+    U = plan.filter_transform(g)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        U = plan.filter_transform(g)
+    e1.record()
+    torch.cuda.synchronize()
+    filter_ms = e0.elapsed_time(e1) / 5
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        plan.conv2d(xs[i % n_sets], U, y=ys[i % n_sets], workspace=ws, flags=flags)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        plan.conv2d(xs[i % n_sets], U, y=ys[i % n_sets], workspace=ws, flags=flags)
+    e1.record()
+    barrier()
+    total_ms = max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = total_ms / args.steps
+    status = plan.device_status()
+
+    # ---- per-kernel durations (events around each kernel, same steps, separate pass)
+    kms = [0.0, 0.0, 0.0]
+    prof_steps = min(args.steps, 20)
+    for i in range(prof_steps):
+        t = plan.conv2d_timed(xs[i % n_sets], U, ys[i % n_sets], ws, flags=flags)
+        kms = [a + b for a, b in zip(kms, t)]
+    kms = [v / prof_steps for v in kms]
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end: host buffers in and out through the C ABI
+    xh = torch.from_numpy(x_np).pin_memory()
+    yh = torch.empty(c.N, c.H, c.W, c.K, dtype=torch.float16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        plan.conv2d_host(xh, U, yh, xs[0], ys[0], ws, flags=flags)
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        plan.conv2d_host(xh, U, yh, xs[i % n_sets], ys[i % n_sets], ws, flags=flags)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = read_peaks()
+    chunks = launches // 3
+    names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
+    n2 = (c.m + 2) ** 2
+    elt = 2
+    # algorithmic bytes / flops per step of each kernel class ("Kernels")
+    alg = [
+        ("hbm", 2.0 * c.N * c.H * c.W * c.C + elt * n2 * P * c.C),        # read x, write V
+        ("tensor", actual),                                                # 2 n^2 K C P flop
+        ("hbm", 4.0 * n2 * P * c.K + 2.0 * c.N * c.H * c.W * c.K),         # read M, write y
+    ]
+    dom = max(range(3), key=lambda i: kms[i])
+    bound, work = alg[dom]
+    dur_launch = kms[dom] * 1e-3 / chunks
+    if bound == "tensor":
+        achieved, peak, runit = work / chunks / dur_launch / 1e12, peaks["tflops_burst"], "TFLOP/s"
+    else:
+        achieved, peak, runit = work / chunks / dur_launch / 1e9, peaks["hbm_gbs"], "GB/s"
+    roof_s = max(actual / (peaks["tflops_burst"] * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
+    value = world * direct / (ms_per_step * 1e-3) / 1e12
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 (f32 accumulate)", "data": "synthetic",
+        "config": {
+            "workload": "%s: F(%dx%d,3x3) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
+                        % (c.name, c.m, c.m, args.points, c.N, c.C, c.K, c.H),
+            "step": "nova_conv2d_fwd (input transform, tcgen05 product, output transform); filter transform once per layer",
+            "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 126 MB L2)" % (n_sets, n_sets * (x_np.nbytes + ys[0].numel() * 2) / 1e6),
+            "workspace_mb": ws_bytes / (1 << 20), "chunks": chunks, "gemm": args.gemm,
+        },
+        "tflops_actual": world * actual / (ms_per_step * 1e-3) / 1e12,
+        "path_roofline": {"roofline_us": roof_s * 1e6, "achieved_us": ms_per_step * 1e3,
+                          "frac": roof_s / (ms_per_step * 1e-3), "peaks": peaks["source"],
+                          "tensor_us": actual / (peaks["tflops_burst"] * 1e12) * 1e6,
+                          "hbm_us": min_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
+        "kernels_ms_per_step": dict(zip(names, kms)),
+        "filter_transform_ms": filter_ms,
+        "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
+                     "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
+                     "launch_us": dur_launch * 1e6},
+        "e2e": {"value": world * direct / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(x_np.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)},
+        "gpu_launches": launches * args.steps,
+        "device_status": status,
+        "kappa2_V": plan.kappa(),
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = time_oracle(c)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--points", default="nova")
+    ap.add_argument("--gemm", default="auto", choices=["auto", "tcgen05", "simt"])
+    ap.add_argument("--workspace-mb", type=float, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,17 @@ int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev,
                     void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream);
 
 /*
+ * Measurement aid: the same work as nova_conv2d_fwd with CUDA events recorded
+ * on `stream` around each kernel; synchronises the stream and writes the summed
+ * device time in milliseconds of the three kernel classes to kernel_ms_host[0..2]
+ * (input transform, transformed-domain product, output transform).
+ */
+int nova_conv2d_fwd_timed(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
+                          int N, int H, int W, int C, int K,
+                          void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream,
+                          float* kernel_ms_host);
+
+/*
  * The same call for host tensors: copies x_host to x_stage_dev, runs
  * nova_conv2d_fwd, copies the result to y_host, all on `stream`.  The staging
  * buffers are device memory of the sizes of x and y.  Host buffers should be

@@ -15,7 +15,7 @@ EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
-    "nova_conv2d_fwd_host", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
+    "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
     "nova_status_string",
 )
 
@@ -62,6 +62,8 @@ def lib():
         getattr(L, name).restype = sz
     L.nova_conv2d_fwd.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, sz, i, vp]
     L.nova_conv2d_fwd.restype = i
+    L.nova_conv2d_fwd_timed.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, sz, i, vp, fp]
+    L.nova_conv2d_fwd_timed.restype = i
     L.nova_conv2d_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, vp, sz, i, vp]
     L.nova_conv2d_fwd_host.restype = i
     L.nova_conv2d_launch_count.argtypes = [vp, i, i, i, i, i, sz, i]
@@ -180,6 +182,16 @@ class Plan:
                                      workspace.data_ptr(), workspace.numel(), flags, _stream()),
                "nova_conv2d_fwd")
         return y
+
+    def conv2d_timed(self, x, U, y, workspace, flags=0):
+        """Synchronous; returns (input, product, output) kernel milliseconds."""
+        N, H, W, C = x.shape
+        K = U.shape[1]
+        ms = (ctypes.c_float * 3)()
+        _check(lib().nova_conv2d_fwd_timed(self._h, x.data_ptr(), U.data_ptr(), y.data_ptr(), N, H, W, C, K,
+                                           workspace.data_ptr(), workspace.numel(), flags, _stream(), ms),
+               "nova_conv2d_fwd_timed")
+        return tuple(ms)
 
     def conv2d_host(self, x_host, U, y_host, x_stage, y_stage, workspace, flags=0):
         """Host tensors in and out (pinned for asynchronous copies)."""

@@ -97,9 +97,11 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
   return 3 * c.chunks;
 }
 
-extern "C" int nova_conv2d_fwd(const nova_plan* p, const void* x, const void* U, void* y, int N, int H,
-                               int W, int C, int K, void* ws, size_t ws_bytes, int flags,
-                               nova_stream stream) {
+namespace {
+// Shared body of nova_conv2d_fwd and nova_conv2d_fwd_timed.  With `ev` non-null,
+// four events per chunk bracket the three kernels.
+int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, int N, int H, int W, int C,
+                    int K, void* ws, size_t ws_bytes, int flags, nova_stream stream, cudaEvent_t* ev) {
   if (!p || !aligned16(x) || !aligned16(U) || !aligned16(y) || !shape_ok(N, H, W, C, K))
     return NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
@@ -112,16 +114,53 @@ extern "C" int nova_conv2d_fwd(const nova_plan* p, const void* x, const void* U,
   char* Vb = static_cast<char*>(ws);
   float* Mb = reinterpret_cast<float*>(Vb + c.v_bytes);
   const int nfreq = g.n * g.n;
-  for (long long p0 = 0; p0 < g.P; p0 += c.pc) {
+  cudaStream_t s = (cudaStream_t)stream;
+  int ci = 0;
+  for (long long p0 = 0; p0 < g.P; p0 += c.pc, ++ci) {
     const int pc = (int)((g.P - p0) < c.pc ? (g.P - p0) : c.pc);
+    if (ev) cudaEventRecord(ev[4 * ci + 0], s);
     if (launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream)) return NOVA_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[4 * ci + 1], s);
     const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream)
                      : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);
     if (e) return NOVA_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[4 * ci + 2], s);
     if (launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, (flags & NOVA_RELU) ? 1 : 0, stream))
       return NOVA_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[4 * ci + 3], s);
   }
   return NOVA_OK;
+}
+}  // namespace
+
+extern "C" int nova_conv2d_fwd(const nova_plan* p, const void* x, const void* U, void* y, int N, int H,
+                               int W, int C, int K, void* ws, size_t ws_bytes, int flags,
+                               nova_stream stream) {
+  return conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, nullptr);
+}
+
+extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const void* U, void* y, int N,
+                                     int H, int W, int C, int K, void* ws, size_t ws_bytes, int flags,
+                                     nova_stream stream, float* kernel_ms) {
+  if (!kernel_ms) return NOVA_ERR_INVALID_ARG;
+  const int launches = nova_conv2d_launch_count(p, N, H, W, C, K, ws_bytes, flags);
+  if (launches < 0) return launches;
+  const int chunks = launches / 3;
+  cudaEvent_t* ev = new cudaEvent_t[4 * chunks];
+  for (int i = 0; i < 4 * chunks; ++i) cudaEventCreate(&ev[i]);
+  int st = conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, ev);
+  if (st == NOVA_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st = NOVA_ERR_CUDA;
+  kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
+  if (st == NOVA_OK)
+    for (int c = 0; c < chunks; ++c)
+      for (int k = 0; k < 3; ++k) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, ev[4 * c + k], ev[4 * c + k + 1]);
+        kernel_ms[k] += ms;
+      }
+  for (int i = 0; i < 4 * chunks; ++i) cudaEventDestroy(ev[i]);
+  delete[] ev;
+  return st;
 }
 
 extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, const void* U, void* y_host,
