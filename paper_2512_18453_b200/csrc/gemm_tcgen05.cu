@@ -9,8 +9,9 @@
 //   warp 1    issues tcgen05.mma (kind::f16, M=128, N=BLOCK_N, K=16) from
 //             shared-memory descriptors into one of two TMEM accumulators;
 //   warps 2-5 epilogue: tcgen05.ld the finished accumulator (one TMEM lane
-//             quadrant per warp) and store float rows of M, overlapping the
-//             next item's MMAs on the other accumulator.
+//             quadrant per warp), stage it in swizzled shared memory and TMA-
+//             store float boxes of M, overlapping the next item's MMAs on the
+//             other accumulator.
 // Every wait is bounded; on expiry the kernel records a status and drains.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -70,6 +71,18 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       : "memory");
 }
 
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // Shared-memory matrix descriptor for a K-major operand tile stored as
 // [rows][64 halves] with the 128-byte swizzle: 8-row groups are 1024 bytes
 // apart (stride byte offset), descriptor version 1, layout type 2.
@@ -120,14 +133,16 @@ struct SmemLayout {
   static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
   static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBarrierOffset = kStages * kStageBytes;
-  static constexpr int kTotal = kBarrierOffset + 256 + 1024;   // barriers + alignment slack
+  static constexpr int kOutOffset = kStages * kStageBytes;        // epilogue staging
+  static constexpr int kOutBytesPerWarp = 2 * 32 * 128;           // two [32 rows][32 floats] boxes
+  static constexpr int kBarrierOffset = kOutOffset + 4 * kOutBytesPerWarp;
+  static constexpr int kTotal = kBarrierOffset + 256 + 1024;     // barriers + alignment slack
 };
 
 template <int BLOCK_N>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
-                    float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
+                    const __grid_constant__ CUtensorMap tmM, int nfreq, int pc, int C, int K,
                     int* __restrict__ status) {
   using L = SmemLayout<BLOCK_N>;
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
@@ -215,9 +230,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       }
     }
   } else {
-    // ---------------- epilogue (warps 2..5); a warp may only read TMEM lanes 32*(warp%4)..+31
+    // ---------------- epilogue (warps 2..5); a warp may only read TMEM lanes 32*(warp%4)..+31.
+    // Each warp moves its 32 rows in [32 rows][32 floats] boxes: TMEM -> registers ->
+    // 128B-swizzled shared memory -> TMA store (which clips rows >= pc and columns >= K).
     const int quad = warp & 3;
-    uint32_t local = 0;
+    uint8_t* stage_out = smem + L::kOutOffset + (warp - 2) * L::kOutBytesPerWarp;
+    uint32_t local = 0, nbox = 0;
     for (long long it = blockIdx.x; it < num_items && !timed_out; it += gridDim.x, ++local) {
       const int kb = (int)(it % num_kb);
       const int pb = (int)((it / num_kb) % num_pb);
@@ -225,27 +243,33 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
       if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int row = pb * BLOCK_M + quad * 32 + lane;
-      float* out_row = Mo + ((size_t)f * pc_pad + row) * K + (size_t)kb * BLOCK_N;
+      const int row0 = pb * BLOCK_M + quad * 32;
       const int k_left = K - kb * BLOCK_N;
 #pragma unroll 1
-      for (int cb = 0; cb < BLOCK_N; cb += 32) {
+      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32, ++nbox) {
+        uint8_t* buf = stage_out + (nbox & 1) * (32 * 128);
+        if (lane == 0) bulk_wait_read<1>();          // the store that last read this buffer is done
+        __syncwarp();
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + cb, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < pc) {
+        uint8_t* my_row = buf + lane * 128;
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            if (cb + j + 3 < k_left)
-              *reinterpret_cast<float4*>(out_row + cb + j) =
-                  make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                              __uint_as_float(r[j + 3]));
+        for (int j = 0; j < 8; ++j)                  // 16-byte chunk j of row `lane` lives at chunk j ^ (lane & 7)
+          *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) =
+              make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < pc) tma_store_3d(&tmM, buf, kb * BLOCK_N + cb, row0, f);
+          bulk_commit();   // one group per box, stored or not, so "at most one pending" always means the other buffer
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
     }
+    if (lane == 0) bulk_wait_all();
   }
 
   if (timed_out) {
@@ -280,17 +304,18 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// [nfreq][rows (stride row_stride)][C] halves; box = [1][box_rows][64].
-bool make_operand_map(CUtensorMap* map, const void* base, int C, int rows, long long freq_stride_elems,
-                      int nfreq, int box_rows) {
+// [nfreq][rows][inner] elements of `esize` bytes, frequency stride in elements;
+// box = [1][box_rows][box_inner], 128-byte swizzle (box_inner * esize == 128).
+bool make_map_3d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base, int inner, int rows,
+                 long long freq_stride_elems, int nfreq, int box_inner, int box_rows) {
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)rows, (cuuint64_t)nfreq};
-  cuuint64_t strides[2] = {(cuuint64_t)C * 2, (cuuint64_t)freq_stride_elems * 2};
-  cuuint32_t box[3] = {(cuuint32_t)BLOCK_K, (cuuint32_t)box_rows, 1};
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)nfreq};
+  cuuint64_t strides[2] = {(cuuint64_t)inner * esize, (cuuint64_t)freq_stride_elems * esize};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  return enc(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -305,16 +330,18 @@ int launch_n(const void* V, const void* U, float* M, int nfreq, int pc, int pc_p
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
-  CUtensorMap tmV, tmU;
-  if (!make_operand_map(&tmV, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_M)) return (int)cudaErrorUnknown;
-  if (!make_operand_map(&tmU, U, C, K, (long long)K * C, nfreq, BLOCK_N)) return (int)cudaErrorUnknown;
+  CUtensorMap tmV, tmU, tmM;
+  const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  if (!make_map_3d(&tmV, f16, 2, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
+      !make_map_3d(&tmU, f16, 2, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N) ||
+      !make_map_3d(&tmM, f32, 4, M, K, pc, (long long)pc_pad * K, nfreq, 32, 32))
+    return (int)cudaErrorUnknown;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const long long items = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M) * ((K + BLOCK_N - 1) / BLOCK_N);
   const int grid = (int)(items < sms ? items : sms);
-  gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K,
-                                                                      status);
+  gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, tmM, nfreq, pc, C, K, status);
   return (int)cudaGetLastError();
 }
 

@@ -144,6 +144,19 @@ def test_tcgen05_and_simt_products_agree_elementwise(m):
     assert (d > 0).mean() < 0.25
 
 
+def test_ragged_last_row_block_after_full_blocks():
+    """532 tiles = 4 full 128-row blocks + 20 rows, 36 x 5 work items on 148 SMs: a CTA
+    that handles a full block and then the ragged one must not reuse an epilogue
+    staging buffer that a pending store still reads (short items, C = 8)."""
+    x, g = make_conv_inputs(1, 76, 112, 8, 64, "fp16", True, True, seed=405)
+    pts = point_set("nova", 4)
+    yb, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC, nv.GEMM_SIMT)
+    for _ in range(3):
+        ya, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC, nv.GEMM_TCGEN05)
+        d = np.abs(ya.astype(np.float32) - yb.astype(np.float32))
+        assert d.max() <= 4 * 2.0 ** -10 * np.abs(yb.astype(np.float32)).max()
+
+
 def test_gpu_is_close_to_emulation_elementwise():
     x, g = make_conv_inputs(2, 24, 24, 64, 64, "fp16", True, True, seed=410)
     pts = point_set("nova", 4)
