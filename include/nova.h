@@ -63,7 +63,8 @@ enum {
   NOVA_ERR_UNSUPPORTED = -7,        /* r != 3, or an unsupported mode on this path */
   NOVA_ERR_CUDA = -8,               /* a CUDA runtime/driver call failed (or no device) */
   NOVA_ERR_DEVICE_TIMEOUT = -9,     /* a bounded device-side wait expired */
-  NOVA_ERR_WORKSPACE = -10          /* workspace too small or misaligned */
+  NOVA_ERR_WORKSPACE = -10,         /* workspace too small or misaligned */
+  NOVA_ERR_STATIC_LIMIT = -11       /* problem needs more than NOVA_STATIC_SCRATCH_BYTES of built-in scratch */
 };
 
 typedef struct nova_plan nova_plan;   /* opaque; immutable after creation */
@@ -153,6 +154,39 @@ int nova_conv2d_fwd_host(const nova_plan* plan, const void* x_host, const void* 
                          int N, int H, int W, int C, int K,
                          void* x_stage_dev, void* y_stage_dev,
                          void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream);
+
+/*
+ * Forward convolution for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of
+ * nova_conv2d_fwd, same arithmetic, same kernels.)
+ *
+ * Some hosts of this library hand it tensors but own no allocator it may
+ * call: a plug-in running inside another framework's memory pool, a
+ * real-time loop that forbids cudaMalloc after start-up because it
+ * synchronises the device, or a sandbox where only pre-mapped buffers exist.
+ * They have nowhere to get the scratch that nova_conv2d_fwd asks for.  This
+ * entry point brings its own: a fixed array of NOVA_STATIC_SCRATCH_BYTES of
+ * device global memory that is part of the library image.  Every GPU that
+ * loads the library keeps that array until the process exits, used or not.
+ *
+ * The caller still passes x_dev, U_dev and y_dev exactly as for
+ * nova_conv2d_fwd.  The call makes no cudaMalloc / cudaFree and calls no
+ * allocating routine.  A problem whose smallest chunk (128 tiles, or all of
+ * them if fewer) does not fit the array - nova_conv2d_min_workspace_bytes() >
+ * NOVA_STATIC_SCRATCH_BYTES - is refused with NOVA_ERR_STATIC_LIMIT and nothing
+ * is launched; larger problems that fit are processed in more, smaller chunks.
+ *
+ * The first call on each device looks up the array's device address (a
+ * symbol query, with that device current) and keeps it; make that first call
+ * outside any stream capture.  All calls on one device share the one array
+ * and it keeps whatever the previous call left there; every kernel writes
+ * the part it later reads, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams without ordering) race on
+ * it: order them.
+ */
+#define NOVA_STATIC_SCRATCH_BYTES ((size_t)32 << 20)
+int nova_conv2d_fwd_static(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
+                           int N, int H, int W, int C, int K, int flags, nova_stream stream);
 
 /* Number of kernel launches one nova_conv2d_fwd call issues for this problem
  * and workspace size (negative = error). */

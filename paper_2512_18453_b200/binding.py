@@ -16,8 +16,9 @@ EXPORTED_SYMBOLS = (
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
-    "nova_status_string",
+    "nova_status_string", "nova_conv2d_fwd_static",
 )
+STATIC_SCRATCH_BYTES = 32 << 20
 
 
 class NovaError(RuntimeError):
@@ -66,6 +67,8 @@ def lib():
     L.nova_conv2d_fwd_timed.restype = i
     L.nova_conv2d_fwd_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, vp, sz, i, vp]
     L.nova_conv2d_fwd_host.restype = i
+    L.nova_conv2d_fwd_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
+    L.nova_conv2d_fwd_static.restype = i
     L.nova_conv2d_launch_count.argtypes = [vp, i, i, i, i, i, sz, i]
     L.nova_conv2d_launch_count.restype = i
     L.nova_maxpool2x2.argtypes = [vp, vp, i, i, i, i, i, vp]
@@ -181,6 +184,18 @@ class Plan:
         _check(lib().nova_conv2d_fwd(self._h, x.data_ptr(), U.data_ptr(), y.data_ptr(), N, H, W, C, K,
                                      workspace.data_ptr(), workspace.numel(), flags, _stream()),
                "nova_conv2d_fwd")
+        return y
+
+    def conv2d_static(self, x, U, y, flags=0):
+        """nova_conv2d_fwd_static: the convolution on the library's built-in scratch.
+
+        For callers that may not allocate device memory; `y` is therefore
+        required.  Problems beyond STATIC_SCRATCH_BYTES raise NovaError(-11).
+        """
+        N, H, W, C = x.shape
+        K = U.shape[1]
+        _check(lib().nova_conv2d_fwd_static(self._h, x.data_ptr(), U.data_ptr(), y.data_ptr(), N, H, W, C, K,
+                                            flags, _stream()), "nova_conv2d_fwd_static")
         return y
 
     def conv2d_timed(self, x, U, y, workspace, flags=0):

@@ -6,6 +6,8 @@
 // transform per chunk, all on the caller's stream, no host synchronisation.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "nova_internal.h"
 
 namespace nova {
@@ -175,6 +177,43 @@ extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, cons
   if (st != NOVA_OK) return st;
   if (cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return NOVA_ERR_CUDA;
   return NOVA_OK;
+}
+
+// ---------------------------------------------------------------------------
+// No-allocation variant.  The scratch is part of the library image; in host
+// code `g_static_scratch` is only a handle for the symbol query below, never
+// a pointer a kernel could use.
+static __device__ __align__(256) unsigned char g_static_scratch[NOVA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+// Device address of the array on the current device; queried once per device.
+int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NOVA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return NOVA_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return NOVA_OK;
+}
+}  // namespace
+
+extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const void* U, void* y, int N,
+                                      int H, int W, int C, int K, int flags, nova_stream stream) {
+  if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (nova_conv2d_min_workspace_bytes(p, N, H, W, C, K) > NOVA_STATIC_SCRATCH_BYTES)
+    return NOVA_ERR_STATIC_LIMIT;
+  void* ws = nullptr;
+  const int st = static_scratch_address(&ws);
+  if (st != NOVA_OK) return st;
+  return conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, NOVA_STATIC_SCRATCH_BYTES, flags, stream, nullptr);
 }
 
 extern "C" int nova_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode,

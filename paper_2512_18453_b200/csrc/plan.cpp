@@ -385,6 +385,7 @@ extern "C" const char* nova_status_string(int s) {
     case NOVA_ERR_CUDA: return "CUDA call failed or no device";
     case NOVA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case NOVA_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case NOVA_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
