@@ -49,7 +49,9 @@ enum { NOVA_COEF_ROUND_TO_MODE = 0, NOVA_COEF_FP32 = 1 };
 enum {
   NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
   NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
-  NOVA_GEMM_TCGEN05 = 2 << 8 /* force the tcgen05 tensor-core product kernel */
+  NOVA_GEMM_TCGEN05 = 2 << 8, /* force the tcgen05 tensor-core product kernel */
+  NOVA_TRANSFORM_SIMT = 1 << 10 /* evaluate the input transform on CUDA cores even where the
+                                   tensor-core formulation applies (testing) */
 };
 
 enum {
@@ -93,6 +95,15 @@ int nova_plan_get_matrices(const nova_plan* plan, double* AT_host, double* G_hos
 /* The tables as the kernels use them (after rounding to the coefficient
  * precision), as float, same shapes. */
 int nova_plan_get_device_tables(const nova_plan* plan, float* AT_host, float* G_host, float* BT_host);
+
+/* The library indexes the n*n transformed-domain coordinates ("frequencies") of U in an
+ * internal point order: frequency (xi, nu) of U is the pair of caller points
+ * (perm_host[xi], perm_host[nu]).  For a set that is symmetric about 0 ({0, +-a_1, ..,
+ * +-a_q, infinity}, as every set in the paper is) the internal order is 0, +a_1, -a_1, ..,
+ * infinity and *symmetric_host is 1: the transforms then share the even/odd partial sums
+ * of each +-pair and skip the structural zeros (Appendix A, "symmetric point sets").
+ * Any other set keeps the caller's order and dense transforms.  Either pointer may be null. */
+int nova_plan_frequency_order(const nova_plan* plan, int* perm_host, int* symmetric_host);
 
 /* kappa_2 = sigma_max/sigma_min of the Vandermonde matrix V_ij = a_i^j over the
  * n-1 finite points only (Section 2.2, "Vandermonde Conditioning"). */

@@ -10,13 +10,14 @@ COEF_ROUND_TO_MODE, COEF_FP32 = 0, 1
 RELU = 1
 GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
+TRANSFORM_SIMT = 1 << 10
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
-    "nova_status_string", "nova_conv2d_fwd_static",
+    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order",
 )
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -52,6 +53,8 @@ def lib():
     L.nova_plan_get_matrices.restype = i
     L.nova_plan_get_device_tables.argtypes = [vp, fp, fp, fp]
     L.nova_plan_get_device_tables.restype = i
+    L.nova_plan_frequency_order.argtypes = [vp, ctypes.POINTER(i), ctypes.POINTER(i)]
+    L.nova_plan_frequency_order.restype = i
     L.nova_plan_kappa.argtypes = [vp, dp]
     L.nova_plan_kappa.restype = i
     L.nova_filter_transform_bytes.argtypes = [vp, i, i]
@@ -142,6 +145,13 @@ class Plan:
         _check(lib().nova_plan_get_device_tables(self._h, AT.ctypes.data_as(fp), G.ctypes.data_as(fp),
                                                  BT.ctypes.data_as(fp)), "nova_plan_get_device_tables")
         return AT, G, BT
+
+    def frequency_order(self):
+        """(perm, symmetric): internal point i is the caller's point perm[i]."""
+        perm = (ctypes.c_int * self.n)()
+        sym = ctypes.c_int()
+        _check(lib().nova_plan_frequency_order(self._h, perm, ctypes.byref(sym)), "nova_plan_frequency_order")
+        return list(perm), bool(sym.value)
 
     def kappa(self):
         k = ctypes.c_double()

@@ -27,17 +27,18 @@ struct Chunking {
 size_t per_tile_bytes(const nova_plan* p, const Geom& g) {
   return (size_t)g.n * g.n * ((size_t)g.C * elt_bytes(p->mode) + (size_t)g.K * 4);
 }
+inline long long round_up_ll(long long v, long long a) { return (v + a - 1) / a * a; }
 
-// Largest chunk (a multiple of 128 tiles when possible) that fits `bytes`.
+// Largest chunk, a whole number of 128-tile row blocks, that fits `bytes`.  The scratch rows
+// are padded to that multiple: the product kernel writes whole row blocks of M.
 bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* c) {
   const size_t pt = per_tile_bytes(p, g);
-  if (bytes < 2 * kAlign + pt) return false;
-  long long pc = (long long)((bytes - 2 * kAlign) / pt);
-  if (pc >= g.P) pc = g.P;
-  else if (pc >= 128) pc = pc / 128 * 128;
-  else if (pc >= 8) pc = pc / 8 * 8;
-  if (pc < 1) return false;
-  c->pc = (int)pc;
+  if (bytes < 2 * kAlign + 128 * pt) return false;
+  long long pc = (long long)((bytes - 2 * kAlign) / pt) / 128 * 128;
+  const long long p_pad = round_up_ll(g.P, 128);
+  if (pc > p_pad) pc = p_pad;
+  if (pc < 128) return false;
+  c->pc = (int)(pc < g.P ? pc : g.P);
   c->pc_pad = (int)pc;
   c->chunks = (int)((g.P + pc - 1) / pc);
   c->v_bytes = round_up((size_t)g.n * g.n * c->pc_pad * g.C * elt_bytes(p->mode), kAlign);
@@ -75,8 +76,7 @@ extern "C" int nova_filter_transform(const nova_plan* p, const void* g, int K, i
 extern "C" size_t nova_conv2d_min_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
   if (!p || !shape_ok(N, H, W, C, K)) return 0;
   Geom g = make_geom(p, N, H, W, C, K);
-  const long long pc = g.P < 128 ? g.P : 128;
-  return (size_t)pc * per_tile_bytes(p, g) + 4 * kAlign;
+  return (size_t)128 * per_tile_bytes(p, g) + 4 * kAlign;
 }
 
 extern "C" size_t nova_conv2d_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
@@ -85,7 +85,7 @@ extern "C" size_t nova_conv2d_workspace_bytes(const nova_plan* p, int N, int H, 
   const size_t pt = per_tile_bytes(p, g);
   long long pc = (long long)(kTargetChunkBytes / pt) / 128 * 128;
   if (pc < 128) pc = 128;
-  if (pc > g.P) pc = g.P;
+  if (pc > round_up_ll(g.P, 128)) pc = round_up_ll(g.P, 128);
   return (size_t)pc * pt + 4 * kAlign;
 }
 
@@ -121,7 +121,10 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   for (long long p0 = 0; p0 < g.P; p0 += c.pc, ++ci) {
     const int pc = (int)((g.P - p0) < c.pc ? (g.P - p0) : c.pc);
     if (ev) cudaEventRecord(ev[4 * ci + 0], s);
-    if (launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream)) return NOVA_ERR_CUDA;
+    const bool tc_in = tc && p->kron_dev && C >= 64 && !(flags & NOVA_TRANSFORM_SIMT);
+    if (tc_in ? launch_input_transform_tc(p, g, x, Vb, p0, pc, c.pc_pad, stream)
+              : launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream))
+      return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 1], s);
     const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream)
                      : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);

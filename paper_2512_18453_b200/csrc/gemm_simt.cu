@@ -1,6 +1,7 @@
 // Transformed-domain product on CUDA cores (Section 2.1 step 3, summed over
 // input channels): for every frequency f,
-//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c]   (float accumulation).
+//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c]   (float accumulation),
+// stored as [f][K/4][pc_pad][4] like the tensor-core kernel's output.
 // This is the product kernel of the fp32 mode (a single-pass TF32 tensor-core
 // product cannot meet a 1e-5 tolerance) and a cross-check for the tcgen05
 // kernel in fp16 mode.
@@ -28,7 +29,7 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
   const int pb = blockIdx.x * BM, kb = blockIdx.y * BN;
   const T* Vf = V + (size_t)f * pc_pad * C;
   const T* Uf = U + (size_t)f * K * C;
-  float* Mf = Mo + (size_t)f * pc_pad * K;
+  float* Mf = Mo + (size_t)f * pc_pad * K;             // [K/4][pc_pad][4]
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;           // tx -> k, ty -> p
   const int lr = tid >> 2, lc = (tid & 3) * 4;      // loader: row 0..63, 4 channels at lc
@@ -60,14 +61,10 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
   for (int i = 0; i < 4; ++i) {
     const int p = pb + ty * 4 + i;
     if (p >= pc) continue;
-    const int k = kb + tx * 4;
-    if (k + 3 < K) {
-      *reinterpret_cast<float4*>(Mf + (size_t)p * K + k) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (k + j < K) Mf[(size_t)p * K + k + j] = acc[i][j];
-    }
+    const int k = kb + tx * 4;                        // K % 8 == 0: a filter quad is all in or all out
+    if (k < K)
+      *reinterpret_cast<float4*>(Mf + ((size_t)(k >> 2) * pc_pad + p) * 4) =
+          make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
   }
 }
 

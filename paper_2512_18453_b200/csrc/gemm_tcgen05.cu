@@ -9,140 +9,42 @@
 //   warp 1    issues tcgen05.mma (kind::f16, M=128, N=BLOCK_N, K=16) from
 //             shared-memory descriptors into one of two TMEM accumulators;
 //   warps 2-5 epilogue: tcgen05.ld the finished accumulator (one TMEM lane
-//             quadrant per warp), stage it in swizzled shared memory and TMA-
-//             store float boxes of M, overlapping the next item's MMAs on the
-//             other accumulator.
+//             quadrant per warp; a lane is a tile, a column a filter) and
+//             store it straight from registers, overlapping the next item's
+//             MMAs on the other accumulator.  M is laid out
+//             [f][K/4][pc_pad][4]: each 16-byte store instruction of a warp
+//             then covers 512 contiguous bytes (32 tiles x 4 filters).
 // Every wait is bounded; on expiry the kernel records a status and drains.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include "nova_internal.h"
+#include "sm100.cuh"
 
 namespace nova {
 namespace {
+using namespace sm100;
 
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;            // 64 halves = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kStages = 4;
 constexpr int kThreads = 192;
-constexpr uint32_t kSpinLimit = 1u << 24;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the limit is hit or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-    if (mbar_test(bar, parity)) return true;
-    if ((spin & 63u) == 63u && *abort_flag) return false;
-  }
-  return false;
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x,
-                                            int y, int z) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int x, int y, int z) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
-               ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-// Shared-memory matrix descriptor for a K-major operand tile stored as
-// [rows][64 halves] with the 128-byte swizzle: 8-row groups are 1024 bytes
-// apart (stride byte offset), descriptor version 1, layout type 2.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                 // leading byte offset: unused for swizzled K-major
-  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
-  d |= (uint64_t)1 << 46;                 // descriptor version (sm_100)
-  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
-  return d;
-}
-// Instruction descriptor, kind::f16: D float, A and B half, both K-major.
-__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N) {
-  return (1u << 4) | (0u << 7) | (0u << 10) | (0u << 15) | (0u << 16) | ((uint32_t)(N >> 3) << 17) |
-         ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                         uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                   smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
 
 template <int BLOCK_N>
 struct SmemLayout {
   static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
   static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kOutOffset = kStages * kStageBytes;        // epilogue staging
-  static constexpr int kOutBytesPerWarp = 2 * 32 * 128;           // two [32 rows][32 floats] boxes
-  static constexpr int kBarrierOffset = kOutOffset + 4 * kOutBytesPerWarp;
+  static constexpr int kBarrierOffset = kStages * kStageBytes;
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;     // barriers + alignment slack
 };
 
 template <int BLOCK_N>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
-                    const __grid_constant__ CUtensorMap tmM, int nfreq, int pc, int C, int K,
+                    float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
                     int* __restrict__ status) {
   using L = SmemLayout<BLOCK_N>;
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
@@ -231,11 +133,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     }
   } else {
     // ---------------- epilogue (warps 2..5); a warp may only read TMEM lanes 32*(warp%4)..+31.
-    // Each warp moves its 32 rows in [32 rows][32 floats] boxes: TMEM -> registers ->
-    // 128B-swizzled shared memory -> TMA store (which clips rows >= pc and columns >= K).
+    // Rows >= pc of the last row block are zeros (the TMA loads of V fill them) and land in the
+    // padding rows pc..pc_pad-1 of M.
     const int quad = warp & 3;
-    uint8_t* stage_out = smem + L::kOutOffset + (warp - 2) * L::kOutBytesPerWarp;
-    uint32_t local = 0, nbox = 0;
+    const int k4 = K >> 2;
+    uint32_t local = 0;
     for (long long it = blockIdx.x; it < num_items && !timed_out; it += gridDim.x, ++local) {
       const int kb = (int)(it % num_kb);
       const int pb = (int)((it / num_kb) % num_pb);
@@ -243,33 +145,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
       if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int row0 = pb * BLOCK_M + quad * 32;
+      const int row = pb * BLOCK_M + quad * 32 + lane;
       const int k_left = K - kb * BLOCK_N;
+      float* dst = Mo + (((size_t)f * k4 + (size_t)(kb * BLOCK_N >> 2)) * pc_pad + row) * 4;
+      const size_t q_stride = (size_t)pc_pad * 4;        // floats between consecutive filter quads
 #pragma unroll 1
-      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32, ++nbox) {
-        uint8_t* buf = stage_out + (nbox & 1) * (32 * 128);
-        if (lane == 0) bulk_wait_read<1>();          // the store that last read this buffer is done
-        __syncwarp();
+      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + cb, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        uint8_t* my_row = buf + lane * 128;
 #pragma unroll
-        for (int j = 0; j < 8; ++j)                  // 16-byte chunk j of row `lane` lives at chunk j ^ (lane & 7)
-          *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) =
-              make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) {
-          if (row0 < pc) tma_store_3d(&tmM, buf, kb * BLOCK_N + cb, row0, f);
-          bulk_commit();   // one group per box, stored or not, so "at most one pending" always means the other buffer
-        }
+        for (int j = 0; j < 8; ++j)
+          if (cb + 4 * j < k_left)
+            *reinterpret_cast<uint4*>(dst + (size_t)((cb >> 2) + j) * q_stride) =
+                make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
     }
-    if (lane == 0) bulk_wait_all();
   }
 
   if (timed_out) {
@@ -330,18 +224,17 @@ int launch_n(const void* V, const void* U, float* M, int nfreq, int pc, int pc_p
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
-  CUtensorMap tmV, tmU, tmM;
-  const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  CUtensorMap tmV, tmU;
+  const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
   if (!make_map_3d(&tmV, f16, 2, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
-      !make_map_3d(&tmU, f16, 2, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N) ||
-      !make_map_3d(&tmM, f32, 4, M, K, pc, (long long)pc_pad * K, nfreq, 32, 32))
+      !make_map_3d(&tmU, f16, 2, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N))
     return (int)cudaErrorUnknown;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const long long items = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M) * ((K + BLOCK_N - 1) / BLOCK_N);
   const int grid = (int)(items < sms ? items : sms);
-  gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, tmM, nfreq, pc, C, K, status);
+  gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K, status);
   return (int)cudaGetLastError();
 }
 

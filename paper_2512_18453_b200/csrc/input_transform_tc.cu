@@ -1,0 +1,321 @@
+// Input-tile transform on the sm_100a tensor cores (Section 2.1 step 1 in its 2-D nested
+// form, Appendix B.5): V = B^T d B written as one contraction over the n*n patch elements,
+//   V[(xi,nu)][p][c] = sum_{(a,b)} (B^T (x) B^T)[(xi,nu)][(a,b)] * d_p[(a,b)][c],
+// half x half -> float, rounded once to half.
+//
+// The n^2 x n^2 constant matrix is the Kronecker product of the plan's rounded B^T table
+// with itself.  A product of two half values needs up to 22 significant bits, so the plan
+// stores it as hi + lo (two half matrices, hi = fl16(prod), lo = fl16(prod - hi)) and the
+// kernel issues the MMAs of both into the same accumulator: the result is the float
+// accumulation of exact products of the rounded coefficients with the inputs, i.e. the
+// same quantity the CUDA-core transform evaluates, in a different summation order.
+//
+// One work unit = (tile p, block of 128 channels):
+//   warp 0     TMA producer: the n x n x 64-channel patch boxes of the unit (two boxes, one
+//              per 64 channels) straight from x [N,H,W,C]; rows/columns outside the image
+//              and channels >= C are zero-filled by the TMA unit (the pad-1 halo and ragged
+//              tiles cost nothing).  The box lands as n*n rows of 128 bytes with the 128-byte
+//              swizzle, which is the MN-major operand layout of tcgen05.mma (M = channels).
+//   warp 1     MMA issuer: D[128 channels][n^2 frequencies] (TMEM, 4 accumulators in flight)
+//              = patch (A, MN-major, from the ring) x Kronecker matrix (B, K-major, resident
+//              in shared memory for the whole kernel).
+//   warps 2-9  epilogue, two groups of four warps alternating units: tcgen05.ld, convert to
+//              half, store V[f][p][c] (a lane is a channel: 64 contiguous bytes per warp store).
+// Every wait is bounded; on expiry the kernel records a status and drains.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+#include "sm100.cuh"
+
+namespace nova {
+namespace {
+using namespace sm100;
+
+constexpr int kTcThreads = 320;
+constexpr int kAccCols = 128;          // TMEM columns reserved per accumulator
+constexpr int kNumAcc = 4;
+
+template <int M>
+struct TcCfg {
+  static constexpr int N = M + 2;
+  static constexpr int NF = N * N;                       // frequencies = patch elements
+  static constexpr int KP = (NF + 15) / 16 * 16;         // contraction length, padded to the MMA K
+  static constexpr int NFP = KP;                         // MMA N, padded to a multiple of 16
+  static constexpr int KA = (KP + 63) / 64;              // 64-wide K atoms of the K-major operand
+  static constexpr int kHalfBytes = KP * 128;            // one 64-channel half of a stage
+  static constexpr int kStageBytes = 2 * kHalfBytes;
+  static constexpr int kKronBytes = 2 * KA * NFP * 128;  // hi and lo
+  static constexpr int kStages = (kStageBytes <= 16384) ? 8 : 5;
+  static constexpr int kBarrierOffset = kKronBytes + kStages * kStageBytes;
+  static constexpr int kTotal = kBarrierOffset + 512 + 1024;
+};
+
+template <int NR>
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+template <int M>
+__global__ void __launch_bounds__(kTcThreads, 1)
+input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
+                          __half* __restrict__ V, int C, int Th, int Tw, long long p0, int pc, int pc_pad,
+                          int* __restrict__ status) {
+  using Cfg = TcCfg<M>;
+  constexpr int kStages = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* kron = smem;
+  uint8_t* ring = smem + Cfg::kKronBytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarrierOffset);
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full = empty_bar + kStages;         // [kNumAcc]
+  uint64_t* tmem_empty = tmem_full + kNumAcc;        // [kNumAcc]
+  uint64_t* kron_bar = tmem_empty + kNumAcc;
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(kron_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int CB = (C + 127) / 128;
+  const long long num_units = (long long)pc * CB;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < kNumAcc; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    mbar_init(kron_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_base_slot, kNumAcc * kAccCols);
+  // Rows NF .. KP-1 of every stage half are never written by the TMA boxes; the matching
+  // Kronecker columns are zero, so the rows only have to be finite: clear them once.
+  if constexpr (Cfg::KP > Cfg::NF) {
+    constexpr int pad16 = (Cfg::KP - Cfg::NF) * 8;   // 16-byte pieces per half
+    for (int i = threadIdx.x; i < kStages * 2 * pad16; i += kTcThreads) {
+      const int half = i / pad16, off = i % pad16;
+      *reinterpret_cast<uint4*>(ring + (size_t)half * Cfg::kHalfBytes + Cfg::NF * 128 + off * 16) =
+          make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+  bool timed_out = false;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(kron_bar, Cfg::kKronBytes);
+      for (int b = 0; b < 2 * Cfg::KA; ++b)
+        tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, &tmKron, kron_bar, 0, b * Cfg::NFP);
+    }
+    uint32_t stage = 0, phase = 0;
+    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x) {
+      const int cblk = (int)(u % CB);
+      const long long p = p0 + u / CB;
+      const int tw = (int)(p % Tw);
+      const int th = (int)((p / Tw) % Th);
+      const int img = (int)(p / ((long long)Tw * Th));
+      if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (lane == 0) {
+        uint8_t* dst = ring + (size_t)stage * Cfg::kStageBytes;
+        mbar_expect_tx(&full_bar[stage], 2 * Cfg::NF * 128);
+        tma_load_4d(dst, &tmX, &full_bar[stage], cblk * 128, M * tw - 1, M * th - 1, img);
+        tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - 1, M * th - 1, img);
+      }
+      __syncwarp();
+      if (++stage == kStages) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    constexpr uint32_t idesc = umma_idesc_f16_amn(128, Cfg::NFP);
+    uint32_t stage = 0, phase = 0, local = 0;
+    if (!mbar_wait(kron_bar, 0, abort_flag)) timed_out = true;
+    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x, ++local) {
+      const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
+      if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t sa = smem_u32(ring + (size_t)stage * Cfg::kStageBytes);
+        const uint32_t sk = smem_u32(kron);
+        const uint32_t tmem_d = tmem_base + acc * kAccCols;
+#pragma unroll
+        for (int hl = 0; hl < 2; ++hl)
+#pragma unroll
+          for (int ks = 0; ks < Cfg::KP / 16; ++ks) {
+            const uint64_t ad = umma_desc_mn_sw128(sa + ks * 2048, Cfg::kHalfBytes);
+            const uint64_t bd = umma_desc_sw128(sk + (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
+            umma_f16(tmem_d, ad, bd, idesc, (hl > 0 || ks > 0) ? 1u : 0u);
+          }
+        umma_commit(&empty_bar[stage]);
+        umma_commit(&tmem_full[acc]);
+      }
+      __syncwarp();
+      if (++stage == kStages) { stage = 0; phase ^= 1; }
+    }
+  } else {
+    // ---------------- epilogue: warps 2-5 take even units, warps 6-9 odd units.
+    const int quad = warp & 3;                    // the TMEM lane quadrant this warp may read
+    const int group = (warp - 2) >> 2;
+    const size_t f_stride = (size_t)pc_pad * C;
+    uint32_t local = 0;
+    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x, ++local) {
+      if ((int)(local & 1) != group) continue;
+      const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
+      const int cblk = (int)(u % CB);
+      const int pl = (int)(u / CB);
+      const int c = cblk * 128 + quad * 32 + lane;
+      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
+      __half* dst = V + (size_t)pl * C + c;
+#pragma unroll
+      for (int col0 = 0; col0 < Cfg::NFP; col0 += 64) {
+        constexpr int kMaxCols = 64;
+        uint32_t r[kMaxCols];
+#pragma unroll
+        for (int cc = 0; cc < kMaxCols; cc += 16)
+          if (col0 + cc < Cfg::NFP) tmem_ld16<16>(taddr + col0 + cc, r + cc);
+        tmem_ld_wait();
+        if (col0 + 64 >= Cfg::NFP) {              // everything of this accumulator is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+        }
+        if (c < C) {
+#pragma unroll
+          for (int cc = 0; cc < kMaxCols; ++cc) {
+            const int f = col0 + cc;
+            if (f < Cfg::NF) dst[(size_t)f * f_stride] = __float2half_rn(__uint_as_float(r[cc]));
+          }
+        }
+      }
+    }
+  }
+
+  if (timed_out) {
+    *abort_flag = 1;
+    if (lane == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kNumAcc * kAccCols);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+template <int M>
+int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc, int pc_pad,
+             cudaStream_t stream) {
+  using Cfg = TcCfg<M>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
+    if (e != cudaSuccess) return (int)e;
+    attr_set = true;
+  }
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return (int)cudaErrorUnknown;
+  CUtensorMap tmX, tmK;
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+    cuuint64_t strides[3] = {(cuuint64_t)g.C * 2, (cuuint64_t)g.W * g.C * 2, (cuuint64_t)g.H * g.W * g.C * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)Cfg::N, (cuuint32_t)Cfg::N, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(&tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return (int)cudaErrorUnknown;
+  }
+  {
+    cuuint64_t dims[2] = {64, (cuuint64_t)(2 * Cfg::KA * Cfg::NFP)};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {64, (cuuint32_t)Cfg::NFP};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmK, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, plan->kron_dev, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return (int)cudaErrorUnknown;
+  }
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const long long units = (long long)pc * ((g.C + 127) / 128);
+  const int grid = (int)(units < sms ? units : sms);
+  input_transform_tc_kernel<M><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
+      tmX, tmK, (__half*)V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev);
+  return (int)cudaGetLastError();
+}
+
+}  // namespace
+
+size_t kron_table_halves(int m) {
+  const int n = m + 2, nf = n * n, kp = (nf + 15) / 16 * 16, ka = (kp + 63) / 64;
+  return (size_t)2 * ka * kp * 64;
+}
+
+// Host image of the device table: [hi|lo][K atom][frequency row, padded][64 halves].
+void build_kron_table(const nova_plan* plan, unsigned short* out) {
+  const int n = plan->n, nf = n * n, kp = (nf + 15) / 16 * 16, ka = (kp + 63) / 64;
+  for (size_t i = 0; i < kron_table_halves(plan->m); ++i) out[i] = 0;
+  for (int xi = 0; xi < n; ++xi)
+    for (int nu = 0; nu < n; ++nu)
+      for (int a = 0; a < n; ++a)
+        for (int b = 0; b < n; ++b) {
+          const int f = xi * n + nu, k = a * n + b;
+          const double prod = (double)plan->kcoefs.BT[xi][a] * (double)plan->kcoefs.BT[nu][b];
+          const __half hi = __double2half(prod);
+          const double hid = (double)__half2float(hi);
+          __half lo = __float2half(0.f);
+          if (hid - hid == 0.0) lo = __double2half(prod - hid);      // hi finite
+          const size_t at = ((size_t)(k / 64) * kp + f) * 64 + (k % 64);
+          out[at] = __half_as_ushort(hi);
+          out[(size_t)ka * kp * 64 + at] = __half_as_ushort(lo);
+        }
+}
+
+int launch_input_transform_tc(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0,
+                              int pc, int pc_pad, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  switch (plan->m) {
+    case 2: return launch_m<2>(plan, g, x, V, p0, pc, pc_pad, s);
+    case 4: return launch_m<4>(plan, g, x, V, p0, pc, pc_pad, s);
+    case 6: return launch_m<6>(plan, g, x, V, p0, pc, pc_pad, s);
+    case 8: return launch_m<8>(plan, g, x, V, p0, pc, pc_pad, s);
+  }
+  return (int)cudaErrorInvalidValue;
+}
+
+}  // namespace nova

@@ -29,7 +29,17 @@ struct nova_plan {
   double G[nova::kMaxN * nova::kR];       // n x r
   double BT[nova::kMaxN * nova::kMaxN];   // n x n
   double kappa2_V;
-  nova::Coefs coefs;                      // rounded to the coefficient precision
+  nova::Coefs coefs;                      // rounded to the coefficient precision, caller's point order
+  // The kernels index frequencies in an internal point order: perm[i] is the
+  // caller's index of internal point i.  For a symmetric set {0, +-a_1, ..,
+  // +-a_q, infinity} the internal order is 0, +a_1, -a_1, .., +a_q, -a_q,
+  // infinity, the rounded tables have the even/odd structure the SYM kernel
+  // paths rely on (checked entry by entry), and symmetric = 1; otherwise the
+  // order is the caller's and the kernels evaluate dense products.
+  nova::Coefs kcoefs;
+  int perm[nova::kMaxN];
+  int symmetric;
+  void* kron_dev;                         // device table of the tensor-core input transform (may be null)
   int* status_dev;                        // device status word (null without a device)
   int device;                             // device that owns status_dev
 };
@@ -56,6 +66,10 @@ inline Geom make_geom(const nova_plan* p, int N, int H, int W, int C, int K) {
 int launch_filter_transform(const nova_plan* plan, const void* g, int K, int C, void* U, void* stream);
 int launch_input_transform(const nova_plan* plan, const Geom& g, const void* x, void* V,
                            long long p0, int pc, int pc_pad, void* stream);
+int launch_input_transform_tc(const nova_plan* plan, const Geom& g, const void* x, void* V,
+                              long long p0, int pc, int pc_pad, void* stream);
+size_t kron_table_halves(int m);
+void build_kron_table(const nova_plan* plan, unsigned short* out);
 int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y,
                             long long p0, int pc, int pc_pad, int relu, void* stream);
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,

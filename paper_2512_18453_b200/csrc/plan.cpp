@@ -311,6 +311,63 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
   for (int p = 0; p < n; ++p)
     for (int j = 0; j < n; ++j) pl->coefs.BT[p][j] = rnd(pl->BT[p * n + j]);
 
+  // Internal point order and kernel tables.
+  for (int i = 0; i < n; ++i) pl->perm[i] = i;
+  pl->symmetric = 0;
+  {
+    int order[nova::kMaxN], cnt = 0, zero_at = -1;
+    bool used[nova::kMaxN] = {};
+    for (int i = 0; i < nf; ++i)
+      if (al[i].n == 0) zero_at = i;
+    bool sym = zero_at >= 0 && (nf % 2) == 1;
+    if (sym) {
+      order[cnt++] = zero_at;
+      used[zero_at] = true;
+      for (int i = 0; i < nf && sym; ++i) {
+        if (used[i]) continue;
+        int mate = -1;
+        for (int j = 0; j < nf; ++j)
+          if (!used[j] && j != i && al[j].d == al[i].d && al[j].n == -al[i].n) mate = j;
+        if (mate < 0) { sym = false; break; }
+        const int pos = al[i].n > 0 ? i : mate, neg = al[i].n > 0 ? mate : i;
+        order[cnt++] = pos;
+        order[cnt++] = neg;
+        used[i] = used[mate] = true;
+      }
+      if (sym) order[cnt++] = n - 1;
+    }
+    if (sym && cnt == n)
+      for (int i = 0; i < n; ++i) pl->perm[i] = order[i];
+    nova::Coefs& k = pl->kcoefs;
+    for (int i = 0; i < m; ++i)
+      for (int p = 0; p < n; ++p) k.AT[i][p] = pl->coefs.AT[i][pl->perm[p]];
+    for (int p = 0; p < n; ++p) {
+      for (int kk = 0; kk < r; ++kk) k.G[p][kk] = pl->coefs.G[pl->perm[p]][kk];
+      for (int j = 0; j < n; ++j) k.BT[p][j] = pl->coefs.BT[pl->perm[p]][j];
+    }
+    // The SYM kernel paths skip the structural zeros and share even/odd partial sums of a
+    // +-pair; they are used only if the rounded tables have exactly that structure.
+    if (sym && cnt == n) {
+      bool ok = true;
+      for (int j = 0; j < n; ++j) {
+        if ((j & 1) && k.BT[0][j] != 0.f) ok = false;
+        if (!(j & 1) && k.BT[n - 1][j] != 0.f) ok = false;
+      }
+      for (int i = 0; i < m; ++i) {
+        if (k.AT[i][0] != (i == 0 ? 1.f : 0.f)) ok = false;
+        if (k.AT[i][n - 1] != (i == m - 1 ? 1.f : 0.f)) ok = false;
+      }
+      for (int q = 1; q + 1 < n - 1; q += 2) {
+        if (k.BT[q][n - 1] != 0.f || k.BT[q + 1][n - 1] != 0.f) ok = false;
+        for (int j = 0; j < n; ++j)
+          if (k.BT[q + 1][j] != ((j & 1) ? -k.BT[q][j] : k.BT[q][j])) ok = false;
+        for (int i = 0; i < m; ++i)
+          if (k.AT[i][q + 1] != ((i & 1) ? -k.AT[i][q] : k.AT[i][q])) ok = false;
+      }
+      pl->symmetric = ok ? 1 : 0;
+    }
+  }
+
   std::vector<double> V(nf * nf);
   for (int i = 0; i < nf; ++i) {
     double a = rat_to_double(al[i]), pw = 1.0;
@@ -331,6 +388,16 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
         pl->status_dev = w;
         pl->device = dev;
       }
+      // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
+      if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
+        std::vector<unsigned short> img(nova::kron_table_halves(m));
+        nova::build_kron_table(pl, img.data());
+        void* kd = nullptr;
+        if (cudaMalloc(&kd, img.size() * 2) == cudaSuccess) {
+          if (cudaMemcpy(kd, img.data(), img.size() * 2, cudaMemcpyHostToDevice) == cudaSuccess) pl->kron_dev = kd;
+          else cudaFree(kd);
+        }
+      }
     }
   }
   (void)cudaGetLastError();
@@ -341,6 +408,7 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
 extern "C" void nova_plan_destroy(nova_plan* plan) {
   if (!plan) return;
   if (plan->status_dev) cudaFree(plan->status_dev);
+  if (plan->kron_dev) cudaFree(plan->kron_dev);
   delete plan;
 }
 
@@ -363,6 +431,14 @@ extern "C" int nova_plan_get_device_tables(const nova_plan* p, float* AT, float*
   for (int q = 0; q < p->n; ++q)
     for (int j = 0; j < p->n; ++j)
       if (BT) BT[q * p->n + j] = p->coefs.BT[q][j];
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_frequency_order(const nova_plan* p, int* perm, int* symmetric) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  if (perm)
+    for (int i = 0; i < p->n; ++i) perm[i] = p->perm[i];
+  if (symmetric) *symmetric = p->symmetric;
   return NOVA_OK;
 }
 

@@ -23,6 +23,28 @@ __device__ __forceinline__ float2 fma2(float a, float2 b, float2 c) {
 }
 __device__ __forceinline__ float2 mul2(float a, float2 b) { return make_float2(a * b.x, a * b.y); }
 
+// Scalar / 2-vector arithmetic used by the output transform (VEC filters per thread).
+template <int VEC> struct VecOf;
+template <> struct VecOf<1> { using type = float; };
+template <> struct VecOf<2> { using type = float2; };
+template <typename V> __device__ __forceinline__ V vzero();
+template <> __device__ __forceinline__ float vzero<float>() { return 0.f; }
+template <> __device__ __forceinline__ float2 vzero<float2>() { return make_float2(0.f, 0.f); }
+__device__ __forceinline__ float vmul(float a, float b) { return a * b; }
+__device__ __forceinline__ float2 vmul(float a, float2 b) { return mul2(a, b); }
+__device__ __forceinline__ float vfma(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ float2 vfma(float a, float2 b, float2 c) { return fma2(a, b, c); }
+__device__ __forceinline__ float vadd(float a, float b) { return a + b; }
+__device__ __forceinline__ float2 vadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float vsub(float a, float b) { return a - b; }
+__device__ __forceinline__ float2 vsub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float vrelu(float v) { return v < 0.f ? 0.f : v; }
+__device__ __forceinline__ float2 vrelu(float2 v) { return make_float2(v.x < 0.f ? 0.f : v.x, v.y < 0.f ? 0.f : v.y); }
+__device__ __forceinline__ void vstore(__half* p, float v) { *p = __float2half_rn(v); }
+__device__ __forceinline__ void vstore(float* p, float v) { *p = v; }
+__device__ __forceinline__ void vstore(__half* p, float2 v) { st2(p, v); }
+__device__ __forceinline__ void vstore(float* p, float2 v) { st2(p, v); }
+
 // ---------------------------------------------------------------- U = G g G^T
 // One thread per (filter k, channel pair).  g [K,3,3,C] -> U [n*n][K][C].
 template <int M, typename T>
@@ -61,19 +83,162 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
     }
 }
 
-// ---------------------------------------------------------------- V = B^T d B
-// One thread per (tile, channel pair, column group).  x [N,H,W,C] ->
-// V [n*n][pc_pad][C] for the tiles p0 .. p0+pc-1.  SPLITS threads share one
-// patch; each produces the frequencies (xi, nu) with nu in its column group.
-template <int M, typename T, int SPLITS, int SPLIT>
-__device__ __forceinline__ void input_transform_body(const Coefs& cf, const T* __restrict__ x,
-                                                     T* __restrict__ V, int H, int W, int C, int Th,
-                                                     int Tw, long long p0, int pc, int pc_pad) {
+// ---------------------------------------------------------------- 1-D building blocks
+// For a point set that is symmetric about 0 (internal order 0, +a, -a, .., infinity) the
+// rounded tables satisfy, entry by entry (checked when the plan is built):
+//   B^T row 0 has only even columns, row n-1 only odd columns, rows +a / -a have equal even
+//   columns and opposite odd columns, and no finite row reaches column n-1;
+//   A^T column 0 is e_0, column n-1 is e_{m-1}, columns +a / -a are equal in even rows and
+//   opposite in odd rows.
+// SYM = true evaluates the same sums with the zeros skipped and the even/odd partial sums of
+// a +-pair shared; SYM = false is the dense product.
+
+// Two rows of B^T applied to one n-vector.  Group g = 0 gives rows (0, n-1); g >= 1 gives the
+// pair (2g-1, 2g).
+template <int N, bool SYM, int G>
+__device__ __forceinline__ void bt_two_rows(const Coefs& cf, const float2 (&in)[N], float2& oa, float2& ob) {
+  constexpr int RA = (G == 0) ? 0 : 2 * G - 1;
+  constexpr int RB = (G == 0) ? N - 1 : 2 * G;
+  if constexpr (!SYM) {
+    float2 a = mul2(cf.BT[RA][0], in[0]), b = mul2(cf.BT[RB][0], in[0]);
+#pragma unroll
+    for (int j = 1; j < N; ++j) {
+      a = fma2(cf.BT[RA][j], in[j], a);
+      b = fma2(cf.BT[RB][j], in[j], b);
+    }
+    oa = a; ob = b;
+  } else if constexpr (G == 0) {
+    float2 e = mul2(cf.BT[0][0], in[0]);
+#pragma unroll
+    for (int j = 2; j < N; j += 2) e = fma2(cf.BT[0][j], in[j], e);
+    float2 o = mul2(cf.BT[N - 1][1], in[1]);
+#pragma unroll
+    for (int j = 3; j < N; j += 2) o = fma2(cf.BT[N - 1][j], in[j], o);
+    oa = e; ob = o;
+  } else {
+    float2 e = mul2(cf.BT[RA][0], in[0]);
+#pragma unroll
+    for (int j = 2; j < N; j += 2) e = fma2(cf.BT[RA][j], in[j], e);
+    float2 o = mul2(cf.BT[RA][1], in[1]);
+#pragma unroll
+    for (int j = 3; j < N - 1; j += 2) o = fma2(cf.BT[RA][j], in[j], o);
+    oa = make_float2(e.x + o.x, e.y + o.y);
+    ob = make_float2(e.x - o.x, e.y - o.y);
+  }
+}
+
+// All n rows of B^T applied to one n-vector.
+template <int N, bool SYM>
+__device__ __forceinline__ void bt_all_rows(const Coefs& cf, const float2 (&in)[N], float2 (&out)[N]) {
+  if constexpr (!SYM) {
+#pragma unroll
+    for (int p = 0; p < N; ++p) {
+      float2 s = mul2(cf.BT[p][0], in[0]);
+#pragma unroll
+      for (int j = 1; j < N; ++j) s = fma2(cf.BT[p][j], in[j], s);
+      out[p] = s;
+    }
+  } else {
+    bt_two_rows<N, true, 0>(cf, in, out[0], out[N - 1]);
+    if constexpr (N >= 4) bt_two_rows<N, true, 1>(cf, in, out[1], out[2]);
+    if constexpr (N >= 6) bt_two_rows<N, true, 2>(cf, in, out[3], out[4]);
+    if constexpr (N >= 8) bt_two_rows<N, true, 3>(cf, in, out[5], out[6]);
+    if constexpr (N >= 10) bt_two_rows<N, true, 4>(cf, in, out[7], out[8]);
+  }
+}
+
+// z[i] = sum_p A^T[i][p] * in[p], i < M.
+template <int M, bool SYM, typename V>
+__device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[M + 2], V (&z)[M]) {
   constexpr int N = M + 2;
-  constexpr int NU = N / SPLITS;
-  constexpr int NU0 = SPLIT * NU;
+  if constexpr (!SYM) {
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+      V s = vmul(cf.AT[i][0], in[0]);
+#pragma unroll
+      for (int p = 1; p < N; ++p) s = vfma(cf.AT[i][p], in[p], s);
+      z[i] = s;
+    }
+  } else {
+    V sm[M / 2], df[M / 2];
+#pragma unroll
+    for (int q = 0; q < M / 2; ++q) {
+      sm[q] = vadd(in[1 + 2 * q], in[2 + 2 * q]);
+      df[q] = vsub(in[1 + 2 * q], in[2 + 2 * q]);
+    }
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+      V s = (i & 1) ? vmul(cf.AT[i][1], df[0]) : vmul(cf.AT[i][1], sm[0]);
+#pragma unroll
+      for (int q = 1; q < M / 2; ++q)
+        s = (i & 1) ? vfma(cf.AT[i][1 + 2 * q], df[q], s) : vfma(cf.AT[i][1 + 2 * q], sm[q], s);
+      if (i == 0) s = vadd(s, in[0]);
+      if (i == M - 1) s = vadd(s, in[N - 1]);
+      z[i] = s;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- V = B^T d B
+// x [N,H,W,C] -> V [n*n][pc_pad][C] for the tiles p0 .. p0+pc-1.  A thread owns one
+// (tile, channel pair) and one group of two B^T rows: it applies those two rows along the
+// patch's columns (nu), keeps the n x 2 intermediate in registers, applies all n rows along
+// the patch's rows (xi) and stores the 2n frequencies (xi, nu in its group).  The n/2 groups
+// of a patch sit in one block, so the patch is read from DRAM once and from L1 afterwards.
+template <int M, typename T, bool SYM, int G>
+__device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* __restrict__ x,
+                                                      T* __restrict__ V, int H, int W, int C, int h0,
+                                                      int w0, long long img, size_t out_off,
+                                                      size_t f_stride) {
+  constexpr int N = M + 2;
+  constexpr int RA = (G == 0) ? 0 : 2 * G - 1;
+  constexpr int RB = (G == 0) ? N - 1 : 2 * G;
+  float2 ta[N], tb[N];
+  const bool interior = h0 >= 0 && w0 >= 0 && h0 + N <= H && w0 + N <= W;
+  if (interior) {
+    const T* base = x + (((size_t)img * H + h0) * W + w0) * C;
+#pragma unroll
+    for (int a = 0; a < N; ++a) {
+      float2 d[N];
+#pragma unroll
+      for (int b = 0; b < N; ++b) d[b] = ld2(base + ((size_t)a * W + b) * C);
+      bt_two_rows<N, SYM, G>(cf, d, ta[a], tb[a]);
+    }
+  } else {
+#pragma unroll
+    for (int a = 0; a < N; ++a) {
+      const int h = h0 + a;
+      const bool hv = (h >= 0) && (h < H);
+      float2 d[N];
+#pragma unroll
+      for (int b = 0; b < N; ++b) {
+        const int w = w0 + b;
+        d[b] = make_float2(0.f, 0.f);
+        if (hv && w >= 0 && w < W) d[b] = ld2(x + (((size_t)img * H + h) * W + w) * C);
+      }
+      bt_two_rows<N, SYM, G>(cf, d, ta[a], tb[a]);
+    }
+  }
+  float2 oa[N], ob[N];
+  bt_all_rows<N, SYM>(cf, ta, oa);
+  bt_all_rows<N, SYM>(cf, tb, ob);
+#pragma unroll
+  for (int xi = 0; xi < N; ++xi) {
+    st2(V + out_off + (size_t)(xi * N + RA) * f_stride, oa[xi]);
+    st2(V + out_off + (size_t)(xi * N + RB) * f_stride, ob[xi]);
+  }
+}
+
+template <int M, typename T, bool SYM>
+__global__ void __launch_bounds__(32 * (M + 2) * 2)
+input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, T* __restrict__ V,
+                       int H, int W, int C, int Th, int Tw, long long p0, int pc, int pc_pad) {
+  constexpr int N = M + 2;
+  constexpr int WORK = 128;                       // (tile, channel pair) items per block
+  // threads [g*128, g*128+128) form group g (warp-uniform)
+  const int g = threadIdx.x / WORK;
   const int c2 = C >> 1;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long idx = (long long)blockIdx.x * WORK + (threadIdx.x % WORK);
   if (idx >= (long long)pc * c2) return;
   const int pl = (int)(idx / c2);
   const int c = (int)(idx % c2) * 2;
@@ -82,87 +247,97 @@ __device__ __forceinline__ void input_transform_body(const Coefs& cf, const T* _
   const int th = (int)((p / Tw) % Th);
   const long long img = p / ((long long)Tw * Th);
   const int h0 = M * th - 1, w0 = M * tw - 1;
-
-  float2 t[N][NU];
-#pragma unroll
-  for (int a = 0; a < N; ++a) {
-    const int h = h0 + a;
-    const bool hv = (h >= 0) && (h < H);
-    float2 d[N];
-#pragma unroll
-    for (int b = 0; b < N; ++b) {
-      const int w = w0 + b;
-      d[b] = make_float2(0.f, 0.f);
-      if (hv && w >= 0 && w < W) d[b] = ld2(x + (((size_t)img * H + h) * W + w) * C + c);
-    }
-#pragma unroll
-    for (int j = 0; j < NU; ++j) {
-      float2 s = mul2(cf.BT[NU0 + j][0], d[0]);
-#pragma unroll
-      for (int b = 1; b < N; ++b) s = fma2(cf.BT[NU0 + j][b], d[b], s);
-      t[a][j] = s;
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < NU; ++j)
-#pragma unroll
-    for (int xi = 0; xi < N; ++xi) {
-      float2 s = mul2(cf.BT[xi][0], t[0][j]);
-#pragma unroll
-      for (int a = 1; a < N; ++a) s = fma2(cf.BT[xi][a], t[a][j], s);
-      st2(V + ((size_t)(xi * N + NU0 + j) * pc_pad + pl) * C + c, s);
-    }
-}
-
-template <int M, typename T, int SPLITS>
-__global__ void __launch_bounds__(128)
-input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, T* __restrict__ V,
-                       int H, int W, int C, int Th, int Tw, long long p0, int pc, int pc_pad) {
-  if constexpr (SPLITS == 1) {
-    input_transform_body<M, T, 1, 0>(cf, x, V, H, W, C, Th, Tw, p0, pc, pc_pad);
-  } else {
-    if (blockIdx.y == 0) input_transform_body<M, T, 2, 0>(cf, x, V, H, W, C, Th, Tw, p0, pc, pc_pad);
-    else input_transform_body<M, T, 2, 1>(cf, x, V, H, W, C, Th, Tw, p0, pc, pc_pad);
+  const size_t out_off = (size_t)pl * C + c;
+  const size_t f_stride = (size_t)pc_pad * C;
+  const T* xc = x + c;
+  switch (g) {
+    case 0: input_transform_group<M, T, SYM, 0>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 1: input_transform_group<M, T, SYM, 1>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 2: if constexpr (N >= 6) input_transform_group<M, T, SYM, 2>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 3: if constexpr (N >= 8) input_transform_group<M, T, SYM, 3>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 4: if constexpr (N >= 10) input_transform_group<M, T, SYM, 4>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
   }
 }
 
 // ---------------------------------------------------------------- Y = A^T M A
-// One thread per (tile, filter pair).  M [n*n][pc_pad][K] float -> y [N,H,W,K].
-template <int M, typename T>
-__global__ void __launch_bounds__(128)
+// M is stored [n*n][K/4][pc_pad][4] (filter quads outermost, then tiles): the product kernel
+// writes it and this kernel reads it in 32-byte pieces.  A thread owns one tile and VEC
+// consecutive filters; a warp covers 2 tiles x 16 such units, so that its M reads are whole
+// 32-byte sectors and its y stores are 32*VEC contiguous bytes per pixel.
+template <int M, typename T, bool SYM, int VEC>
+__global__ void __launch_bounds__(256, (M == 8 || VEC == 1) ? 2 : 2)
 output_transform_kernel(const __grid_constant__ Coefs cf, const float* __restrict__ Mb,
                         T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
                         int pc_pad, int relu) {
   constexpr int N = M + 2;
-  const int k2 = K >> 1;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (long long)pc * k2) return;
-  const int pl = (int)(idx / k2);
-  const int k = (int)(idx % k2) * 2;
+  using Vv = typename VecOf<VEC>::type;
+  const int t = threadIdx.x;
+  const int unit = blockIdx.x * 128 + (t & 15) + 16 * (t >> 5);
+  const int pl = blockIdx.y * 2 + ((t >> 4) & 1);
+  const int k = unit * VEC;
+  if (k >= K || pl >= pc) return;
   const long long p = p0 + pl;
   const int tw = (int)(p % Tw);
   const int th = (int)((p / Tw) % Th);
   const long long img = p / ((long long)Tw * Th);
+  const size_t f_stride = (size_t)(K >> 2) * pc_pad * 4;
+  const float* src = Mb + ((size_t)(k >> 2) * pc_pad + pl) * 4 + (k & 3);
 
-  float2 Y[M][M];
+  Vv Y[M][M];
+  auto load_row = [&](int xi, Vv (&z)[M]) {
+    Vv in[N];
 #pragma unroll
-  for (int i = 0; i < M; ++i)
+    for (int nu = 0; nu < N; ++nu) in[nu] = *reinterpret_cast<const Vv*>(src + (size_t)(xi * N + nu) * f_stride);
+    at_apply<M, SYM, Vv>(cf, in, z);
+  };
+  if constexpr (!SYM) {
 #pragma unroll
-    for (int j = 0; j < M; ++j) Y[i][j] = make_float2(0.f, 0.f);
-
+    for (int i = 0; i < M; ++i)
 #pragma unroll
-  for (int nu = 0; nu < N; ++nu) {
-    float2 mm[N];
+      for (int j = 0; j < M; ++j) Y[i][j] = vzero<Vv>();
 #pragma unroll
-    for (int xi = 0; xi < N; ++xi)
-      mm[xi] = *reinterpret_cast<const float2*>(Mb + ((size_t)(xi * N + nu) * pc_pad + pl) * K + k);
+    for (int xi = 0; xi < N; ++xi) {
+      Vv z[M];
+      load_row(xi, z);
 #pragma unroll
-    for (int i = 0; i < M; ++i) {
-      float2 z = mul2(cf.AT[i][0], mm[0]);
+      for (int i = 0; i < M; ++i)
 #pragma unroll
-      for (int xi = 1; xi < N; ++xi) z = fma2(cf.AT[i][xi], mm[xi], z);
+        for (int j = 0; j < M; ++j) Y[i][j] = vfma(cf.AT[i][xi], z[j], Y[i][j]);
+    }
+  } else {
+    // A^T column 0 is e_0 and column n-1 is e_{m-1}; columns +a / -a share |coefficients|.
+    {
+      Vv zp[M], zm[M];
+      load_row(1, zp);
+      load_row(2, zm);
 #pragma unroll
-      for (int j = 0; j < M; ++j) Y[i][j] = fma2(cf.AT[j][nu], z, Y[i][j]);
+      for (int j = 0; j < M; ++j) {
+        const Vv s = vadd(zp[j], zm[j]), d = vsub(zp[j], zm[j]);
+#pragma unroll
+        for (int i = 0; i < M; ++i) Y[i][j] = vmul(cf.AT[i][1], (i & 1) ? d : s);
+      }
+    }
+#pragma unroll
+    for (int q = 3; q < N - 1; q += 2) {
+      Vv zp[M], zm[M];
+      load_row(q, zp);
+      load_row(q + 1, zm);
+#pragma unroll
+      for (int j = 0; j < M; ++j) {
+        const Vv s = vadd(zp[j], zm[j]), d = vsub(zp[j], zm[j]);
+#pragma unroll
+        for (int i = 0; i < M; ++i) Y[i][j] = vfma(cf.AT[i][q], (i & 1) ? d : s, Y[i][j]);
+      }
+    }
+    {
+      Vv z0[M], zi[M];
+      load_row(0, z0);
+      load_row(N - 1, zi);
+#pragma unroll
+      for (int j = 0; j < M; ++j) {
+        Y[0][j] = vadd(Y[0][j], z0[j]);
+        Y[M - 1][j] = vadd(Y[M - 1][j], zi[j]);
+      }
     }
   }
 #pragma unroll
@@ -173,12 +348,9 @@ output_transform_kernel(const __grid_constant__ Coefs cf, const float* __restric
     for (int j = 0; j < M; ++j) {
       const int w = M * tw + j;
       if (w >= W) continue;
-      float2 v = Y[i][j];
-      if (relu) {
-        v.x = v.x < 0.f ? 0.f : v.x;   // NaN and +inf pass through
-        v.y = v.y < 0.f ? 0.f : v.y;
-      }
-      st2(y + (((size_t)img * H + h) * W + w) * K + k, v);
+      Vv v = Y[i][j];
+      if (relu) v = vrelu(v);                     // NaN and +inf pass through
+      vstore(y + (((size_t)img * H + h) * W + w) * K + k, v);
     }
   }
 }
@@ -226,25 +398,34 @@ inline unsigned blocks_for(long long work, int threads) {
 template <int M, typename T>
 int filter_launch(const nova_plan* plan, const void* g, int K, int C, void* U, cudaStream_t s) {
   const long long work = (long long)K * (C / 2);
-  filter_transform_kernel<M, T><<<blocks_for(work, 256), 256, 0, s>>>(plan->coefs, (const T*)g, (T*)U, K, C);
+  filter_transform_kernel<M, T><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, (T*)U, K, C);
   return (int)cudaGetLastError();
 }
 template <int M, typename T>
 int input_launch(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc,
                  int pc_pad, cudaStream_t s) {
+  constexpr int THREADS = 32 * (M + 2) * 2;       // n/2 groups of 128 work items
   const long long work = (long long)pc * (g.C / 2);
-  constexpr int SPLITS = (M == 8) ? 2 : 1;
-  dim3 grid(blocks_for(work, 128), SPLITS);
-  input_transform_kernel<M, T, SPLITS><<<grid, 128, 0, s>>>(plan->coefs, (const T*)x, (T*)V, g.H, g.W, g.C,
-                                                           g.Th, g.Tw, p0, pc, pc_pad);
+  const unsigned grid = blocks_for(work, 128);
+  if (plan->symmetric)
+    input_transform_kernel<M, T, true><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, (T*)V, g.H, g.W,
+                                                                g.C, g.Th, g.Tw, p0, pc, pc_pad);
+  else
+    input_transform_kernel<M, T, false><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, (T*)V, g.H, g.W,
+                                                                 g.C, g.Th, g.Tw, p0, pc, pc_pad);
   return (int)cudaGetLastError();
 }
 template <int M, typename T>
 int output_launch(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0, int pc,
                   int pc_pad, int relu, cudaStream_t s) {
-  const long long work = (long long)pc * (g.K / 2);
-  output_transform_kernel<M, T><<<blocks_for(work, 128), 128, 0, s>>>(
-      plan->coefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
+  constexpr int VEC = (M == 8) ? 1 : 2;
+  dim3 grid(blocks_for(g.K / VEC, 128), (unsigned)((pc + 1) / 2));
+  if (plan->symmetric)
+    output_transform_kernel<M, T, true, VEC><<<grid, 256, 0, s>>>(
+        plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
+  else
+    output_transform_kernel<M, T, false, VEC><<<grid, 256, 0, s>>>(
+        plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
   return (int)cudaGetLastError();
 }
 

@@ -133,7 +133,7 @@ def test_fp16_mode_within_twice_the_emulation(kind, m, shape, flags):
 def test_tcgen05_and_simt_products_agree_elementwise(m):
     x, g = make_conv_inputs(2, 26, 26, 72, 136, "fp16", True, True, seed=400 + m)
     pts = point_set("nova", m)
-    ya, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.GEMM_TCGEN05)
+    ya, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.GEMM_TCGEN05 | nv.TRANSFORM_SIMT)
     yb, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.GEMM_SIMT)
     # same operands, float accumulation in a different order: the outputs differ by
     # final-rounding flips only, far below the pipeline's own error
@@ -142,6 +142,22 @@ def test_tcgen05_and_simt_products_agree_elementwise(m):
     d = np.abs(ya.astype(np.float32) - yb.astype(np.float32))
     assert d.max() <= 4 * 2.0 ** -10 * np.abs(yb.astype(np.float32)).max()
     assert (d > 0).mean() < 0.25
+
+
+@pytest.mark.parametrize("kind,m", [("std", 2), ("nova", 4), ("nova", 6), ("half", 6), ("nova", 8)])
+@pytest.mark.parametrize("shape", [(2, 26, 26, 72, 136), (1, 9, 31, 64, 8), (2, 14, 14, 264, 64)])
+def test_tensor_core_and_cuda_core_input_transforms_agree(kind, m, shape):
+    """Same rounded coefficients, float accumulation in a different order: the two input
+    transforms may differ by final-rounding flips of V only."""
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=470 + m)
+    pts = point_set(kind, m)
+    ya, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC)
+    yb, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.TRANSFORM_SIMT)
+    y1 = conv.direct_conv_fp64(x, g)
+    ea, eb = conv.rel_l2(ya, y1), conv.rel_l2(yb, y1)
+    assert abs(ea - eb) <= 0.05 * eb
+    assert conv.rel_l2(ya, yb) < 0.3 * eb
 
 
 def test_ragged_last_row_block_after_full_blocks():
