@@ -63,6 +63,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const int num_kb = (K + BLOCK_N - 1) / BLOCK_N;
   const int num_ks = (C + BLOCK_K - 1) / BLOCK_K;
   const long long num_items = (long long)nfreq * num_pb * num_kb;
+  // each CTA takes a contiguous range of items (f outermost, then pb, then kb) and advances
+  // the three indices incrementally
+  const long long it_begin = num_items * blockIdx.x / gridDim.x;
+  const long long it_end = num_items * (blockIdx.x + 1) / gridDim.x;
+  const int kb0 = (int)(it_begin % num_kb);
+  const int pb0 = (int)((it_begin / num_kb) % num_pb);
+  const int f0 = (int)(it_begin / ((long long)num_kb * num_pb));
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -86,12 +93,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   if (warp == 0) {
     // ---------------- TMA producer
     uint32_t stage = 0, phase = 0;
-    for (long long it = blockIdx.x; it < num_items && !timed_out; it += gridDim.x) {
-      const int kb = (int)(it % num_kb);
-      const int pb = (int)((it / num_kb) % num_pb);
-      const int f = (int)(it / ((long long)num_kb * num_pb));
+    int kb = kb0, pb = pb0, f = f0;
+    for (long long it = it_begin; it < it_end && !timed_out; ++it) {
       for (int ks = 0; ks < num_ks; ++ks) {
-        if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+        if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
         if (lane == 0) {
           uint8_t* sa = smem + stage * L::kStageBytes;
           uint8_t* sb = sa + L::kABytes;
@@ -102,18 +107,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         __syncwarp();
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
+      if (++kb == num_kb) { kb = 0; if (++pb == num_pb) { pb = 0; ++f; } }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
     constexpr uint32_t idesc = umma_idesc_f16(BLOCK_M, BLOCK_N);
     uint32_t stage = 0, phase = 0, local = 0;
-    for (long long it = blockIdx.x; it < num_items && !timed_out; it += gridDim.x, ++local) {
+    for (long long it = it_begin; it < it_end && !timed_out; ++it, ++local) {
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
-      if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tmem_d = tmem_base + acc * BLOCK_N;
       for (int ks = 0; ks < num_ks; ++ks) {
-        if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+        if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (lane == 0) {
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
@@ -138,12 +144,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int quad = warp & 3;
     const int k4 = K >> 2;
     uint32_t local = 0;
-    for (long long it = blockIdx.x; it < num_items && !timed_out; it += gridDim.x, ++local) {
-      const int kb = (int)(it % num_kb);
-      const int pb = (int)((it / num_kb) % num_pb);
-      const int f = (int)(it / ((long long)num_kb * num_pb));
+    int kb = kb0, pb = pb0, f = f0;
+    for (long long it = it_begin; it < it_end && !timed_out; ++it, ++local) {
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
-      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = pb * BLOCK_M + quad * 32 + lane;
       const int k_left = K - kb * BLOCK_N;
@@ -163,6 +167,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+      if (++kb == num_kb) { kb = 0; if (++pb == num_pb) { pb = 0; ++f; } }
     }
   }
 
@@ -214,7 +219,7 @@ bool make_map_3d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void
 }
 
 template <int BLOCK_N>
-int launch_n(const void* V, const void* U, float* M, int nfreq, int pc, int pc_pad, int C, int K,
+int launch_n(int sms, const void* V, const void* U, float* M, int nfreq, int pc, int pc_pad, int C, int K,
              int* status, cudaStream_t stream) {
   using L = SmemLayout<BLOCK_N>;
   static bool attr_set = false;
@@ -229,9 +234,6 @@ int launch_n(const void* V, const void* U, float* M, int nfreq, int pc, int pc_p
   if (!make_map_3d(&tmV, f16, 2, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
       !make_map_3d(&tmU, f16, 2, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N))
     return (int)cudaErrorUnknown;
-  int dev = 0, sms = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const long long items = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M) * ((K + BLOCK_N - 1) / BLOCK_N);
   const int grid = (int)(items < sms ? items : sms);
   gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K, status);
@@ -242,11 +244,11 @@ int launch_n(const void* V, const void* U, float* M, int nfreq, int pc, int pc_p
 
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M, int nfreq, int pc,
                         int pc_pad, int C, int K, int* status_dev, void* stream) {
-  (void)plan;
   cudaStream_t s = (cudaStream_t)stream;
-  if (K > 128) return launch_n<256>(V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
-  if (K > 64) return launch_n<128>(V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
-  return launch_n<64>(V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  const int sms = plan->sm_count;
+  if (K > 128) return launch_n<256>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  if (K > 64) return launch_n<128>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  return launch_n<64>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
 }
 
 }  // namespace nova

@@ -11,16 +11,21 @@
 // same quantity the CUDA-core transform evaluates, in a different summation order.
 //
 // One work unit = (tile p, block of 128 channels):
-//   warp 0     TMA producer: the n x n x 64-channel patch boxes of the unit (two boxes, one
-//              per 64 channels) straight from x [N,H,W,C]; rows/columns outside the image
-//              and channels >= C are zero-filled by the TMA unit (the pad-1 halo and ragged
-//              tiles cost nothing).  The box lands as n*n rows of 128 bytes with the 128-byte
-//              swizzle, which is the MN-major operand layout of tcgen05.mma (M = channels).
-//   warp 1     MMA issuer: D[128 channels][n^2 frequencies] (TMEM, 4 accumulators in flight)
-//              = patch (A, MN-major, from the ring) x Kronecker matrix (B, K-major, resident
-//              in shared memory for the whole kernel).
-//   warps 2-9  epilogue, two groups of four warps alternating units: tcgen05.ld, convert to
-//              half, store V[f][p][c] (a lane is a channel: 64 contiguous bytes per warp store).
+// The units of a CTA (a contiguous range) are numbered i = 0, 1, ..; unit i uses ring stage
+// i % kStages and TMEM accumulator i % kNumAcc.  Issuing a TMA box or a small MMA costs the
+// issuing thread a few hundred cycles, so every role is spread over several warps:
+//   warps 0-3   TMA producers, unit i by warp i%4: the n x n x 64-channel patch boxes of the
+//               unit (two boxes, one per 64 channels) straight from x [N,H,W,C]; rows/columns
+//               outside the image and channels >= C are zero-filled by the TMA unit (the pad-1
+//               halo and ragged tiles cost nothing).  A box lands as n*n rows of 128 bytes with
+//               the 128-byte swizzle, which is the MN-major operand layout of tcgen05.mma
+//               (M = channels).
+//   warps 4-7   MMA issuers, unit i by warp 4 + i%4: D[128 channels][n^2 frequencies] (TMEM)
+//               = patch (A, MN-major, from the ring) x Kronecker matrix (B, K-major, resident
+//               in shared memory for the whole kernel).
+//   warps 8-23  epilogue, four groups of four warps (one per TMEM lane quadrant), unit i by
+//               group i%4: tcgen05.ld, convert to half, store V[f][p][c] (a lane is a channel:
+//               64 contiguous bytes per warp store).
 // Every wait is bounded; on expiry the kernel records a status and drains.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -33,9 +38,10 @@ namespace nova {
 namespace {
 using namespace sm100;
 
-constexpr int kTcThreads = 320;
-constexpr int kAccCols = 128;          // TMEM columns reserved per accumulator
-constexpr int kNumAcc = 4;
+constexpr int kProdWarps = 4;
+constexpr int kMmaWarps = 4;
+constexpr int kEpiGroups = 4;
+constexpr int kTcThreads = 32 * (kProdWarps + kMmaWarps + 4 * kEpiGroups);
 
 template <int M>
 struct TcCfg {
@@ -48,6 +54,8 @@ struct TcCfg {
   static constexpr int kStageBytes = 2 * kHalfBytes;
   static constexpr int kKronBytes = 2 * KA * NFP * 128;  // hi and lo
   static constexpr int kStages = (kStageBytes <= 16384) ? 8 : 5;
+  static constexpr int kAccCols = (NFP <= 64) ? 64 : 128;   // TMEM columns per accumulator
+  static constexpr int kNumAcc = 512 / kAccCols;            // 8 or 4 accumulators in flight
   static constexpr int kBarrierOffset = kKronBytes + kStages * kStageBytes;
   static constexpr int kTotal = kBarrierOffset + 512 + 1024;
 };
@@ -70,6 +78,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
                           int* __restrict__ status) {
   using Cfg = TcCfg<M>;
   constexpr int kStages = Cfg::kStages;
+  constexpr int kNumAcc = Cfg::kNumAcc;
+  constexpr int kAccCols = Cfg::kAccCols;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* kron = smem;
@@ -86,6 +96,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
   const int lane = threadIdx.x & 31;
   const int CB = (C + 127) / 128;
   const long long num_units = (long long)pc * CB;
+  const long long u_begin = num_units * blockIdx.x / gridDim.x;
+  const uint32_t n_local = (uint32_t)(num_units * (blockIdx.x + 1) / gridDim.x - u_begin);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -94,7 +106,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(tmem_base_slot, kNumAcc * kAccCols);
+  if (warp == kProdWarps) tmem_alloc(tmem_base_slot, 512);
   // Rows NF .. KP-1 of every stage half are never written by the TMA boxes; the matching
   // Kronecker columns are zero, so the rows only have to be finite: clear them once.
   if constexpr (Cfg::KP > Cfg::NF) {
@@ -112,21 +124,22 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
   const uint32_t tmem_base = *tmem_base_slot;
   bool timed_out = false;
 
-  if (warp == 0) {
-    // ---------------- TMA producer
-    if (lane == 0) {
+  if (warp < kProdWarps) {
+    // ---------------- TMA producers
+    if (warp == 0 && lane == 0) {
       mbar_expect_tx(kron_bar, Cfg::kKronBytes);
       for (int b = 0; b < 2 * Cfg::KA; ++b)
         tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, &tmKron, kron_bar, 0, b * Cfg::NFP);
     }
-    uint32_t stage = 0, phase = 0;
-    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x) {
-      const int cblk = (int)(u % CB);
-      const long long p = p0 + u / CB;
-      const int tw = (int)(p % Tw);
-      const int th = (int)((p / Tw) % Th);
-      const int img = (int)(p / ((long long)Tw * Th));
-      if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+    // tile coordinates of this warp's first unit, then advanced kProdWarps units at a time
+    // without divisions
+    const long long ufirst = u_begin + warp;
+    int cblk = (int)(ufirst % CB);
+    const long long pfirst = p0 + ufirst / CB;
+    int tw = (int)(pfirst % Tw), th = (int)((pfirst / Tw) % Th), img = (int)(pfirst / ((long long)Tw * Th));
+    for (uint32_t local = warp; local < n_local && !timed_out; local += kProdWarps) {
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
       if (lane == 0) {
         uint8_t* dst = ring + (size_t)stage * Cfg::kStageBytes;
         mbar_expect_tx(&full_bar[stage], 2 * Cfg::NF * 128);
@@ -134,21 +147,26 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
         tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - 1, M * th - 1, img);
       }
       __syncwarp();
-      if (++stage == kStages) { stage = 0; phase ^= 1; }
+#pragma unroll
+      for (int s = 0; s < kProdWarps; ++s)
+        if (++cblk == CB) {
+          cblk = 0;
+          if (++tw == Tw) { tw = 0; if (++th == Th) { th = 0; ++img; } }
+        }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer
+  } else if (warp < kProdWarps + kMmaWarps) {
+    // ---------------- MMA issuers
     constexpr uint32_t idesc = umma_idesc_f16_amn(128, Cfg::NFP);
-    uint32_t stage = 0, phase = 0, local = 0;
-    if (!mbar_wait(kron_bar, 0, abort_flag)) timed_out = true;
-    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x, ++local) {
+    if (!mbar_wait_warp(kron_bar, 0, abort_flag)) timed_out = true;
+    const uint32_t sk = smem_u32(kron);
+    for (uint32_t local = warp - kProdWarps; local < n_local && !timed_out; local += kMmaWarps) {
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
-      if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
-      if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       if (lane == 0) {
         const uint32_t sa = smem_u32(ring + (size_t)stage * Cfg::kStageBytes);
-        const uint32_t sk = smem_u32(kron);
         const uint32_t tmem_d = tmem_base + acc * kAccCols;
 #pragma unroll
         for (int hl = 0; hl < 2; ++hl)
@@ -162,21 +180,18 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
         umma_commit(&tmem_full[acc]);
       }
       __syncwarp();
-      if (++stage == kStages) { stage = 0; phase ^= 1; }
     }
   } else {
-    // ---------------- epilogue: warps 2-5 take even units, warps 6-9 odd units.
+    // ---------------- epilogue
     const int quad = warp & 3;                    // the TMEM lane quadrant this warp may read
-    const int group = (warp - 2) >> 2;
+    const int group = (warp - kProdWarps - kMmaWarps) >> 2;
     const size_t f_stride = (size_t)pc_pad * C;
-    uint32_t local = 0;
-    for (long long u = blockIdx.x; u < num_units && !timed_out; u += gridDim.x, ++local) {
-      if ((int)(local & 1) != group) continue;
+    const long long ufirst = u_begin + group;
+    int cblk = (int)(ufirst % CB), pl = (int)(ufirst / CB);
+    for (uint32_t local = group; local < n_local && !timed_out; local += kEpiGroups) {
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
-      const int cblk = (int)(u % CB);
-      const int pl = (int)(u / CB);
       const int c = cblk * 128 + quad * 32 + lane;
-      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
       __half* dst = V + (size_t)pl * C + c;
@@ -195,12 +210,16 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
         }
         if (c < C) {
 #pragma unroll
-          for (int cc = 0; cc < kMaxCols; ++cc) {
-            const int f = col0 + cc;
-            if (f < Cfg::NF) dst[(size_t)f * f_stride] = __float2half_rn(__uint_as_float(r[cc]));
-          }
+          for (int cc = 0; cc < kMaxCols; ++cc)
+            if (col0 + cc < Cfg::NF) {
+              *dst = __float2half_rn(__uint_as_float(r[cc]));
+              dst += f_stride;
+            }
         }
       }
+#pragma unroll
+      for (int s = 0; s < kEpiGroups; ++s)
+        if (++cblk == CB) { cblk = 0; ++pl; }
     }
   }
 
@@ -210,9 +229,9 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kProdWarps) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kNumAcc * kAccCols);
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -269,9 +288,7 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return (int)cudaErrorUnknown;
   }
-  int dev = 0, sms = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = plan->sm_count;
   const long long units = (long long)pc * ((g.C + 127) / 128);
   const int grid = (int)(units < sms ? units : sms);
   input_transform_tc_kernel<M><<<grid, kTcThreads, Cfg::kTotal, stream>>>(

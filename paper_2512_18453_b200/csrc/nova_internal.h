@@ -42,6 +42,7 @@ struct nova_plan {
   void* kron_dev;                         // device table of the tensor-core input transform (may be null)
   int* status_dev;                        // device status word (null without a device)
   int device;                             // device that owns status_dev
+  int sm_count;                           // multiprocessors of that device
 };
 
 namespace nova {

@@ -387,6 +387,7 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
         cudaMemset(w, 0, sizeof(int));
         pl->status_dev = w;
         pl->device = dev;
+        cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev);
       }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
       if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
