@@ -50,8 +50,9 @@ enum {
   NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
   NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
   NOVA_GEMM_TCGEN05 = 2 << 8, /* force the tcgen05 tensor-core product kernel */
-  NOVA_TRANSFORM_SIMT = 1 << 10 /* evaluate the input transform on CUDA cores even where the
-                                   tensor-core formulation applies (testing) */
+  NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
+                                   where the tensor-core formulation applies, the output transform
+                                   without TMA staging (testing) */
 };
 
 enum {

@@ -130,7 +130,10 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
                      : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
-    if (launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, (flags & NOVA_RELU) ? 1 : 0, stream))
+    const int relu = (flags & NOVA_RELU) ? 1 : 0;
+    if ((p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
+            ? launch_output_transform_tma(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
+            : launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream))
       return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 3], s);
   }

@@ -73,6 +73,8 @@ size_t kron_table_halves(int m);
 void build_kron_table(const nova_plan* plan, unsigned short* out);
 int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y,
                             long long p0, int pc, int pc_pad, int relu, void* stream);
+int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void* M, void* y,
+                                long long p0, int pc, int pc_pad, int relu, void* stream);
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,
                      int nfreq, int pc, int pc_pad, int C, int K, void* stream);
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M,

@@ -1,0 +1,270 @@
+// Output transform Y = A^T M A (Section 2.1 step 4 in its 2-D nested form, Appendix B.5),
+// evaluated in float and rounded once to the storage type, with the transformed-domain
+// product M staged through shared memory by TMA.
+//
+// M is stored [n*n][K/4][pc_pad][4] floats (frequency, filter quad, tile, filter in quad).
+// One work unit = 8 consecutive tiles x 16 consecutive filters, all n*n frequencies: one TMA
+// box of n*n*4 rows of 128 bytes (128-byte swizzle).
+//   warp 0      TMA producer, one box per unit into a ring of stages.
+//   warps 1-12  three consumer groups of four warps, unit i by group i%3.  Warp w of a group
+//               owns tiles w and w+4 of the unit, a lane one (tile, filter): its n*n values sit
+//               in conflict-free banks (the swizzle separates tiles w and w+4), and a warp's
+//               store of one output pixel covers 16 consecutive filters (32 bytes) of two tiles.
+// The arithmetic is transform_math.cuh's (dense, or the shared even/odd sums of a symmetric
+// point set).  Every wait is bounded; on expiry the kernel records a status and drains.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+#include "sm100.cuh"
+#include "transform_math.cuh"
+
+namespace nova {
+namespace {
+using namespace sm100;
+using namespace xf;
+
+constexpr int kConsGroups = 3;
+constexpr int kOtThreads = 32 * (1 + 4 * kConsGroups);
+
+template <int M>
+struct OtCfg {
+  static constexpr int N = M + 2;
+  static constexpr int NF = N * N;
+  static constexpr int kStageBytes = NF * 512;        // NF * 4 rows of 128 bytes; a multiple of 1024
+  static constexpr int kStages = (200 * 1024 / kStageBytes) < 8 ? (200 * 1024 / kStageBytes) : 8;
+  static constexpr int kBarrierOffset = kStages * kStageBytes;
+  static constexpr int kTotal = kBarrierOffset + 256 + 1024;
+};
+
+template <int M, typename T, bool SYM>
+__global__ void __launch_bounds__(kOtThreads, 1)
+output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
+                            T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
+                            int pc_pad, int relu, int* __restrict__ status) {
+  using Cfg = OtCfg<M>;
+  constexpr int N = Cfg::N;
+  constexpr int kStages = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarrierOffset);
+  uint64_t* empty_bar = full_bar + kStages;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kStages);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int KG = (K + 15) >> 4;                       // filter groups of 16
+  const int TG = pc_pad >> 3;                         // tile groups of 8 (pc_pad is a multiple of 128)
+  const long long num_units = (long long)TG * KG;
+  const long long u_begin = num_units * blockIdx.x / gridDim.x;
+  const uint32_t n_local = (uint32_t)(num_units * (blockIdx.x + 1) / gridDim.x - u_begin);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool timed_out = false;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    int kg = (int)(u_begin % KG), tg = (int)(u_begin / KG);
+    for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (lane == 0) {
+        mbar_expect_tx(&full_bar[stage], Cfg::kStageBytes);
+        tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, &tmM, &full_bar[stage], tg * 32, kg * 4, 0);
+      }
+      __syncwarp();
+      if (++kg == KG) { kg = 0; ++tg; }
+    }
+  } else {
+    // ---------------- consumers
+    const int group = (warp - 1) >> 2;
+    const int w = (warp - 1) & 3;
+    const int t = w + 4 * (lane >> 4);                // tile within the unit's 8
+    const int kq = (lane & 15) >> 2, kk = lane & 3;   // filter quad within the unit's 4, filter in quad
+    // byte offsets of this lane's value inside an even / odd frequency's 4 rows (128B swizzle:
+    // the 16-byte chunk index is XORed with the row index modulo 8)
+    const uint32_t off_even = kq * 128 + ((t ^ kq) << 4) + kk * 4;
+    const uint32_t off_odd = kq * 128 + ((t ^ (kq + 4)) << 4) + kk * 4;
+    const long long ufirst = u_begin + group;
+    int kg = (int)(ufirst % KG), tg = (int)(ufirst / KG);
+    for (uint32_t local = group; local < n_local && !timed_out; local += kConsGroups) {
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+      const uint8_t* sb = smem + (size_t)stage * Cfg::kStageBytes;
+      auto ldm = [&](int f) -> float {
+        return *reinterpret_cast<const float*>(sb + f * 512 + ((f & 1) ? off_odd : off_even));
+      };
+      auto load_row = [&](int xi, float (&z)[M]) {
+        float in[N];
+#pragma unroll
+        for (int nu = 0; nu < N; ++nu) in[nu] = ldm(xi * N + nu);
+        at_apply<M, SYM, float>(cf, in, z);
+      };
+      float Y[M][M];
+      if constexpr (!SYM) {
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+          for (int j = 0; j < M; ++j) Y[i][j] = 0.f;
+#pragma unroll
+        for (int xi = 0; xi < N; ++xi) {
+          float z[M];
+          load_row(xi, z);
+#pragma unroll
+          for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = 0; j < M; ++j) Y[i][j] = fmaf(cf.AT[i][xi], z[j], Y[i][j]);
+        }
+      } else {
+        // A^T column 0 is e_0 and column n-1 is e_{m-1}; columns +a / -a share |coefficients|.
+        {
+          float zp[M], zm[M];
+          load_row(1, zp);
+          load_row(2, zm);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
+#pragma unroll
+            for (int i = 0; i < M; ++i) Y[i][j] = cf.AT[i][1] * ((i & 1) ? d : s);
+          }
+        }
+#pragma unroll
+        for (int q = 3; q < N - 1; q += 2) {
+          float zp[M], zm[M];
+          load_row(q, zp);
+          load_row(q + 1, zm);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
+#pragma unroll
+            for (int i = 0; i < M; ++i) Y[i][j] = fmaf(cf.AT[i][q], (i & 1) ? d : s, Y[i][j]);
+          }
+        }
+        {
+          float z0[M], zi[M];
+          load_row(0, z0);
+          load_row(N - 1, zi);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            Y[0][j] += z0[j];
+            Y[M - 1][j] += zi[j];
+          }
+        }
+      }
+      // the stage's values are all in registers: hand it back to the producer
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty_bar[stage]);
+
+      const int pl = tg * 8 + t;
+      const int k = kg * 16 + (lane & 15);
+      if (pl < pc && k < K) {
+        const unsigned p = (unsigned)(p0 + pl);
+        const unsigned tw = p % (unsigned)Tw, q2 = p / (unsigned)Tw;
+        const unsigned th = q2 % (unsigned)Th, img = q2 / (unsigned)Th;
+        const int h0 = M * (int)th, w0 = M * (int)tw;
+        T* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+          if (h0 + i >= H) continue;
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            if (w0 + j >= W) continue;
+            float v = Y[i][j];
+            if (relu) v = v < 0.f ? 0.f : v;          // NaN and +inf pass through
+            vstore(dst + ((size_t)i * W + j) * K, v);
+          }
+        }
+      }
+#pragma unroll
+      for (int s = 0; s < kConsGroups; ++s)
+        if (++kg == KG) { kg = 0; ++tg; }
+    }
+  }
+
+  if (timed_out) {
+    *abort_flag = 1;
+    if (lane == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+template <int M, typename T, bool SYM>
+int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
+               int pc_pad, int relu, cudaStream_t stream) {
+  using Cfg = OtCfg<M>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
+    if (e != cudaSuccess) return (int)e;
+    attr_set = true;
+  }
+  const long long units = (long long)(pc_pad / 8) * ((g.K + 15) / 16);
+  const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
+  output_transform_tma_kernel<M, T, SYM><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
+      tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev);
+  return (int)cudaGetLastError();
+}
+
+template <int M>
+int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0, int pc, int pc_pad,
+             int relu, cudaStream_t stream) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return (int)cudaErrorUnknown;
+  CUtensorMap tmM;
+  const int k4 = g.K / 4;
+  cuuint64_t dims[3] = {(cuuint64_t)pc_pad * 4, (cuuint64_t)k4, (cuuint64_t)(g.n * g.n)};
+  cuuint64_t strides[2] = {(cuuint64_t)pc_pad * 16, (cuuint64_t)k4 * pc_pad * 16};
+  cuuint32_t box[3] = {32, 4, (cuuint32_t)(g.n * g.n)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  if (enc(&tmM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(Mb), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return (int)cudaErrorUnknown;
+  const bool f32 = plan->mode == NOVA_FP32;
+  if (plan->symmetric)
+    return f32 ? launch_one<M, float, true>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
+               : launch_one<M, __half, true>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
+  return f32 ? launch_one<M, float, false>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
+             : launch_one<M, __half, false>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
+}
+
+}  // namespace
+
+int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0,
+                                int pc, int pc_pad, int relu, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  switch (plan->m) {
+    case 2: return launch_m<2>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
+    case 4: return launch_m<4>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
+    case 6: return launch_m<6>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
+    case 8: return launch_m<8>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
+  }
+  return (int)cudaErrorInvalidValue;
+}
+
+}  // namespace nova
