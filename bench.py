@@ -225,6 +225,10 @@ def run_ours(args):
         else int(args.workspace_mb * (1 << 20))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     flags = {"auto": 0, "tcgen05": nv.GEMM_TCGEN05, "simt": nv.GEMM_SIMT}[args.gemm]
+    if args.fused:
+        flags |= nv.FUSED
+    if args.split:
+        plan.set_role_split(*[int(v) for v in args.split.split(",")])
     launches = plan.launch_count(c.N, c.H, c.W, c.C, c.K, ws_bytes, flags)
 
     # S1, once per layer: timed on its own
@@ -312,7 +316,8 @@ def run_ours(args):
         return
 
     peaks = read_peaks()
-    chunks = launches // 3
+    fused = launches == 1
+    chunks = 1 if fused else launches // 3
     names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
     n2 = (c.m + 2) ** 2
     elt = 2
@@ -324,6 +329,12 @@ def run_ours(args):
     ]
     dom = max(range(3), key=lambda i: kms[i])
     bound, work = alg[dom]
+    if fused:
+        # one kernel does the whole step: its work is the path's (the larger of the two ceilings)
+        names = ["-", "fused_conv (input transform | tcgen05 product | output transform roles)", "-"]
+        t_tensor = actual / (peaks["tflops_burst"] * 1e12)
+        t_hbm = min_bytes / (peaks["hbm_gbs"] * 1e9)
+        bound, work = ("tensor", actual) if t_tensor > t_hbm else ("hbm", min_bytes)
     dur_launch = kms[dom] * 1e-3 / chunks
     if bound == "tensor":
         achieved, peak, runit = work / chunks / dur_launch / 1e12, peaks["tflops_burst"], "TFLOP/s"
@@ -348,7 +359,7 @@ def run_ours(args):
                           "frac": roof_s / (ms_per_step * 1e-3), "peaks": peaks["source"],
                           "tensor_us": actual / (peaks["tflops_burst"] * 1e12) * 1e6,
                           "hbm_us": min_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
-        "kernels_ms_per_step": dict(zip(names, kms)),
+        "kernels_ms_per_step": {n_: v for n_, v in zip(names, kms) if n_ != "-"},
         "filter_transform_ms": filter_ms,
         "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
                      "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
@@ -378,6 +389,8 @@ def main():
     ap.add_argument("--gemm", default="auto", choices=["auto", "tcgen05", "simt"])
     ap.add_argument("--workspace-mb", type=float, default=None)
     ap.add_argument("--launch", default="graph", choices=["graph", "direct"])
+    ap.add_argument("--fused", action="store_true", help="the single role-specialised kernel instead of one kernel per step")
+    ap.add_argument("--split", default="", help="CTAs for the input-transform and product roles, e.g. 30,60")
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -50,6 +50,9 @@ enum {
   NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
   NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
   NOVA_GEMM_TCGEN05 = 2 << 8, /* force the tcgen05 tensor-core product kernel */
+  NOVA_FUSED = 1 << 11,     /* run the three steps as ONE persistent kernel whose CTAs are specialised
+                               by role and exchange tiles through L2-resident rings (half mode, C >= 64;
+                               otherwise ignored); the default is one kernel per step */
   NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
                                    where the tensor-core formulation applies, the output transform
                                    without TMA staging (testing) */
@@ -105,6 +108,11 @@ int nova_plan_get_device_tables(const nova_plan* plan, float* AT_host, float* G_
  * of each +-pair and skip the structural zeros (Appendix A, "symmetric point sets").
  * Any other set keeps the caller's order and dense transforms.  Either pointer may be null. */
 int nova_plan_frequency_order(const nova_plan* plan, int* perm_host, int* symmetric_host);
+
+/* Tuning: how many CTAs of the single-kernel path run the input transform and the
+ * transformed-domain product (the remaining ones run the output transform); 0, 0 restores
+ * the default split.  Not thread-safe against concurrent nova_conv2d_fwd on the same plan. */
+int nova_plan_set_role_split(nova_plan* plan, int n_input, int n_product);
 
 /* kappa_2 = sigma_max/sigma_min of the Vandermonde matrix V_ij = a_i^j over the
  * n-1 finite points only (Section 2.2, "Vandermonde Conditioning"). */

@@ -11,13 +11,14 @@ RELU = 1
 GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
 TRANSFORM_SIMT = 1 << 10
+FUSED = 1 << 11
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
-    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order",
+    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split",
 )
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -55,6 +56,8 @@ def lib():
     L.nova_plan_get_device_tables.restype = i
     L.nova_plan_frequency_order.argtypes = [vp, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.nova_plan_frequency_order.restype = i
+    L.nova_plan_set_role_split.argtypes = [vp, i, i]
+    L.nova_plan_set_role_split.restype = i
     L.nova_plan_kappa.argtypes = [vp, dp]
     L.nova_plan_kappa.restype = i
     L.nova_filter_transform_bytes.argtypes = [vp, i, i]
@@ -152,6 +155,9 @@ class Plan:
         sym = ctypes.c_int()
         _check(lib().nova_plan_frequency_order(self._h, perm, ctypes.byref(sym)), "nova_plan_frequency_order")
         return list(perm), bool(sym.value)
+
+    def set_role_split(self, n_input, n_product):
+        _check(lib().nova_plan_set_role_split(self._h, n_input, n_product), "nova_plan_set_role_split")
 
     def kappa(self):
         k = ctypes.c_double()

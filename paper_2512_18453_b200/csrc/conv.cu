@@ -14,7 +14,7 @@ namespace nova {
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr size_t kTargetChunkBytes = (size_t)64 << 20;
+constexpr size_t kTargetChunkBytes = (size_t)1 << 30;   // one chunk unless the problem is huge: fewest launches
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Chunking {
@@ -50,6 +50,23 @@ bool shape_ok(int N, int H, int W, int C, int K) {
   return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
 }
 bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// The single-kernel path applies in half mode with the tensor-core transforms, when the
+// scratch holds a ring of at least two 128-tile blocks (or all of them).  *R = ring length.
+bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R) {
+  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev) return false;
+  if (!(flags & NOVA_FUSED) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT))) return false;
+  if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
+  const long long NB = (g.P + 127) / 128;
+  if (bytes < 2 * kAlign) return false;
+  long long r = (long long)((bytes - 2 * kAlign) / fused_block_bytes(p, g.C, g.K));
+  if (r > NB) r = NB;
+  if (r < 2 && r < NB) return false;
+  if (r < 1) return false;
+  if (r > 64) r = 64;
+  *R = (int)r;
+  return true;
+}
 
 bool use_tcgen05(const nova_plan* p, int flags) {
   if (p->mode == NOVA_FP32) return false;
@@ -94,6 +111,8 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
   (void)flags;
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
   Geom g = make_geom(p, N, H, W, C, K);
+  int R = 0;
+  if (fused_applies(p, g, workspace_bytes, flags, &R)) return 1;
   Chunking c;
   if (!choose_chunking(p, g, workspace_bytes, &c)) return NOVA_ERR_WORKSPACE;
   return 3 * c.chunks;
@@ -109,6 +128,14 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if ((flags & NOVA_GEMM_TCGEN05) && p->mode == NOVA_FP32) return NOVA_ERR_UNSUPPORTED;
   Geom g = make_geom(p, N, H, W, C, K);
+  int R = 0;
+  if (fused_applies(p, g, ws_bytes, flags, &R)) {
+    cudaStream_t s = (cudaStream_t)stream;
+    if (ev) cudaEventRecord(ev[1], s);
+    const int e = launch_fused_conv(p, g, x, U, y, ws, R, (flags & NOVA_RELU) ? 1 : 0, stream);
+    if (ev) cudaEventRecord(ev[2], s);
+    return e ? NOVA_ERR_CUDA : NOVA_OK;
+  }
   Chunking c;
   if (!choose_chunking(p, g, ws_bytes, &c)) return NOVA_ERR_WORKSPACE;
   const bool tc = use_tcgen05(p, flags);
@@ -153,13 +180,16 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   if (!kernel_ms) return NOVA_ERR_INVALID_ARG;
   const int launches = nova_conv2d_launch_count(p, N, H, W, C, K, ws_bytes, flags);
   if (launches < 0) return launches;
-  const int chunks = launches / 3;
+  const bool fused = launches == 1;
+  const int chunks = fused ? 1 : launches / 3;
   cudaEvent_t* ev = new cudaEvent_t[4 * chunks];
   for (int i = 0; i < 4 * chunks; ++i) cudaEventCreate(&ev[i]);
   int st = conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, ev);
   if (st == NOVA_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st = NOVA_ERR_CUDA;
   kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
-  if (st == NOVA_OK)
+  if (st == NOVA_OK && fused) {
+    cudaEventElapsedTime(&kernel_ms[1], ev[1], ev[2]);      // the one kernel does all three steps
+  } else if (st == NOVA_OK)
     for (int c = 0; c < chunks; ++c)
       for (int k = 0; k < 3; ++k) {
         float ms = 0.f;

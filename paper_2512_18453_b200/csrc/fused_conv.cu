@@ -1,0 +1,768 @@
+// The whole forward convolution (Section 2.1 steps 1, 3, 4 in their 2-D nested form,
+// Appendix B.5) as ONE persistent kernel whose CTAs are specialised by role and exchange
+// work through rings of transformed tiles that stay in the L2 cache:
+//
+//   role I  (nI CTAs)  input transform on the tensor cores, x -> V ring       (see input_transform_tc.cu)
+//   role G  (nG CTAs)  transformed-domain product, V ring x U -> M ring        (see gemm_tcgen05.cu)
+//   role O  (the rest) output transform, M ring -> y                           (see output_transform_tma.cu)
+//
+// The tiles are grouped in blocks of 128; the rings hold R blocks (row = tile mod 128 R).
+// Three counters per block order the roles:
+//   v_ready[b]  += 1 by every epilogue warp of role I after its stores of a unit of block b
+//   g_done[b]   += 1 by every epilogue warp of role G after its stores of an item of block b
+//   o_done[b]   += 1 by every consumer warp of role O after it has read a unit of block b
+// and the TMA producer of a role waits, before it loads anything of block b, for
+//   role I: g_done[b-R] complete (the V rows are free again);
+//   role G: v_ready[b] complete and o_done[b-R] complete (the M rows are free again);
+//   role O: g_done[b] complete.
+// Every wait names a block that precedes b in each role's own order, every CTA walks its
+// role's work in increasing block order (work item = rank + j * role size), and all CTAs are
+// co-resident (cooperative launch, one CTA per SM), so the oldest unfinished block can always
+// make progress.  All waits are bounded; one that expires sets a flag every CTA polls.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+#include "sm100.cuh"
+#include "transform_math.cuh"
+
+namespace nova {
+namespace {
+using namespace sm100;
+using namespace xf;
+
+constexpr int kFusedThreads = 416;     // 13 warps: the largest role (O) needs them all
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;
+constexpr int kGemmStages = 4;
+constexpr uint32_t kCtrSpinLimit = 1u << 20;
+
+struct RingParams {
+  uint32_t* v_ready;     // [NB]
+  uint32_t* g_done;      // [NB]
+  uint32_t* o_done;      // [NB]
+  int* abort_all;        // set by any CTA that gives up
+  int R;                 // ring length in 128-tile blocks
+  int P;                 // tiles
+  int nI, nG;            // CTAs of role I and G; the rest are role O
+};
+
+struct ConvShape {
+  int H, W, C, K, Th, Tw, relu;
+};
+
+// ---------------------------------------------------------------- counters
+__device__ __forceinline__ bool ctr_wait(const uint32_t* ctr, uint32_t target, volatile int* abort_flag,
+                                         const int* abort_all) {
+  for (uint32_t i = 0; i < kCtrSpinLimit; ++i) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if (v >= target) return true;
+    if ((i & 31u) == 31u && (*abort_flag || *reinterpret_cast<const volatile int*>(abort_all))) return false;
+    __nanosleep(64);
+  }
+  return false;
+}
+__device__ __forceinline__ bool ctr_wait_warp(const uint32_t* ctr, uint32_t target, volatile int* abort_flag,
+                                              const int* abort_all) {
+  uint32_t ok = 1;
+  if ((threadIdx.x & 31) == 0) ok = ctr_wait(ctr, target, abort_flag, abort_all) ? 1u : 0u;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Called by all lanes of a warp after their global stores (or shared-memory reads) of a unit.
+__device__ __forceinline__ void ctr_signal(uint32_t* ctr) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) {
+    __threadfence();
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+  }
+}
+__device__ __forceinline__ void async_proxy_acquire() {
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  tmem_ld16(taddr, r);
+  tmem_ld16(taddr + 16, r + 16);
+}
+
+// ---------------------------------------------------------------- configuration
+template <int M>
+struct ICfg {
+  static constexpr int N = M + 2;
+  static constexpr int NF = N * N;
+  static constexpr int KP = (NF + 15) / 16 * 16;
+  static constexpr int NFP = KP;
+  static constexpr int KA = (KP + 63) / 64;
+  static constexpr int kHalfBytes = KP * 128;
+  static constexpr int kStageBytes = 2 * kHalfBytes;
+  static constexpr int kKronBytes = 2 * KA * NFP * 128;
+  static constexpr int kStages = (kStageBytes <= 16384) ? 6 : 2;
+  static constexpr int kAccCols = (NFP <= 64) ? 64 : 128;
+  static constexpr int kNumAcc = 512 / kAccCols;
+  static constexpr int kProd = 2, kMma = 2, kEpi = 2;       // producer warps, issuer warps, epilogue groups
+  // epilogue staging: per warp two buffers of [NF frequencies][32 channels] halves
+  static constexpr int kOutBufBytes = (NF * 64 + 127) / 128 * 128;
+  static constexpr int kOutOffset = kKronBytes + kStages * kStageBytes;
+  static constexpr int kBytes = kOutOffset + 4 * kEpi * 2 * kOutBufBytes;
+  // a slot of a ring is always handled by the same warp (group): see the note in input_transform_tc.cu
+  static_assert(kStages % kProd == 0 && kStages % kMma == 0 && kNumAcc % kMma == 0 && kNumAcc % kEpi == 0, "rings");
+};
+template <int BLOCK_N>
+struct GCfg {
+  static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
+  static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBytes = kGemmStages * kStageBytes;
+};
+template <int M>
+struct OCfg {
+  static constexpr int N = M + 2;
+  static constexpr int NF = N * N;
+  static constexpr int kStageBytes = NF * 512;
+  static constexpr int kGroups = 3;
+  static constexpr int kStages = ((200 * 1024 / kStageBytes) >= 6 ? 6 : 3);
+  static constexpr int kBytes = kStages * kStageBytes;
+  static_assert(kStages % kGroups == 0, "stage ring");
+};
+constexpr int cmax(int a, int b) { return a > b ? a : b; }
+template <int M, int BLOCK_N>
+struct FusedCfg {
+  static constexpr int kDataBytes = cmax(ICfg<M>::kBytes, cmax(GCfg<BLOCK_N>::kBytes, OCfg<M>::kBytes));
+  static constexpr int kBarrierOffset = kDataBytes;
+  static constexpr int kTotal = kBarrierOffset + 512 + 1024;
+};
+
+// ---------------------------------------------------------------- role I
+template <int M>
+__device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
+                                           volatile int* abort_flag, const CUtensorMap* tmX,
+                                           const CUtensorMap* tmKron, const CUtensorMap* tmVst,
+                                           const ConvShape& cs, const RingParams& rp, int rank, bool& timed_out) {
+  using Cfg = ICfg<M>;
+  constexpr int kStages = Cfg::kStages, kNumAcc = Cfg::kNumAcc, kAccCols = Cfg::kAccCols;
+  uint8_t* kron = smem;
+  uint8_t* ring = smem + Cfg::kKronBytes;
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full = empty_bar + kStages;
+  uint64_t* tmem_empty = tmem_full + kNumAcc;
+  uint64_t* kron_bar = tmem_empty + kNumAcc;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int C = cs.C;
+  const unsigned CB = (unsigned)((C + 127) / 128);
+  const unsigned num_units = (unsigned)rp.P * CB;
+  const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + rp.nI - 1) / rp.nI : 0u;
+  const int RP = rp.R * 128;
+  const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((cs.K + 255) / 256) * 4u;   // see role G
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < kNumAcc; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    mbar_init(kron_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == Cfg::kProd) tmem_alloc(tmem_base_slot, 512);
+  if constexpr (Cfg::KP > Cfg::NF) {
+    constexpr int pad16 = (Cfg::KP - Cfg::NF) * 8;
+    for (int i = threadIdx.x; i < kStages * 2 * pad16; i += kFusedThreads) {
+      const int half = i / pad16, off = i % pad16;
+      *reinterpret_cast<uint4*>(ring + (size_t)half * Cfg::kHalfBytes + Cfg::NF * 128 + off * 16) =
+          make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  if (warp < Cfg::kProd) {
+    if (warp == 0 && lane == 0) {
+      mbar_expect_tx(kron_bar, Cfg::kKronBytes);
+      for (int b = 0; b < 2 * Cfg::KA; ++b)
+        tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, tmKron, kron_bar, 0, b * Cfg::NFP);
+    }
+    for (unsigned local = warp; local < n_local && !timed_out; local += Cfg::kProd) {
+      const unsigned u = rank + local * rp.nI;
+      const unsigned p = u / CB, cblk = u % CB;
+      const unsigned tw = p % (unsigned)cs.Tw, q2 = p / (unsigned)cs.Tw;
+      const unsigned th = q2 % (unsigned)cs.Th, img = q2 / (unsigned)cs.Th;
+      const int b = (int)(p >> 7);
+      if (b >= rp.R && !ctr_wait_warp(rp.g_done + (b - rp.R), g_target, abort_flag, rp.abort_all)) {
+        timed_out = true; break;
+      }
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (lane == 0) {
+        uint8_t* dst = ring + (size_t)stage * Cfg::kStageBytes;
+        mbar_expect_tx(&full_bar[stage], 2 * Cfg::NF * 128);
+        tma_load_4d(dst, tmX, &full_bar[stage], (int)cblk * 128, M * (int)tw - 1, M * (int)th - 1, (int)img);
+        tma_load_4d(dst + Cfg::kHalfBytes, tmX, &full_bar[stage], (int)cblk * 128 + 64, M * (int)tw - 1,
+                    M * (int)th - 1, (int)img);
+      }
+      __syncwarp();
+    }
+  } else if (warp < Cfg::kProd + Cfg::kMma) {
+    constexpr uint32_t idesc = umma_idesc_f16_amn(128, Cfg::NFP);
+    if (!mbar_wait_warp(kron_bar, 0, abort_flag)) timed_out = true;
+    const uint32_t sk = smem_u32(kron);
+    for (unsigned local = warp - Cfg::kProd; local < n_local && !timed_out; local += Cfg::kMma) {
+      const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t sa = smem_u32(ring + (size_t)stage * Cfg::kStageBytes);
+        const uint32_t tmem_d = tmem_base + acc * kAccCols;
+#pragma unroll
+        for (int hl = 0; hl < 2; ++hl)
+#pragma unroll
+          for (int ks = 0; ks < Cfg::KP / 16; ++ks) {
+            const uint64_t ad = umma_desc_mn_sw128(sa + ks * 2048, Cfg::kHalfBytes);
+            const uint64_t bd = umma_desc_sw128(sk + (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
+            umma_f16(tmem_d, ad, bd, idesc, (hl > 0 || ks > 0) ? 1u : 0u);
+          }
+        umma_commit(&empty_bar[stage]);
+        umma_commit(&tmem_full[acc]);
+      }
+      __syncwarp();
+    }
+  } else if (warp < Cfg::kProd + Cfg::kMma + 4 * Cfg::kEpi) {
+    // Epilogue.  A warp turns its 32 channels x NF frequencies into a [NF][32] half tile in
+    // shared memory and TMA-stores it (one instruction per unit) to V[f][row][c0..c0+31]; the
+    // store clips channels >= C.  The block counter is raised once the store is complete,
+    // one unit later, so the warp never waits for its own store.
+    const int quad = warp & 3;
+    const int ew = warp - Cfg::kProd - Cfg::kMma;          // epilogue warp index
+    const int group = ew >> 2;
+    uint8_t* out0 = smem + Cfg::kOutOffset + (size_t)ew * 2 * Cfg::kOutBufBytes;
+    int pending_block = -1;
+    uint32_t n_mine = 0;
+    for (unsigned local = group; local < n_local && !timed_out; local += Cfg::kEpi, ++n_mine) {
+      const unsigned u = rank + local * rp.nI;
+      const unsigned p = u / CB, cblk = u % CB;
+      const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
+      const int c0 = (int)cblk * 128 + quad * 32;
+      if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
+      uint8_t* buf = out0 + (n_mine & 1) * Cfg::kOutBufBytes;
+      if (lane == 0) bulk_wait_read<1>();                  // the store that last read this buffer is done with it
+      __syncwarp();
+      __half* mine = reinterpret_cast<__half*>(buf) + lane;
+#pragma unroll
+      for (int col0 = 0; col0 < Cfg::NFP; col0 += 64) {
+        constexpr int kMaxCols = 64;
+        uint32_t r[kMaxCols];
+#pragma unroll
+        for (int cc = 0; cc < kMaxCols; cc += 16)
+          if (col0 + cc < Cfg::NFP) tmem_ld16(taddr + col0 + cc, r + cc);
+        tmem_ld_wait();
+        if (col0 + 64 >= Cfg::NFP) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+        }
+#pragma unroll
+        for (int cc = 0; cc < kMaxCols; ++cc)
+          if (col0 + cc < Cfg::NF) mine[(col0 + cc) * 32] = __float2half_rn(__uint_as_float(r[cc]));
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if (c0 < C) tma_store_3d(tmVst, buf, c0, (int)(p % (unsigned)RP), 0);
+        bulk_commit();
+        if (pending_block >= 0) {
+          bulk_wait_done<1>();                             // the previous unit's store is complete
+          __threadfence();
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(rp.v_ready + pending_block) : "memory");
+        }
+      }
+      pending_block = (int)(p >> 7);
+    }
+    if (lane == 0) {
+      bulk_wait_done<0>();
+      if (pending_block >= 0 && !timed_out) {
+        __threadfence();
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(rp.v_ready + pending_block) : "memory");
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == Cfg::kProd) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------- role G
+template <int NF, int BLOCK_N>
+__device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
+                                          volatile int* abort_flag, const CUtensorMap* tmV,
+                                          const CUtensorMap* tmU, float* __restrict__ Mo, const ConvShape& cs,
+                                          const RingParams& rp, int rank, bool& timed_out) {
+  using L = GCfg<BLOCK_N>;
+  constexpr int kStages = kGemmStages;
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full = empty_bar + kStages;
+  uint64_t* tmem_empty = tmem_full + 2;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int C = cs.C, K = cs.K;
+  const unsigned NB = (unsigned)((rp.P + 127) >> 7);
+  const unsigned num_kb = (unsigned)((K + BLOCK_N - 1) / BLOCK_N);
+  const int num_ks = (C + BLOCK_K - 1) / BLOCK_K;
+  const unsigned per_block = (unsigned)NF * num_kb;
+  const unsigned num_items = NB * per_block;
+  const unsigned n_local = (num_items > (unsigned)rank) ? (num_items - rank + rp.nG - 1) / rp.nG : 0u;
+  const int RP = rp.R * 128;
+  const unsigned CB = (unsigned)((C + 127) / 128);
+  const uint32_t o_target = 16u * (uint32_t)((K + 15) >> 4) * 4u;     // see role O
+  constexpr uint32_t kTmemCols = (2 * BLOCK_N < 32) ? 32 : 2 * BLOCK_N;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_base_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  if (warp == 0) {
+    uint32_t stage = 0, phase = 0;
+    for (unsigned local = 0; local < n_local && !timed_out; ++local) {
+      const unsigned it = rank + local * rp.nG;
+      const unsigned pb = it / per_block, rem = it % per_block;
+      const unsigned f = rem / num_kb, kb = rem % num_kb;
+      int tiles = rp.P - (int)pb * 128;
+      tiles = tiles > 128 ? 128 : tiles;
+      if (!ctr_wait_warp(rp.v_ready + pb, (uint32_t)tiles * CB * 4u, abort_flag, rp.abort_all)) {
+        timed_out = true; break;
+      }
+      if ((int)pb >= rp.R && !ctr_wait_warp(rp.o_done + (pb - rp.R), o_target, abort_flag, rp.abort_all)) {
+        timed_out = true; break;
+      }
+      async_proxy_acquire();
+      const int row0 = (int)(pb % (unsigned)rp.R) * 128;
+      for (int ks = 0; ks < num_ks; ++ks) {
+        if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+        if (lane == 0) {
+          uint8_t* sa = smem + stage * L::kStageBytes;
+          uint8_t* sb = sa + L::kABytes;
+          mbar_expect_tx(&full_bar[stage], L::kStageBytes);
+          tma_load_3d(sa, tmV, &full_bar[stage], ks * BLOCK_K, row0, (int)f);
+          tma_load_3d(sb, tmU, &full_bar[stage], ks * BLOCK_K, (int)kb * BLOCK_N, (int)f);
+        }
+        __syncwarp();
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = umma_idesc_f16(BLOCK_M, BLOCK_N);
+    uint32_t stage = 0, phase = 0;
+    for (unsigned local = 0; local < n_local && !timed_out; ++local) {
+      const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+      if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      const uint32_t tmem_d = tmem_base + acc * BLOCK_N;
+      for (int ks = 0; ks < num_ks; ++ks) {
+        if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / 16; ++k) {
+            const uint64_t ad = umma_desc_sw128(sa + k * 32);
+            const uint64_t bd = umma_desc_sw128(sb + k * 32);
+            umma_f16(tmem_d, ad, bd, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[stage]);
+          if (ks == num_ks - 1) umma_commit(&tmem_full[acc]);
+        }
+        __syncwarp();
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp < 6) {
+    const int quad = warp & 3;
+    const int k4 = K >> 2;
+    for (unsigned local = 0; local < n_local && !timed_out; ++local) {
+      const unsigned it = rank + local * rp.nG;
+      const unsigned pb = it / per_block, rem = it % per_block;
+      const unsigned f = rem / num_kb, kb = rem % num_kb;
+      const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+      if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      const int row = (int)(pb % (unsigned)rp.R) * 128 + quad * 32 + lane;
+      const int k_left = K - (int)kb * BLOCK_N;
+      float* dst = Mo + (((size_t)f * k4 + (size_t)((int)kb * BLOCK_N >> 2)) * RP + row) * 4;
+      const size_t q_stride = (size_t)RP * 4;
+#pragma unroll 1
+      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + cb, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (cb + 4 * j < k_left)
+            *reinterpret_cast<uint4*>(dst + (size_t)((cb >> 2) + j) * q_stride) =
+                make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+      ctr_signal(rp.g_done + pb);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------- role O
+template <int M, bool SYM>
+__device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volatile int* abort_flag,
+                                            const CUtensorMap* tmM, const Coefs& cf, __half* __restrict__ y,
+                                            const ConvShape& cs, const RingParams& rp, int rank, int size,
+                                            bool& timed_out) {
+  using Cfg = OCfg<M>;
+  constexpr int N = Cfg::N;
+  constexpr int kStages = Cfg::kStages;
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = full_bar + kStages;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int K = cs.K, H = cs.H, W = cs.W;
+  const unsigned KG = (unsigned)((K + 15) >> 4);
+  const unsigned NB = (unsigned)((rp.P + 127) >> 7);
+  const unsigned num_units = NB * 16u * KG;
+  const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + size - 1) / size : 0u;
+  const int RP = rp.R * 128;
+  const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((K + 255) / 256) * 4u;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    for (unsigned local = 0; local < n_local && !timed_out; ++local) {
+      const unsigned u = rank + local * size;
+      const unsigned tg = u / KG, kg = u % KG;
+      const unsigned b = tg >> 4;
+      if (!ctr_wait_warp(rp.g_done + b, g_target, abort_flag, rp.abort_all)) { timed_out = true; break; }
+      async_proxy_acquire();
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+      if (lane == 0) {
+        mbar_expect_tx(&full_bar[stage], Cfg::kStageBytes);
+        tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, tmM, &full_bar[stage],
+                    (int)((tg * 8u) % (unsigned)RP) * 4, (int)kg * 4, 0);
+      }
+      __syncwarp();
+    }
+  } else {
+    const int group = (warp - 1) >> 2;
+    const int w = (warp - 1) & 3;
+    const int t = w + 4 * (lane >> 4);
+    const int kq = (lane & 15) >> 2, kk = lane & 3;
+    const uint32_t off_even = kq * 128 + ((t ^ kq) << 4) + kk * 4;
+    const uint32_t off_odd = kq * 128 + ((t ^ (kq + 4)) << 4) + kk * 4;
+    for (unsigned local = group; local < n_local && !timed_out; local += Cfg::kGroups) {
+      const unsigned u = rank + local * size;
+      const unsigned tg = u / KG, kg = u % KG;
+      const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
+      if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+      const uint8_t* sb = smem + (size_t)stage * Cfg::kStageBytes;
+      auto ldm = [&](int f) -> float {
+        return *reinterpret_cast<const float*>(sb + f * 512 + ((f & 1) ? off_odd : off_even));
+      };
+      auto load_row = [&](int xi, float (&z)[M]) {
+        float in[N];
+#pragma unroll
+        for (int nu = 0; nu < N; ++nu) in[nu] = ldm(xi * N + nu);
+        at_apply<M, SYM, float>(cf, in, z);
+      };
+      float Y[M][M];
+      if constexpr (!SYM) {
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+          for (int j = 0; j < M; ++j) Y[i][j] = 0.f;
+#pragma unroll
+        for (int xi = 0; xi < N; ++xi) {
+          float z[M];
+          load_row(xi, z);
+#pragma unroll
+          for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = 0; j < M; ++j) Y[i][j] = fmaf(cf.AT[i][xi], z[j], Y[i][j]);
+        }
+      } else {
+        {
+          float zp[M], zm[M];
+          load_row(1, zp);
+          load_row(2, zm);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
+#pragma unroll
+            for (int i = 0; i < M; ++i) Y[i][j] = cf.AT[i][1] * ((i & 1) ? d : s);
+          }
+        }
+#pragma unroll
+        for (int q = 3; q < N - 1; q += 2) {
+          float zp[M], zm[M];
+          load_row(q, zp);
+          load_row(q + 1, zm);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
+#pragma unroll
+            for (int i = 0; i < M; ++i) Y[i][j] = fmaf(cf.AT[i][q], (i & 1) ? d : s, Y[i][j]);
+          }
+        }
+        {
+          float z0[M], zi[M];
+          load_row(0, z0);
+          load_row(N - 1, zi);
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            Y[0][j] += z0[j];
+            Y[M - 1][j] += zi[j];
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty_bar[stage]);
+      ctr_signal(rp.o_done + (tg >> 4));
+
+      const int pl = (int)tg * 8 + t;
+      const int k = (int)kg * 16 + (lane & 15);
+      if (pl < rp.P && k < K) {
+        const unsigned p = (unsigned)pl;
+        const unsigned tw = p % (unsigned)cs.Tw, q2 = p / (unsigned)cs.Tw;
+        const unsigned th = q2 % (unsigned)cs.Th, img = q2 / (unsigned)cs.Th;
+        const int h0 = M * (int)th, w0 = M * (int)tw;
+        __half* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+          if (h0 + i >= H) continue;
+#pragma unroll
+          for (int j = 0; j < M; ++j) {
+            if (w0 + j >= W) continue;
+            float v = Y[i][j];
+            if (cs.relu) v = v < 0.f ? 0.f : v;
+            vstore(dst + ((size_t)i * W + j) * K, v);
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int M, int BLOCK_N, bool SYM>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+fused_conv_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
+                  const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmVst,
+                  const __grid_constant__ Coefs cf, float* __restrict__ Mo, __half* __restrict__ y,
+                  const ConvShape cs, const RingParams rp, int* __restrict__ status) {
+  using F = FusedCfg<M, BLOCK_N>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + F::kBarrierOffset);
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 40);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+  if (threadIdx.x == 0) *abort_flag = 0;
+  __syncthreads();
+
+  bool timed_out = false;
+  const int b = blockIdx.x;
+  if (b < rp.nI)
+    role_input<M>(smem, bars, tmem_base_slot, abort_flag, &tmX, &tmKron, &tmVst, cs, rp, b, timed_out);
+  else if (b < rp.nI + rp.nG)
+    role_gemm<(M + 2) * (M + 2), BLOCK_N>(smem, bars, tmem_base_slot, abort_flag, &tmV, &tmU, Mo, cs, rp,
+                                          b - rp.nI, timed_out);
+  else
+    role_output<M, SYM>(smem, bars, abort_flag, &tmM, cf, y, cs, rp, b - rp.nI - rp.nG,
+                        (int)gridDim.x - rp.nI - rp.nG, timed_out);
+
+  if (timed_out) {
+    *abort_flag = 1;
+    if ((threadIdx.x & 31) == 0) {
+      atomicExch(rp.abort_all, 1);
+      atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+    }
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+bool encode(CUtensorMap* map, CUtensorMapDataType dt, int rank, const void* base, const cuuint64_t* dims,
+            const cuuint64_t* strides, const cuuint32_t* box, CUtensorMapL2promotion promo,
+            CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return enc(map, dt, rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             swz, promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int M, int BLOCK_N, bool SYM>
+int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* Vr,
+                   float* Mr, int R, int relu, cudaStream_t stream) {
+  using F = FusedCfg<M, BLOCK_N>;
+  constexpr int n = M + 2, NF = n * n;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(fused_conv_kernel<M, BLOCK_N, SYM>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, F::kTotal);
+    if (e != cudaSuccess) return (int)e;
+    attr_set = true;
+  }
+  const int RP = R * 128;
+  CUtensorMap tmX, tmK, tmV, tmU, tmM, tmVst;
+  const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  const CUtensorMapL2promotion p256 = CU_TENSOR_MAP_L2_PROMOTION_L2_256B, p128 = CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+    cuuint64_t strides[3] = {(cuuint64_t)g.C * 2, (cuuint64_t)g.W * g.C * 2, (cuuint64_t)g.H * g.W * g.C * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)n, (cuuint32_t)n, 1};
+    if (!encode(&tmX, f16, 4, x, dims, strides, box, p256)) return (int)cudaErrorUnknown;
+  }
+  {
+    using IC = ICfg<M>;
+    cuuint64_t dims[2] = {64, (cuuint64_t)(2 * IC::KA * IC::NFP)};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {64, (cuuint32_t)IC::NFP};
+    if (!encode(&tmK, f16, 2, plan->kron_dev, dims, strides, box, p256)) return (int)cudaErrorUnknown;
+  }
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)g.C, (cuuint64_t)RP, (cuuint64_t)NF};
+    cuuint64_t strides[2] = {(cuuint64_t)g.C * 2, (cuuint64_t)RP * g.C * 2};
+    cuuint32_t box[3] = {BLOCK_K, BLOCK_M, 1};
+    if (!encode(&tmV, f16, 3, Vr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
+    cuuint32_t sbox[3] = {32, 1, (cuuint32_t)NF};            // the epilogue's store box: [NF][1 row][32 channels]
+    if (!encode(&tmVst, f16, 3, Vr, dims, strides, sbox, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return (int)cudaErrorUnknown;
+  }
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)g.C, (cuuint64_t)g.K, (cuuint64_t)NF};
+    cuuint64_t strides[2] = {(cuuint64_t)g.C * 2, (cuuint64_t)g.K * g.C * 2};
+    cuuint32_t box[3] = {BLOCK_K, (cuuint32_t)BLOCK_N, 1};
+    if (!encode(&tmU, f16, 3, U, dims, strides, box, p256)) return (int)cudaErrorUnknown;
+  }
+  {
+    const int k4 = g.K / 4;
+    cuuint64_t dims[3] = {(cuuint64_t)RP * 4, (cuuint64_t)k4, (cuuint64_t)NF};
+    cuuint64_t strides[2] = {(cuuint64_t)RP * 16, (cuuint64_t)k4 * RP * 16};
+    cuuint32_t box[3] = {32, 4, (cuuint32_t)NF};
+    if (!encode(&tmM, f32, 3, Mr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
+  }
+  const int NB = (int)((g.P + 127) / 128);
+  uint32_t* ctr = plan->fused_ctr_dev;
+  if (cudaMemsetAsync(ctr, 0, (size_t)(3 * NB + 4) * sizeof(uint32_t), stream) != cudaSuccess)
+    return (int)cudaErrorUnknown;
+  RingParams rp;
+  rp.v_ready = ctr;
+  rp.g_done = ctr + NB;
+  rp.o_done = ctr + 2 * NB;
+  rp.abort_all = reinterpret_cast<int*>(ctr + 3 * NB);
+  rp.R = R;
+  rp.P = (int)g.P;
+  const int sms = plan->sm_count;
+  int nI = plan->fused_nI, nG = plan->fused_nG;
+  if (nI <= 0 || nG <= 0 || nI + nG >= sms) {         // default split of the SMs between the roles
+    nI = sms * 22 / 100;
+    nG = sms * 40 / 100;
+  }
+  rp.nI = nI;
+  rp.nG = nG;
+  ConvShape cs{g.H, g.W, g.C, g.K, g.Th, g.Tw, relu};
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)sms);
+  cfg.blockDim = dim3(kFusedThreads);
+  cfg.dynamicSmemBytes = F::kTotal;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;        // all CTAs co-resident, or the launch fails
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, fused_conv_kernel<M, BLOCK_N, SYM>, tmX, tmK, tmV, tmU, tmM, tmVst,
+                                 plan->kcoefs, Mr, (__half*)y, cs, rp, plan->status_dev);
+}
+
+template <int M>
+int launch_fused_m(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* Vr,
+                   float* Mr, int R, int relu, cudaStream_t s) {
+  if (plan->symmetric) return launch_fused_t<M, 256, true>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+  return launch_fused_t<M, 256, false>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+}
+
+}  // namespace
+
+size_t fused_block_bytes(const nova_plan* plan, int C, int K) {
+  return (size_t)plan->n * plan->n * 128 * ((size_t)C * 2 + (size_t)K * 4);
+}
+
+int launch_fused_conv(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* ws,
+                      int R, int relu, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t v_bytes = ((size_t)plan->n * plan->n * R * 128 * g.C * 2 + 255) / 256 * 256;
+  void* Vr = ws;
+  float* Mr = reinterpret_cast<float*>(static_cast<char*>(ws) + v_bytes);
+  switch (plan->m) {
+    case 2: return launch_fused_m<2>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+    case 4: return launch_fused_m<4>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+    case 6: return launch_fused_m<6>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+    case 8: return launch_fused_m<8>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+  }
+  return (int)cudaErrorInvalidValue;
+}
+
+}  // namespace nova

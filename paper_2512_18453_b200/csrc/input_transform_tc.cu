@@ -53,11 +53,23 @@ struct TcCfg {
   static constexpr int kHalfBytes = KP * 128;            // one 64-channel half of a stage
   static constexpr int kStageBytes = 2 * kHalfBytes;
   static constexpr int kKronBytes = 2 * KA * NFP * 128;  // hi and lo
-  static constexpr int kStages = (kStageBytes <= 16384) ? 8 : 5;
+  static constexpr int kStages = (kStageBytes <= 16384) ? 8 : 4;
   static constexpr int kAccCols = (NFP <= 64) ? 64 : 128;   // TMEM columns per accumulator
   static constexpr int kNumAcc = 512 / kAccCols;            // 8 or 4 accumulators in flight
   static constexpr int kBarrierOffset = kKronBytes + kStages * kStageBytes;
   static constexpr int kTotal = kBarrierOffset + 512 + 1024;
+};
+
+// Ring discipline: an mbarrier wait names a phase only by its parity, so a warp that could
+// get two phases ahead of a barrier would pass the wait early.  A warp is at most one phase
+// ahead of a barrier it waited on for its own previous use of the same slot; therefore every
+// slot (stage or accumulator) must always be handled by the same warp (group) of a role:
+// the ring lengths are multiples of the number of warps (groups) that share the ring.
+template <int M>
+struct TcCfgCheck {
+  static_assert(TcCfg<M>::kStages % kProdWarps == 0 && TcCfg<M>::kStages % kMmaWarps == 0, "stage ring");
+  static_assert(TcCfg<M>::kNumAcc % kMmaWarps == 0 && TcCfg<M>::kNumAcc % kEpiGroups == 0, "accumulator ring");
+  static constexpr bool ok = true;
 };
 
 template <int NR>
@@ -77,6 +89,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
                           __half* __restrict__ V, int C, int Th, int Tw, long long p0, int pc, int pc_pad,
                           int* __restrict__ status) {
   using Cfg = TcCfg<M>;
+  static_assert(TcCfgCheck<M>::ok, "");
   constexpr int kStages = Cfg::kStages;
   constexpr int kNumAcc = Cfg::kNumAcc;
   constexpr int kAccCols = Cfg::kAccCols;

@@ -33,7 +33,10 @@ struct OtCfg {
   static constexpr int N = M + 2;
   static constexpr int NF = N * N;
   static constexpr int kStageBytes = NF * 512;        // NF * 4 rows of 128 bytes; a multiple of 1024
-  static constexpr int kStages = (200 * 1024 / kStageBytes) < 8 ? (200 * 1024 / kStageBytes) : 8;
+  // a multiple of the number of consumer groups: a stage is always read by the same group, so
+  // no warp can get two phases ahead of a barrier it waits on by parity
+  static constexpr int kStages = ((200 * 1024 / kStageBytes) >= 6 ? 6 : 3);
+  static_assert(kStages % kConsGroups == 0, "stage ring");
   static constexpr int kBarrierOffset = kStages * kStageBytes;
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;
 };
@@ -242,7 +245,7 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
   cuuint32_t box[3] = {32, 4, (cuuint32_t)(g.n * g.n)};
   cuuint32_t estr[3] = {1, 1, 1};
   if (enc(&tmM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(Mb), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return (int)cudaErrorUnknown;
   const bool f32 = plan->mode == NOVA_FP32;

@@ -389,6 +389,14 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
         pl->device = dev;
         cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev);
       }
+      if (pl->status_dev) {
+        const int cap = 1 << 16;                       // blocks of 128 tiles
+        uint32_t* cd = nullptr;
+        if (cudaMalloc((void**)&cd, (size_t)(3 * cap + 4) * sizeof(uint32_t)) == cudaSuccess) {
+          pl->fused_ctr_dev = cd;
+          pl->fused_ctr_blocks = cap;
+        }
+      }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
       if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
         std::vector<unsigned short> img(nova::kron_table_halves(m));
@@ -410,6 +418,7 @@ extern "C" void nova_plan_destroy(nova_plan* plan) {
   if (!plan) return;
   if (plan->status_dev) cudaFree(plan->status_dev);
   if (plan->kron_dev) cudaFree(plan->kron_dev);
+  if (plan->fused_ctr_dev) cudaFree(plan->fused_ctr_dev);
   delete plan;
 }
 
@@ -440,6 +449,13 @@ extern "C" int nova_plan_frequency_order(const nova_plan* p, int* perm, int* sym
   if (perm)
     for (int i = 0; i < p->n; ++i) perm[i] = p->perm[i];
   if (symmetric) *symmetric = p->symmetric;
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_set_role_split(nova_plan* p, int n_input, int n_product) {
+  if (!p || n_input < 0 || n_product < 0) return NOVA_ERR_INVALID_ARG;
+  p->fused_nI = n_input;
+  p->fused_nG = n_product;
   return NOVA_OK;
 }
 

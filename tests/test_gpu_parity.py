@@ -160,6 +160,52 @@ def test_tensor_core_and_cuda_core_input_transforms_agree(kind, m, shape):
     assert conv.rel_l2(ya, yb) < 0.3 * eb
 
 
+@pytest.mark.parametrize("kind,m", [("std", 2), ("nova", 4), ("nova", 6), ("half", 6), ("nova", 8)])
+@pytest.mark.parametrize("shape,ws_blocks", [((2, 26, 26, 72, 136), None), ((3, 50, 50, 64, 64), 2),
+                                             ((1, 40, 47, 136, 264), 3), ((4, 33, 30, 64, 8), None)])
+def test_single_kernel_path_matches_three_kernel_path(kind, m, shape, ws_blocks):
+    """NOVA_FUSED runs the same arithmetic in one role-specialised kernel; with a ring of only
+    ws_blocks 128-tile blocks the roles have to recycle ring rows many times."""
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=480 + m)
+    pts = point_set(kind, m)
+    plan = nv.Plan(m, pts)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    U = plan.filter_transform(gd)
+    n = m + 2
+    nbytes = plan.workspace_bytes(N, H, W, C, K) if ws_blocks is None else \
+        ws_blocks * n * n * 128 * (2 * C + 4 * K) + 1024
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    assert plan.launch_count(N, H, W, C, K, nbytes, nv.FUSED) == 1
+    ya = torch.full((N, H, W, K), float("nan"), dtype=torch.float16, device="cuda")
+    yb = torch.full((N, H, W, K), float("nan"), dtype=torch.float16, device="cuda")
+    for _ in range(2):                                   # twice: the counters are reset per call
+        plan.conv2d(xd, U, y=ya, workspace=ws, flags=nv.FUSED)
+    plan.conv2d(xd, U, y=yb, workspace=torch.empty(plan.workspace_bytes(N, H, W, C, K), dtype=torch.uint8,
+                                                   device="cuda"))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert np.array_equal(ya.cpu().numpy(), yb.cpu().numpy())
+    check_fp16(ya.cpu().numpy(), x, g, m, pts)
+
+
+@pytest.mark.parametrize("kind,m,shape", [("nova", 8, (16, 28, 28, 512, 64)), ("nova", 4, (8, 40, 40, 256, 64)),
+                                          ("std", 2, (8, 32, 32, 128, 64))])
+def test_many_units_per_cta_in_every_ring(kind, m, shape):
+    """Every CTA of the transform kernels walks its stage and accumulator rings several times
+    (many units per CTA, several channel blocks): a slot must always come back to the same warp."""
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=490 + m)
+    pts = point_set(kind, m)
+    ya, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC)
+    yb, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.TRANSFORM_SIMT)
+    y1 = conv.direct_conv_fp64(x, g)
+    ea, eb = conv.rel_l2(ya, y1), conv.rel_l2(yb, y1)
+    assert abs(ea - eb) <= 0.05 * eb and conv.rel_l2(ya, yb) < 0.3 * eb
+    yc, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.FUSED)
+    assert np.array_equal(ya, yc)
+
+
 def test_ragged_last_row_block_after_full_blocks():
     """532 tiles = 4 full 128-row blocks + 20 rows, 36 x 5 work items on 148 SMs: a CTA
     that handles a full block and then the ragged one must not reuse an epilogue
