@@ -218,7 +218,7 @@ __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32
   } else if (warp < Cfg::kProd + Cfg::kMma) {
     constexpr uint32_t idesc = umma_idesc_f16_amn(128, Cfg::NFP);
     if (!mbar_wait_warp(kron_bar, 0, abort_flag)) timed_out = true;
-    const uint32_t sk = smem_u32(kron);
+    const uint64_t bd0 = umma_desc_sw128(smem_u32(kron));
     for (unsigned local = warp - Cfg::kProd; local < n_local && !timed_out; local += Cfg::kMma) {
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
@@ -228,13 +228,15 @@ __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32
       if (lane == 0) {
         const uint32_t sa = smem_u32(ring + (size_t)stage * Cfg::kStageBytes);
         const uint32_t tmem_d = tmem_base + acc * kAccCols;
+const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
 #pragma unroll
         for (int hl = 0; hl < 2; ++hl)
 #pragma unroll
           for (int ks = 0; ks < Cfg::KP / 16; ++ks) {
-            const uint64_t ad = umma_desc_mn_sw128(sa + ks * 2048, Cfg::kHalfBytes);
-            const uint64_t bd = umma_desc_sw128(sk + (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
-            umma_f16(tmem_d, ad, bd, idesc, (hl > 0 || ks > 0) ? 1u : 0u);
+            const uint64_t ad = umma_desc_advance(ad0, ks * 2048);
+            const uint64_t bd = umma_desc_advance(bd0, (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
+            if (hl == 0 && ks == 0) umma_f16_c<false>(tmem_d, ad, bd, idesc);
+            else umma_f16_c<true>(tmem_d, ad, bd, idesc);
           }
         umma_commit(&empty_bar[stage]);
         umma_commit(&tmem_full[acc]);
@@ -392,12 +394,11 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
         if (lane == 0) {
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
+const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
+          umma_f16(tmem_d, ad0, bd0, idesc, ks > 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BLOCK_K / 16; ++k) {
-            const uint64_t ad = umma_desc_sw128(sa + k * 32);
-            const uint64_t bd = umma_desc_sw128(sb + k * 32);
-            umma_f16(tmem_d, ad, bd, idesc, (ks > 0 || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < BLOCK_K / 16; ++k)
+            umma_f16_c<true>(tmem_d, umma_desc_advance(ad0, k * 32), umma_desc_advance(bd0, k * 32), idesc);
           umma_commit(&empty_bar[stage]);
           if (ks == num_ks - 1) umma_commit(&tmem_full[acc]);
         }

@@ -124,12 +124,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         if (lane == 0) {
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
+const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
+          umma_f16(tmem_d, ad0, bd0, idesc, ks > 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t ad = umma_desc_sw128(sa + k * UMMA_K * 2);
-            const uint64_t bd = umma_desc_sw128(sb + k * UMMA_K * 2);
-            umma_f16(tmem_d, ad, bd, idesc, (ks > 0 || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < BLOCK_K / 16; ++k)
+            umma_f16_c<true>(tmem_d, umma_desc_advance(ad0, k * 32), umma_desc_advance(bd0, k * 32), idesc);
           umma_commit(&empty_bar[stage]);                 // frees the smem stage when the MMAs retire
           if (ks == num_ks - 1) umma_commit(&tmem_full[acc]);
         }

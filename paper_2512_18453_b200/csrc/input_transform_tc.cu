@@ -171,7 +171,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
     // ---------------- MMA issuers
     constexpr uint32_t idesc = umma_idesc_f16_amn(128, Cfg::NFP);
     if (!mbar_wait_warp(kron_bar, 0, abort_flag)) timed_out = true;
-    const uint32_t sk = smem_u32(kron);
+    const uint64_t bd0 = umma_desc_sw128(smem_u32(kron));
     for (uint32_t local = warp - kProdWarps; local < n_local && !timed_out; local += kMmaWarps) {
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
@@ -181,13 +181,15 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
       if (lane == 0) {
         const uint32_t sa = smem_u32(ring + (size_t)stage * Cfg::kStageBytes);
         const uint32_t tmem_d = tmem_base + acc * kAccCols;
+const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
 #pragma unroll
         for (int hl = 0; hl < 2; ++hl)
 #pragma unroll
           for (int ks = 0; ks < Cfg::KP / 16; ++ks) {
-            const uint64_t ad = umma_desc_mn_sw128(sa + ks * 2048, Cfg::kHalfBytes);
-            const uint64_t bd = umma_desc_sw128(sk + (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
-            umma_f16(tmem_d, ad, bd, idesc, (hl > 0 || ks > 0) ? 1u : 0u);
+            const uint64_t ad = umma_desc_advance(ad0, ks * 2048);
+            const uint64_t bd = umma_desc_advance(bd0, (hl * Cfg::KA + ks / 4) * Cfg::NFP * 128 + (ks % 4) * 32);
+            if (hl == 0 && ks == 0) umma_f16_c<false>(tmem_d, ad, bd, idesc);
+            else umma_f16_c<true>(tmem_d, ad, bd, idesc);
           }
         umma_commit(&empty_bar[stage]);
         umma_commit(&tmem_full[acc]);
