@@ -79,6 +79,15 @@ __device__ __forceinline__ void ctr_signal(uint32_t* ctr) {
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
   }
 }
+// The same for n units at once.
+__device__ __forceinline__ void ctr_signal_n(uint32_t* ctr, uint32_t n) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) {
+    __threadfence();
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(ctr), "r"(n) : "memory");
+  }
+}
 __device__ __forceinline__ void async_proxy_acquire() {
   asm volatile("fence.proxy.async.global;" ::: "memory");
 }
@@ -112,10 +121,10 @@ struct ICfg {
   static constexpr int kAccCols = (NFP <= 64) ? 64 : 128;
   static constexpr int kNumAcc = 512 / kAccCols;
   static constexpr int kProd = 2, kMma = 2, kEpi = 2;       // producer warps, issuer warps, epilogue groups
-  // epilogue staging: per warp two buffers of [NF frequencies][32 channels] halves
-  static constexpr int kOutBufBytes = (NF * 64 + 127) / 128 * 128;
+  // epilogue staging: per group two buffers of [NF frequencies][128 channels] halves
+  static constexpr int kOutBufBytes = NF * 256;
   static constexpr int kOutOffset = kKronBytes + kStages * kStageBytes;
-  static constexpr int kBytes = kOutOffset + 4 * kEpi * 2 * kOutBufBytes;
+  static constexpr int kBytes = kOutOffset + kEpi * 2 * kOutBufBytes;
   // a slot of a ring is always handled by the same warp (group): see the note in input_transform_tc.cu
   static_assert(kStages % kProd == 0 && kStages % kMma == 0 && kNumAcc % kMma == 0 && kNumAcc % kEpi == 0, "rings");
 };
@@ -148,7 +157,7 @@ struct FusedCfg {
 template <int M>
 __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
                                            volatile int* abort_flag, const CUtensorMap* tmX,
-                                           const CUtensorMap* tmKron, const CUtensorMap* tmVst,
+                                           const CUtensorMap* tmKron, __half* __restrict__ V,
                                            const ConvShape& cs, const RingParams& rp, int rank, bool& timed_out) {
   using Cfg = ICfg<M>;
   constexpr int kStages = Cfg::kStages, kNumAcc = Cfg::kNumAcc, kAccCols = Cfg::kAccCols;
@@ -244,28 +253,35 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
       __syncwarp();
     }
   } else if (warp < Cfg::kProd + Cfg::kMma + 4 * Cfg::kEpi) {
-    // Epilogue.  A warp turns its 32 channels x NF frequencies into a [NF][32] half tile in
-    // shared memory and TMA-stores it (one instruction per unit) to V[f][row][c0..c0+31]; the
-    // store clips channels >= C.  The block counter is raised once the store is complete,
-    // one unit later, so the warp never waits for its own store.
+    // Epilogue.  The four warps of a group turn a unit's accumulator (128 channels x NF
+    // frequencies, a lane = a channel) into a [NF][128] half tile in shared memory, then all
+    // 128 threads copy it out with 16-byte stores: every warp store covers two whole 256-byte
+    // rows V[f][row][c0..c0+127].  The block counter is raised (after a fence) when the warp
+    // moves on to another block or ends, not per unit.
     const int quad = warp & 3;
     const int ew = warp - Cfg::kProd - Cfg::kMma;          // epilogue warp index
     const int group = ew >> 2;
-    uint8_t* out0 = smem + Cfg::kOutOffset + (size_t)ew * 2 * Cfg::kOutBufBytes;
-    int pending_block = -1;
+    const int tg = (ew & 3) * 32 + lane;                   // thread index within the group
+    uint8_t* out0 = smem + Cfg::kOutOffset + (size_t)group * 2 * Cfg::kOutBufBytes;
+    const size_t f_stride = (size_t)RP * C;
+    int pend_block = -1;
+    uint32_t pend_count = 0;
     uint32_t n_mine = 0;
     for (unsigned local = group; local < n_local && !timed_out; local += Cfg::kEpi, ++n_mine) {
       const unsigned u = rank + local * rp.nI;
       const unsigned p = u / CB, cblk = u % CB;
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
-      const int c0 = (int)cblk * 128 + quad * 32;
+      const int blk = (int)(p >> 7);
+      if (blk != pend_block) {
+        if (pend_count) ctr_signal_n(rp.v_ready + pend_block, pend_count);
+        pend_block = blk;
+        pend_count = 0;
+      }
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
       uint8_t* buf = out0 + (n_mine & 1) * Cfg::kOutBufBytes;
-      if (lane == 0) bulk_wait_read<1>();                  // the store that last read this buffer is done with it
-      __syncwarp();
-      __half* mine = reinterpret_cast<__half*>(buf) + lane;
+      __half* mine = reinterpret_cast<__half*>(buf) + quad * 32 + lane;
 #pragma unroll
       for (int col0 = 0; col0 < Cfg::NFP; col0 += 64) {
         constexpr int kMaxCols = 64;
@@ -281,30 +297,27 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
         }
 #pragma unroll
         for (int cc = 0; cc < kMaxCols; ++cc)
-          if (col0 + cc < Cfg::NF) mine[(col0 + cc) * 32] = __float2half_rn(__uint_as_float(r[cc]));
+          if (col0 + cc < Cfg::NF) mine[(col0 + cc) * 128] = __float2half_rn(__uint_as_float(r[cc]));
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) {
-        if (c0 < C) tma_store_3d(tmVst, buf, c0, (int)(p % (unsigned)RP), 0);
-        bulk_commit();
-        if (pending_block >= 0) {
-          bulk_wait_done<1>();                             // the previous unit's store is complete
-          __threadfence();
-          asm volatile("fence.proxy.async.global;" ::: "memory");
-          asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(rp.v_ready + pending_block) : "memory");
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+      {
+        const int chunk = tg & 15;                         // 16-byte piece of a 256-byte row
+        const int c = (int)cblk * 128 + chunk * 8;
+        if (c < C) {
+          __half* dst = V + (size_t)(p % (unsigned)RP) * C + c + (size_t)(tg >> 4) * f_stride;
+          const uint8_t* src = buf + (tg >> 4) * 256 + chunk * 16;
+#pragma unroll
+          for (int f = tg >> 4, j = 0; j < (Cfg::NF + 7) / 8; ++j, f += 8)
+            if (f < Cfg::NF) {
+              *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+              dst += 8 * f_stride;
+              src += 8 * 256;
+            }
         }
       }
-      pending_block = (int)(p >> 7);
+      ++pend_count;
     }
-    if (lane == 0) {
-      bulk_wait_done<0>();
-      if (pending_block >= 0 && !timed_out) {
-        __threadfence();
-        asm volatile("fence.proxy.async.global;" ::: "memory");
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(rp.v_ready + pending_block) : "memory");
-      }
-    }
+    if (pend_count && !timed_out) ctr_signal_n(rp.v_ready + pend_block, pend_count);
   }
   tc_fence_before();
   __syncthreads();
@@ -593,8 +606,8 @@ template <int M, int BLOCK_N, bool SYM>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_conv_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
-                  const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmVst,
-                  const __grid_constant__ Coefs cf, float* __restrict__ Mo, __half* __restrict__ y,
+                  const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
+                  __half* __restrict__ V, float* __restrict__ Mo, __half* __restrict__ y,
                   const ConvShape cs, const RingParams rp, int* __restrict__ status) {
   using F = FusedCfg<M, BLOCK_N>;
   extern __shared__ uint8_t smem_raw[];
@@ -608,7 +621,7 @@ fused_conv_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   bool timed_out = false;
   const int b = blockIdx.x;
   if (b < rp.nI)
-    role_input<M>(smem, bars, tmem_base_slot, abort_flag, &tmX, &tmKron, &tmVst, cs, rp, b, timed_out);
+    role_input<M>(smem, bars, tmem_base_slot, abort_flag, &tmX, &tmKron, V, cs, rp, b, timed_out);
   else if (b < rp.nI + rp.nG)
     role_gemm<(M + 2) * (M + 2), BLOCK_N>(smem, bars, tmem_base_slot, abort_flag, &tmV, &tmU, Mo, cs, rp,
                                           b - rp.nI, timed_out);
@@ -665,7 +678,7 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     attr_set = true;
   }
   const int RP = R * 128;
-  CUtensorMap tmX, tmK, tmV, tmU, tmM, tmVst;
+  CUtensorMap tmX, tmK, tmV, tmU, tmM;
   const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
   const CUtensorMapL2promotion p256 = CU_TENSOR_MAP_L2_PROMOTION_L2_256B, p128 = CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
   {
@@ -686,9 +699,6 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     cuuint64_t strides[2] = {(cuuint64_t)g.C * 2, (cuuint64_t)RP * g.C * 2};
     cuuint32_t box[3] = {BLOCK_K, BLOCK_M, 1};
     if (!encode(&tmV, f16, 3, Vr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
-    cuuint32_t sbox[3] = {32, 1, (cuuint32_t)NF};            // the epilogue's store box: [NF][1 row][32 channels]
-    if (!encode(&tmVst, f16, 3, Vr, dims, strides, sbox, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_SWIZZLE_NONE))
-      return (int)cudaErrorUnknown;
   }
   {
     cuuint64_t dims[3] = {(cuuint64_t)g.C, (cuuint64_t)g.K, (cuuint64_t)NF};
@@ -734,8 +744,8 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return (int)cudaLaunchKernelEx(&cfg, fused_conv_kernel<M, BLOCK_N, SYM>, tmX, tmK, tmV, tmU, tmM, tmVst,
-                                 plan->kcoefs, Mr, (__half*)y, cs, rp, plan->status_dev);
+  return (int)cudaLaunchKernelEx(&cfg, fused_conv_kernel<M, BLOCK_N, SYM>, tmX, tmK, tmV, tmU, tmM, plan->kcoefs,
+                                 (__half*)Vr, Mr, (__half*)y, cs, rp, plan->status_dev);
 }
 
 template <int M>
