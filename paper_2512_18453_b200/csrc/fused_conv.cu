@@ -88,6 +88,13 @@ __device__ __forceinline__ void ctr_signal_n(uint32_t* ctr, uint32_t n) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(ctr), "r"(n) : "memory");
   }
 }
+// "These rows have been read": raised after the data has landed in shared memory (the full
+// barrier was observed) and been loaded into registers, so no fence is needed - and none is
+// wanted: a fence would wait for the warp's own earlier y stores.
+__device__ __forceinline__ void ctr_signal_read(uint32_t* ctr) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+}
 __device__ __forceinline__ void async_proxy_acquire() {
   asm volatile("fence.proxy.async.global;" ::: "memory");
 }
@@ -339,6 +346,7 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* tmem_full = empty_bar + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
+  uint64_t* stored_bar = tmem_empty + 2;           // [2]: the epilogue warps have issued an item's stores
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int C = cs.C, K = cs.K;
@@ -355,7 +363,11 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tmem_full[a], 1);
+      mbar_init(&tmem_empty[a], 8);
+      mbar_init(&stored_bar[a], 8);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(tmem_base_slot, kTmemCols);
@@ -419,9 +431,15 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 10) {
+    // Epilogue: warps 2-5 drain columns [0, BLOCK_N/2), warps 6-9 the other half (each set has
+    // one warp per TMEM lane quadrant).  A warp stores straight from registers (16-byte stores,
+    // 512 contiguous bytes per warp instruction in the quad-major M layout), then arrives on
+    // stored_bar and moves on; warp 10 makes the item's stores visible and raises the counter.
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int k4 = K >> 2;
+    constexpr int HALF_N = BLOCK_N / 2;
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
       const unsigned it = rank + local * rp.nG;
       const unsigned pb = it / per_block, rem = it % per_block;
@@ -430,13 +448,15 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const int row = (int)(pb % (unsigned)rp.R) * 128 + quad * 32 + lane;
-      const int k_left = K - (int)kb * BLOCK_N;
-      float* dst = Mo + (((size_t)f * k4 + (size_t)((int)kb * BLOCK_N >> 2)) * RP + row) * 4;
+      const int col_base = (int)kb * BLOCK_N + half * HALF_N;
+      const int k_left = K - col_base;
+      float* dst = Mo + (((size_t)f * k4 + (size_t)(col_base >> 2)) * RP + row) * 4;
       const size_t q_stride = (size_t)RP * 4;
-#pragma unroll 1
-      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32) {
+#pragma unroll 2
+      for (int cb = 0; cb < HALF_N; cb += 32) {
+        if (cb >= k_left) break;
         uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + cb, r);
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + half * HALF_N + cb, r);
         tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -446,8 +466,25 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tmem_empty[acc]);
-      ctr_signal(rp.g_done + pb);
+      if (lane == 0) {
+        mbar_arrive(&tmem_empty[acc]);
+        mbar_arrive(&stored_bar[acc]);
+      }
+    }
+  } else if (warp == 10) {
+    // Signalling warp: once all eight epilogue warps have issued an item's stores (barrier,
+    // CTA scope), one fence at GPU scope orders them before the counter update.
+    for (unsigned local = 0; local < n_local && !timed_out; ++local) {
+      const unsigned it = rank + local * rp.nG;
+      const unsigned pb = it / per_block;
+      const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+      if (!mbar_wait_warp(&stored_bar[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      if (lane == 0) {
+        __threadfence();
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        asm volatile("red.release.gpu.global.add.u32 [%0], 4;" ::"l"(rp.g_done + pb) : "memory");
+      }
+      __syncwarp();
     }
   }
   tc_fence_before();
@@ -575,7 +612,7 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
-      ctr_signal(rp.o_done + (tg >> 4));
+      ctr_signal_read(rp.o_done + (tg >> 4));
 
       const int pl = (int)tg * 8 + t;
       const int k = (int)kg * 16 + (lane & 15);
