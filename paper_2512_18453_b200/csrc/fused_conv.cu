@@ -25,6 +25,7 @@
 
 #include "nova_internal.h"
 #include "sm100.cuh"
+#include "output_math.cuh"
 #include "transform_math.cuh"
 
 namespace nova {
@@ -161,6 +162,35 @@ struct FusedCfg {
 };
 
 // ---------------------------------------------------------------- role I
+// Epilogue pieces with compile-time shared-memory offsets (one instruction per access).
+template <int CC, int COL0, int NF>
+__device__ __forceinline__ void sts_cols(uint32_t mine, const uint32_t* r) {
+  if constexpr (CC < 64) {
+    if constexpr (COL0 + CC < NF) {
+      sts_b16<(COL0 + CC) * 256>(mine, __half_as_ushort(__float2half_rn(__uint_as_float(r[CC]))));
+      sts_cols<CC + 1, COL0, NF>(mine, r);
+    }
+  }
+}
+// 64 accumulator columns starting at COL0: TMEM -> registers -> half -> column of the staging tile
+template <class Cfg, int COL0>
+__device__ __forceinline__ void epi_pass(uint32_t taddr, uint32_t mine) {
+  uint32_t r[64];
+#pragma unroll
+  for (int cc = 0; cc < 64; cc += 16)
+    if (COL0 + cc < Cfg::NFP) tmem_ld16(taddr + COL0 + cc, r + cc);
+  tmem_ld_wait();
+  sts_cols<0, COL0, Cfg::NF>(mine, r);
+}
+// rows f0, f0+8, f0+16, .. of the staging tile: one 16-byte piece each, to global rows 8 planes apart
+template <class Cfg, int J>
+__device__ __forceinline__ void copy_out(uint32_t src, __half* dst, size_t stride8, int f0) {
+  if constexpr (J < (Cfg::NF + 7) / 8) {
+    if (f0 + 8 * J < Cfg::NF) *reinterpret_cast<uint4*>(dst) = lds_v4<J * 8 * 256>(src);
+    copy_out<Cfg, J + 1>(src, dst + stride8, stride8, f0);
+  }
+}
+
 template <int M>
 __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
                                            volatile int* abort_flag, const CUtensorMap* tmX,
@@ -287,39 +317,20 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
-      uint8_t* buf = out0 + (n_mine & 1) * Cfg::kOutBufBytes;
-      __half* mine = reinterpret_cast<__half*>(buf) + quad * 32 + lane;
-#pragma unroll
-      for (int col0 = 0; col0 < Cfg::NFP; col0 += 64) {
-        constexpr int kMaxCols = 64;
-        uint32_t r[kMaxCols];
-#pragma unroll
-        for (int cc = 0; cc < kMaxCols; cc += 16)
-          if (col0 + cc < Cfg::NFP) tmem_ld16(taddr + col0 + cc, r + cc);
-        tmem_ld_wait();
-        if (col0 + 64 >= Cfg::NFP) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&tmem_empty[acc]);
-        }
-#pragma unroll
-        for (int cc = 0; cc < kMaxCols; ++cc)
-          if (col0 + cc < Cfg::NF) mine[(col0 + cc) * 128] = __float2half_rn(__uint_as_float(r[cc]));
-      }
+      const uint32_t buf = smem_u32(out0) + (n_mine & 1) * Cfg::kOutBufBytes;
+      const uint32_t mine = buf + (quad * 32 + lane) * 2;          // this channel's column of the [NF][128] tile
+      epi_pass<Cfg, 0>(taddr, mine);
+      if constexpr (Cfg::NFP > 64) epi_pass<Cfg, 64>(taddr, mine);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[acc]);
       asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
       {
         const int chunk = tg & 15;                         // 16-byte piece of a 256-byte row
         const int c = (int)cblk * 128 + chunk * 8;
         if (c < C) {
           __half* dst = V + (size_t)(p % (unsigned)RP) * C + c + (size_t)(tg >> 4) * f_stride;
-          const uint8_t* src = buf + (tg >> 4) * 256 + chunk * 16;
-#pragma unroll
-          for (int f = tg >> 4, j = 0; j < (Cfg::NF + 7) / 8; ++j, f += 8)
-            if (f < Cfg::NF) {
-              *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
-              dst += 8 * f_stride;
-              src += 8 * 256;
-            }
+          copy_out<Cfg, 0>(buf + (tg >> 4) * 256 + chunk * 16, dst, 8 * f_stride, tg >> 4);
         }
       }
       ++pend_count;
@@ -550,66 +561,10 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
       const unsigned tg = u / KG, kg = u % KG;
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
-      const uint8_t* sb = smem + (size_t)stage * Cfg::kStageBytes;
-      auto ldm = [&](int f) -> float {
-        return *reinterpret_cast<const float*>(sb + f * 512 + ((f & 1) ? off_odd : off_even));
-      };
-      auto load_row = [&](int xi, float (&z)[M]) {
-        float in[N];
-#pragma unroll
-        for (int nu = 0; nu < N; ++nu) in[nu] = ldm(xi * N + nu);
-        at_apply<M, SYM, float>(cf, in, z);
-      };
+      const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
+      const uint32_t sb_even = sb + off_even, sb_odd = sb + off_odd;
       float Y[M][M];
-      if constexpr (!SYM) {
-#pragma unroll
-        for (int i = 0; i < M; ++i)
-#pragma unroll
-          for (int j = 0; j < M; ++j) Y[i][j] = 0.f;
-#pragma unroll
-        for (int xi = 0; xi < N; ++xi) {
-          float z[M];
-          load_row(xi, z);
-#pragma unroll
-          for (int i = 0; i < M; ++i)
-#pragma unroll
-            for (int j = 0; j < M; ++j) Y[i][j] = fmaf(cf.AT[i][xi], z[j], Y[i][j]);
-        }
-      } else {
-        {
-          float zp[M], zm[M];
-          load_row(1, zp);
-          load_row(2, zm);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
-#pragma unroll
-            for (int i = 0; i < M; ++i) Y[i][j] = cf.AT[i][1] * ((i & 1) ? d : s);
-          }
-        }
-#pragma unroll
-        for (int q = 3; q < N - 1; q += 2) {
-          float zp[M], zm[M];
-          load_row(q, zp);
-          load_row(q + 1, zm);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
-#pragma unroll
-            for (int i = 0; i < M; ++i) Y[i][j] = fmaf(cf.AT[i][q], (i & 1) ? d : s, Y[i][j]);
-          }
-        }
-        {
-          float z0[M], zi[M];
-          load_row(0, z0);
-          load_row(N - 1, zi);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            Y[0][j] += z0[j];
-            Y[M - 1][j] += zi[j];
-          }
-        }
-      }
+      OutputTile<M, SYM>{cf, sb_even, sb_odd}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
       ctr_signal_read(rp.o_done + (tg >> 4));
@@ -622,17 +577,7 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
         const unsigned th = q2 % (unsigned)cs.Th, img = q2 / (unsigned)cs.Th;
         const int h0 = M * (int)th, w0 = M * (int)tw;
         __half* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
-#pragma unroll
-        for (int i = 0; i < M; ++i) {
-          if (h0 + i >= H) continue;
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            if (w0 + j >= W) continue;
-            float v = Y[i][j];
-            if (cs.relu) v = v < 0.f ? 0.f : v;
-            vstore(dst + ((size_t)i * W + j) * K, v);
-          }
-        }
+        store_tile<M, __half>(Y, dst, (size_t)W * K, K, H - h0, W - w0, cs.relu);
       }
     }
   }

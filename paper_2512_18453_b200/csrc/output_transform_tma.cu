@@ -18,6 +18,7 @@
 
 #include "nova_internal.h"
 #include "sm100.cuh"
+#include "output_math.cuh"
 #include "transform_math.cuh"
 
 namespace nova {
@@ -99,68 +100,10 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
     for (uint32_t local = group; local < n_local && !timed_out; local += kConsGroups) {
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
-      const uint8_t* sb = smem + (size_t)stage * Cfg::kStageBytes;
-      auto ldm = [&](int f) -> float {
-        return *reinterpret_cast<const float*>(sb + f * 512 + ((f & 1) ? off_odd : off_even));
-      };
-      auto load_row = [&](int xi, float (&z)[M]) {
-        float in[N];
-#pragma unroll
-        for (int nu = 0; nu < N; ++nu) in[nu] = ldm(xi * N + nu);
-        at_apply<M, SYM, float>(cf, in, z);
-      };
+      const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
+      const uint32_t sb_even = sb + off_even, sb_odd = sb + off_odd;
       float Y[M][M];
-      if constexpr (!SYM) {
-#pragma unroll
-        for (int i = 0; i < M; ++i)
-#pragma unroll
-          for (int j = 0; j < M; ++j) Y[i][j] = 0.f;
-#pragma unroll
-        for (int xi = 0; xi < N; ++xi) {
-          float z[M];
-          load_row(xi, z);
-#pragma unroll
-          for (int i = 0; i < M; ++i)
-#pragma unroll
-            for (int j = 0; j < M; ++j) Y[i][j] = fmaf(cf.AT[i][xi], z[j], Y[i][j]);
-        }
-      } else {
-        // A^T column 0 is e_0 and column n-1 is e_{m-1}; columns +a / -a share |coefficients|.
-        {
-          float zp[M], zm[M];
-          load_row(1, zp);
-          load_row(2, zm);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
-#pragma unroll
-            for (int i = 0; i < M; ++i) Y[i][j] = cf.AT[i][1] * ((i & 1) ? d : s);
-          }
-        }
-#pragma unroll
-        for (int q = 3; q < N - 1; q += 2) {
-          float zp[M], zm[M];
-          load_row(q, zp);
-          load_row(q + 1, zm);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            const float s = zp[j] + zm[j], d = zp[j] - zm[j];
-#pragma unroll
-            for (int i = 0; i < M; ++i) Y[i][j] = fmaf(cf.AT[i][q], (i & 1) ? d : s, Y[i][j]);
-          }
-        }
-        {
-          float z0[M], zi[M];
-          load_row(0, z0);
-          load_row(N - 1, zi);
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            Y[0][j] += z0[j];
-            Y[M - 1][j] += zi[j];
-          }
-        }
-      }
-      // the stage's values are all in registers: hand it back to the producer
+      OutputTile<M, SYM>{cf, sb_even, sb_odd}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
 
@@ -172,17 +115,7 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
         const unsigned th = q2 % (unsigned)Th, img = q2 / (unsigned)Th;
         const int h0 = M * (int)th, w0 = M * (int)tw;
         T* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
-#pragma unroll
-        for (int i = 0; i < M; ++i) {
-          if (h0 + i >= H) continue;
-#pragma unroll
-          for (int j = 0; j < M; ++j) {
-            if (w0 + j >= W) continue;
-            float v = Y[i][j];
-            if (relu) v = v < 0.f ? 0.f : v;          // NaN and +inf pass through
-            vstore(dst + ((size_t)i * W + j) * K, v);
-          }
-        }
+        store_tile<M, T>(Y, dst, (size_t)W * K, K, H - h0, W - w0, relu);
       }
 #pragma unroll
       for (int s = 0; s < kConsGroups; ++s)

@@ -154,6 +154,28 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       : "memory");
 }
 
+// Shared-memory accesses by 32-bit shared address plus a compile-time byte offset: one
+// instruction each (a pointer derived from the aligned dynamic-shared base is generic to the
+// compiler and would cost 64-bit address arithmetic per access).
+template <int OFF>
+__device__ __forceinline__ float lds_f32(uint32_t saddr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(saddr), "n"(OFF));
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ void sts_b16(uint32_t saddr, unsigned short v) {
+  asm volatile("st.shared.b16 [%0+%1], %2;" ::"r"(saddr), "n"(OFF), "h"(v) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ uint4 lds_v4(uint32_t saddr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "r"(saddr), "n"(OFF));
+  return v;
+}
+
 // TMA tile store (shared -> global) and its bulk async-group bookkeeping.
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int x, int y, int z) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
