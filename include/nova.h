@@ -227,6 +227,10 @@ int nova_maxpool2x2(const void* x_dev, void* y_dev, int N, int H, int W, int C,
  */
 int nova_last_device_status(const nova_plan* plan, nova_stream stream);
 
+/* The raw cudaError_t value of the last CUDA call that made a convolution entry point return
+ * NOVA_ERR_CUDA (0 if none so far); not thread-safe, for diagnostics. */
+int nova_last_cuda_error(void);
+
 const char* nova_status_string(int status);
 
 #ifdef __cplusplus

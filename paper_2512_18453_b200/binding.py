@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = (
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
-    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split",
+    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
 )
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -26,7 +26,8 @@ STATIC_SCRATCH_BYTES = 32 << 20
 class NovaError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
-        super().__init__("%s: %s (%d)" % (where, status_string(status), status))
+        extra = " [cudaError %d]" % lib().nova_last_cuda_error() if status == -8 else ""
+        super().__init__("%s: %s (%d)%s" % (where, status_string(status), status, extra))
 
 
 class _Rat(ctypes.Structure):
@@ -58,6 +59,8 @@ def lib():
     L.nova_plan_frequency_order.restype = i
     L.nova_plan_set_role_split.argtypes = [vp, i, i]
     L.nova_plan_set_role_split.restype = i
+    L.nova_last_cuda_error.argtypes = []
+    L.nova_last_cuda_error.restype = i
     L.nova_plan_kappa.argtypes = [vp, dp]
     L.nova_plan_kappa.restype = i
     L.nova_filter_transform_bytes.argtypes = [vp, i, i]

@@ -119,6 +119,7 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
 }
 
 namespace {
+int g_last_cuda_error = 0;          // raw code of the last failed CUDA call on the convolution path
 // Shared body of nova_conv2d_fwd and nova_conv2d_fwd_timed.  With `ev` non-null,
 // four events per chunk bracket the three kernels.
 int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, int N, int H, int W, int C,
@@ -134,6 +135,7 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
     if (ev) cudaEventRecord(ev[1], s);
     const int e = launch_fused_conv(p, g, x, U, y, ws, R, (flags & NOVA_RELU) ? 1 : 0, stream);
     if (ev) cudaEventRecord(ev[2], s);
+    if (e) g_last_cuda_error = e;
     return e ? NOVA_ERR_CUDA : NOVA_OK;
   }
   Chunking c;
@@ -251,6 +253,8 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
   if (st != NOVA_OK) return st;
   return conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, NOVA_STATIC_SCRATCH_BYTES, flags, stream, nullptr);
 }
+
+extern "C" int nova_last_cuda_error(void) { return g_last_cuda_error; }
 
 extern "C" int nova_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode,
                                nova_stream stream) {

@@ -2,9 +2,13 @@
 // Appendix B.5) as ONE persistent kernel whose CTAs are specialised by role and exchange
 // work through rings of transformed tiles that stay in the L2 cache:
 //
-//   role I  (nI CTAs)  input transform on the tensor cores, x -> V ring       (see input_transform_tc.cu)
-//   role G  (nG CTAs)  transformed-domain product, V ring x U -> M ring        (see gemm_tcgen05.cu)
-//   role O  (the rest) output transform, M ring -> y                           (see output_transform_tma.cu)
+//   role I  (nI CTAs)      input transform on the tensor cores, x -> V ring   (see input_transform_tc.cu)
+//   role G  (the others)   transformed-domain product, V ring x U -> M ring    (see gemm_tcgen05.cu)
+//   role O  (every CTA)    output transform, M ring -> y                       (see output_transform_tma.cu)
+// Every CTA runs role O on its last nine warps next to role I or role G on the first ones:
+// G is bound by the SM's store bandwidth (its epilogue writes 128 KB of M per item while the
+// tensor pipe and the issue slots idle), I mostly by latencies, O by instruction issue, so O
+// fills the issue slots of every SM while the stores of V and M spread over the chip.
 //
 // The tiles are grouped in blocks of 128; the rings hold R blocks (row = tile mod 128 R).
 // Three counters per block order the roles:
@@ -33,10 +37,12 @@ namespace {
 using namespace sm100;
 using namespace xf;
 
-constexpr int kFusedThreads = 416;     // 13 warps: the largest role (O) needs them all
+constexpr int kFusedThreads = 640;     // 20 warps (5 per scheduler x 96 registers fill its register file):
+                                       // 11 of role I or G, then 9 of role O
+constexpr int kGWarps = 11;
+constexpr int kOWarpBase = 11;
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;
-constexpr int kGemmStages = 4;
 constexpr uint32_t kCtrSpinLimit = 1u << 20;
 
 struct RingParams {
@@ -46,7 +52,7 @@ struct RingParams {
   int* abort_all;        // set by any CTA that gives up
   int R;                 // ring length in 128-tile blocks
   int P;                 // tiles
-  int nI, nG;            // CTAs of role I and G; the rest are role O
+  int nI, nGO;           // CTAs of role I; the others run roles G and O together
 };
 
 struct ConvShape {
@@ -125,10 +131,10 @@ struct ICfg {
   static constexpr int kHalfBytes = KP * 128;
   static constexpr int kStageBytes = 2 * kHalfBytes;
   static constexpr int kKronBytes = 2 * KA * NFP * 128;
-  static constexpr int kStages = (kStageBytes <= 16384) ? 6 : 2;
+  static constexpr int kStages = (kStageBytes <= 16384) ? 4 : 2;
   static constexpr int kAccCols = (NFP <= 64) ? 64 : 128;
   static constexpr int kNumAcc = 512 / kAccCols;
-  static constexpr int kProd = 2, kMma = 2, kEpi = 2;       // producer warps, issuer warps, epilogue groups
+  static constexpr int kProd = 1, kMma = 2, kEpi = 2;       // producer warps, issuer warps, epilogue groups
   // epilogue staging: per group two buffers of [NF frequencies][128 channels] halves
   static constexpr int kOutBufBytes = NF * 256;
   static constexpr int kOutOffset = kKronBytes + kStages * kStageBytes;
@@ -136,27 +142,32 @@ struct ICfg {
   // a slot of a ring is always handled by the same warp (group): see the note in input_transform_tc.cu
   static_assert(kStages % kProd == 0 && kStages % kMma == 0 && kNumAcc % kMma == 0 && kNumAcc % kEpi == 0, "rings");
 };
-template <int BLOCK_N>
-struct GCfg {
-  static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
-  static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBytes = kGemmStages * kStageBytes;
-};
 template <int M>
 struct OCfg {
   static constexpr int N = M + 2;
   static constexpr int NF = N * N;
   static constexpr int kStageBytes = NF * 512;
-  static constexpr int kGroups = 3;
-  static constexpr int kStages = ((200 * 1024 / kStageBytes) >= 6 ? 6 : 3);
+  static constexpr int kGroups = 2;
+  static constexpr int kStages = 2;
   static constexpr int kBytes = kStages * kStageBytes;
   static_assert(kStages % kGroups == 0, "stage ring");
+};
+template <int M, int BLOCK_N>
+struct GCfg {
+  static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
+  static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (OCfg<M>::kBytes > 70 * 1024) ? 2 : 3;   // what role O leaves of the SM's shared memory
+  static constexpr int kBytes = kStages * kStageBytes;
 };
 constexpr int cmax(int a, int b) { return a > b ? a : b; }
 template <int M, int BLOCK_N>
 struct FusedCfg {
-  static constexpr int kDataBytes = cmax(ICfg<M>::kBytes, cmax(GCfg<BLOCK_N>::kBytes, OCfg<M>::kBytes));
+  // role O's ring sits behind role I's or role G's data, whichever the CTA runs; where both
+  // do not fit next to role I (F(8,3)), the role-I CTAs run without role O
+  static constexpr bool kOWithI = ICfg<M>::kBytes + OCfg<M>::kBytes <= 220 * 1024;
+  static constexpr int kOOffset = kOWithI ? cmax(ICfg<M>::kBytes, GCfg<M, BLOCK_N>::kBytes) : GCfg<M, BLOCK_N>::kBytes;
+  static constexpr int kDataBytes = cmax(ICfg<M>::kBytes, kOOffset + OCfg<M>::kBytes);
   static constexpr int kBarrierOffset = kDataBytes;
   static constexpr int kTotal = kBarrierOffset + 512 + 1024;
 };
@@ -191,8 +202,36 @@ __device__ __forceinline__ void copy_out(uint32_t src, __half* dst, size_t strid
   }
 }
 
+// All threads of the CTA, before the CTA-wide barrier: role I's barriers and the pad rows of its ring.
 template <int M>
-__device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
+__device__ __forceinline__ void input_prologue(uint8_t* smem, uint64_t* bars) {
+  using Cfg = ICfg<M>;
+  constexpr int kStages = Cfg::kStages, kNumAcc = Cfg::kNumAcc;
+  uint8_t* ring = smem + Cfg::kKronBytes;
+  if (threadIdx.x == 0) {
+    uint64_t* full_bar = bars;
+    uint64_t* empty_bar = full_bar + kStages;
+    uint64_t* tmem_full = empty_bar + kStages;
+    uint64_t* tmem_empty = tmem_full + kNumAcc;
+    uint64_t* kron_bar = tmem_empty + kNumAcc;
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < kNumAcc; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    mbar_init(kron_bar, 1);
+  }
+  if constexpr (Cfg::KP > Cfg::NF) {
+    constexpr int pad16 = (Cfg::KP - Cfg::NF) * 8;
+    for (int i = threadIdx.x; i < kStages * 2 * pad16; i += kFusedThreads) {
+      const int half = i / pad16, off = i % pad16;
+      *reinterpret_cast<uint4*>(ring + (size_t)half * Cfg::kHalfBytes + Cfg::NF * 128 + off * 16) =
+          make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+}
+constexpr int kIBarriers = 40;      // barrier slots reserved for role I or G; role O's follow
+// Warps 0 .. 10 of the CTA; barriers and TMEM are set up by the caller.
+template <int M>
+__device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32_t tmem_base,
                                            volatile int* abort_flag, const CUtensorMap* tmX,
                                            const CUtensorMap* tmKron, __half* __restrict__ V,
                                            const ConvShape& cs, const RingParams& rp, int rank, bool& timed_out) {
@@ -213,27 +252,6 @@ __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32
   const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + rp.nI - 1) / rp.nI : 0u;
   const int RP = rp.R * 128;
   const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((cs.K + 255) / 256) * 4u;   // see role G
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < kNumAcc; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
-    mbar_init(kron_bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == Cfg::kProd) tmem_alloc(tmem_base_slot, 512);
-  if constexpr (Cfg::KP > Cfg::NF) {
-    constexpr int pad16 = (Cfg::KP - Cfg::NF) * 8;
-    for (int i = threadIdx.x; i < kStages * 2 * pad16; i += kFusedThreads) {
-      const int half = i / pad16, off = i % pad16;
-      *reinterpret_cast<uint4*>(ring + (size_t)half * Cfg::kHalfBytes + Cfg::NF * 128 + off * 16) =
-          make_uint4(0, 0, 0, 0);
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_base_slot;
 
   if (warp < Cfg::kProd) {
     if (warp == 0 && lane == 0) {
@@ -337,22 +355,33 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
     }
     if (pend_count && !timed_out) ctr_signal_n(rp.v_ready + pend_block, pend_count);
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == Cfg::kProd) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
-  }
 }
 
 // ---------------------------------------------------------------- role G
-template <int NF, int BLOCK_N>
-__device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_t* tmem_base_slot,
+template <int M, int BLOCK_N>
+__device__ __forceinline__ void gemm_init(uint64_t* bars) {
+  constexpr int kStages = GCfg<M, BLOCK_N>::kStages;
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full = empty_bar + kStages;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint64_t* stored_bar = tmem_empty + 2;
+  for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+  for (int a = 0; a < 2; ++a) {
+    mbar_init(&tmem_full[a], 1);
+    mbar_init(&tmem_empty[a], 8);
+    mbar_init(&stored_bar[a], 8);
+  }
+}
+// Warps 0 .. kGWarps-1 of the CTA; barriers and TMEM are set up by the caller.
+template <int M, int BLOCK_N>
+__device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_t tmem_base,
                                           volatile int* abort_flag, const CUtensorMap* tmV,
                                           const CUtensorMap* tmU, float* __restrict__ Mo, const ConvShape& cs,
                                           const RingParams& rp, int rank, bool& timed_out) {
-  using L = GCfg<BLOCK_N>;
-  constexpr int kStages = kGemmStages;
+  using L = GCfg<M, BLOCK_N>;
+  constexpr int NF = (M + 2) * (M + 2);
+  constexpr int kStages = L::kStages;
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* tmem_full = empty_bar + kStages;
@@ -366,31 +395,15 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
   const int num_ks = (C + BLOCK_K - 1) / BLOCK_K;
   const unsigned per_block = (unsigned)NF * num_kb;
   const unsigned num_items = NB * per_block;
-  const unsigned n_local = (num_items > (unsigned)rank) ? (num_items - rank + rp.nG - 1) / rp.nG : 0u;
+  const unsigned n_local = (num_items > (unsigned)rank) ? (num_items - rank + rp.nGO - 1) / rp.nGO : 0u;
   const int RP = rp.R * 128;
   const unsigned CB = (unsigned)((C + 127) / 128);
   const uint32_t o_target = 16u * (uint32_t)((K + 15) >> 4) * 4u;     // see role O
-  constexpr uint32_t kTmemCols = (2 * BLOCK_N < 32) ? 32 : 2 * BLOCK_N;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(&tmem_full[a], 1);
-      mbar_init(&tmem_empty[a], 8);
-      mbar_init(&stored_bar[a], 8);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) tmem_alloc(tmem_base_slot, kTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_base_slot;
 
   if (warp == 0) {
     uint32_t stage = 0, phase = 0;
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
-      const unsigned it = rank + local * rp.nG;
+      const unsigned it = rank + local * rp.nGO;
       const unsigned pb = it / per_block, rem = it % per_block;
       const unsigned f = rem / num_kb, kb = rem % num_kb;
       int tiles = rp.P - (int)pb * 128;
@@ -452,7 +465,7 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
     const int k4 = K >> 2;
     constexpr int HALF_N = BLOCK_N / 2;
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
-      const unsigned it = rank + local * rp.nG;
+      const unsigned it = rank + local * rp.nGO;
       const unsigned pb = it / per_block, rem = it % per_block;
       const unsigned f = rem / num_kb, kb = rem % num_kb;
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
@@ -486,7 +499,7 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
     // Signalling warp: once all eight epilogue warps have issued an item's stores (barrier,
     // CTA scope), one fence at GPU scope orders them before the counter update.
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
-      const unsigned it = rank + local * rp.nG;
+      const unsigned it = rank + local * rp.nGO;
       const unsigned pb = it / per_block;
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
       if (!mbar_wait_warp(&stored_bar[acc], acc_phase, abort_flag)) { timed_out = true; break; }
@@ -498,17 +511,18 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       __syncwarp();
     }
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
-  }
 }
 
 // ---------------------------------------------------------------- role O
+template <int M>
+__device__ __forceinline__ void output_init(uint64_t* bars) {
+  constexpr int kStages = OCfg<M>::kStages;
+  for (int s = 0; s < kStages; ++s) { mbar_init(&bars[s], 1); mbar_init(&bars[kStages + s], 4); }
+}
+// Warps kGWarps .. kGWarps+8 of the CTA (`warp` is relative to kGWarps): one TMA producer and
+// two consumer groups of four warps.
 template <int M, bool SYM>
-__device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volatile int* abort_flag,
+__device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* bars, volatile int* abort_flag,
                                             const CUtensorMap* tmM, const Coefs& cf, __half* __restrict__ y,
                                             const ConvShape& cs, const RingParams& rp, int rank, int size,
                                             bool& timed_out) {
@@ -518,7 +532,7 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = full_bar + kStages;
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31;
   const int K = cs.K, H = cs.H, W = cs.W;
   const unsigned KG = (unsigned)((K + 15) >> 4);
   const unsigned NB = (unsigned)((rp.P + 127) >> 7);
@@ -526,12 +540,6 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
   const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + size - 1) / size : 0u;
   const int RP = rp.R * 128;
   const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((K + 255) / 256) * 4u;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 4); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
 
   if (warp == 0) {
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
@@ -549,7 +557,7 @@ __device__ __forceinline__ void role_output(uint8_t* smem, uint64_t* bars, volat
       }
       __syncwarp();
     }
-  } else {
+  } else if (warp <= 4 * Cfg::kGroups) {
     const int group = (warp - 1) >> 2;
     const int w = (warp - 1) & 3;
     const int t = w + 4 * (lane >> 4);
@@ -595,21 +603,46 @@ fused_conv_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + F::kBarrierOffset);
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 40);
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 48);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
   if (threadIdx.x == 0) *abort_flag = 0;
   __syncthreads();
 
   bool timed_out = false;
   const int b = blockIdx.x;
-  if (b < rp.nI)
-    role_input<M>(smem, bars, tmem_base_slot, abort_flag, &tmX, &tmKron, V, cs, rp, b, timed_out);
-  else if (b < rp.nI + rp.nG)
-    role_gemm<(M + 2) * (M + 2), BLOCK_N>(smem, bars, tmem_base_slot, abort_flag, &tmV, &tmU, Mo, cs, rp,
-                                          b - rp.nI, timed_out);
-  else
-    role_output<M, SYM>(smem, bars, abort_flag, &tmM, cf, y, cs, rp, b - rp.nI - rp.nG,
-                        (int)gridDim.x - rp.nI - rp.nG, timed_out);
+  const int warp = threadIdx.x >> 5;
+  const bool is_input = b < rp.nI;
+  constexpr uint32_t kTmemCols = 512;
+  if (is_input) input_prologue<M>(smem, bars);
+  if (threadIdx.x == 0) {
+    if (!is_input) gemm_init<M, BLOCK_N>(bars);
+    output_init<M>(bars + kIBarriers);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_base_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+  // role O: every CTA (except next to role I where the shared memory does not hold both)
+  const bool o_here = F::kOWithI || !is_input;
+  const int o_rank = F::kOWithI ? b : b - rp.nI;
+  const int o_size = F::kOWithI ? (int)gridDim.x : rp.nGO;
+  if (warp >= kOWarpBase) {
+    if (o_here)
+      role_output<M, SYM>(warp - kOWarpBase, smem + F::kOOffset, bars + kIBarriers, abort_flag, &tmM, cf, y, cs, rp,
+                          o_rank, o_size, timed_out);
+  } else if (is_input) {
+    role_input<M>(smem, bars, tmem_base, abort_flag, &tmX, &tmKron, V, cs, rp, b, timed_out);
+  } else if (warp < kGWarps) {
+    role_gemm<M, BLOCK_N>(smem, bars, tmem_base, abort_flag, &tmV, &tmU, Mo, cs, rp, b - rp.nI, timed_out);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
 
   if (timed_out) {
     *abort_flag = 1;
@@ -707,13 +740,10 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
   rp.R = R;
   rp.P = (int)g.P;
   const int sms = plan->sm_count;
-  int nI = plan->fused_nI, nG = plan->fused_nG;
-  if (nI <= 0 || nG <= 0 || nI + nG >= sms) {         // default split of the SMs between the roles
-    nI = sms * 22 / 100;
-    nG = sms * 40 / 100;
-  }
+  int nI = plan->fused_nI;
+  if (nI <= 0 || nI >= sms) nI = sms * 30 / 100;      // default share of the SMs for role I
   rp.nI = nI;
-  rp.nG = nG;
+  rp.nGO = sms - nI;
   ConvShape cs{g.H, g.W, g.C, g.K, g.Th, g.Tw, relu};
 
   cudaLaunchConfig_t cfg = {};
