@@ -8,7 +8,8 @@
 //             into a 4-stage shared-memory ring, completion on mbarriers;
 //   warp 1    issues tcgen05.mma (kind::f16, M=128, N=BLOCK_N, K=16) from
 //             shared-memory descriptors into one of two TMEM accumulators;
-//   warps 2-5 epilogue: tcgen05.ld the finished accumulator (one TMEM lane
+//   warps 2-9 epilogue, warps 2-5 for the first half of the columns and warps
+//             6-9 for the second: tcgen05.ld the finished accumulator (one TMEM lane
 //             quadrant per warp; a lane is a tile, a column a filter) and
 //             store it straight from registers, overlapping the next item's
 //             MMAs on the other accumulator.  M is laid out
@@ -30,7 +31,7 @@ constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;            // 64 halves = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kStages = 4;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;          // producer, MMA issuer, 2 x 4 epilogue warps
 
 template <int BLOCK_N>
 struct SmemLayout {
@@ -73,7 +74,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -137,10 +138,12 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       }
     }
   } else {
-    // ---------------- epilogue (warps 2..5); a warp may only read TMEM lanes 32*(warp%4)..+31.
+    // ---------------- epilogue (warps 2..9); a warp may only read TMEM lanes 32*(warp%4)..+31.
     // Rows >= pc of the last row block are zeros (the TMA loads of V fill them) and land in the
     // padding rows pc..pc_pad-1 of M.
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;                    // which half of the BLOCK_N columns
+    constexpr int HALF_N = BLOCK_N / 2;
     const int k4 = K >> 2;
     uint32_t local = 0;
     int kb = kb0, pb = pb0, f = f0;
@@ -149,13 +152,14 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = pb * BLOCK_M + quad * 32 + lane;
-      const int k_left = K - kb * BLOCK_N;
-      float* dst = Mo + (((size_t)f * k4 + (size_t)(kb * BLOCK_N >> 2)) * pc_pad + row) * 4;
+      const int col_base = kb * BLOCK_N + half * HALF_N;
+      const int k_left = K - col_base;
+      float* dst = Mo + (((size_t)f * k4 + (size_t)(col_base >> 2)) * pc_pad + row) * 4;
       const size_t q_stride = (size_t)pc_pad * 4;        // floats between consecutive filter quads
 #pragma unroll 1
-      for (int cb = 0; cb < BLOCK_N && cb < k_left; cb += 32) {
+      for (int cb = 0; cb < HALF_N && cb < k_left; cb += 32) {
         uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + cb, r);
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * BLOCK_N + half * HALF_N + cb, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
         for (int j = 0; j < 8; ++j)
