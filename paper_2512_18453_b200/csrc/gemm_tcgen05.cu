@@ -64,13 +64,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const int num_kb = (K + BLOCK_N - 1) / BLOCK_N;
   const int num_ks = (C + BLOCK_K - 1) / BLOCK_K;
   const long long num_items = (long long)nfreq * num_pb * num_kb;
-  // each CTA takes a contiguous range of items (f outermost, then pb, then kb) and advances
-  // the three indices incrementally
-  const long long it_begin = num_items * blockIdx.x / gridDim.x;
-  const long long it_end = num_items * (blockIdx.x + 1) / gridDim.x;
-  const int kb0 = (int)(it_begin % num_kb);
-  const int pb0 = (int)((it_begin / num_kb) % num_pb);
-  const int f0 = (int)(it_begin / ((long long)num_kb * num_pb));
+  // Item i of this CTA is item blockIdx.x + i * gridDim.x, with the row block outermost and
+  // DESCENDING (then frequency, then filter block): the input transform wrote V in ascending
+  // tile order, so the highest row blocks are the ones still in L2; and the row blocks this
+  // kernel finishes last - the lowest - are the ones the output transform reads first.
+  const unsigned per_pb = (unsigned)nfreq * (unsigned)num_kb;
+  const uint32_t n_local = num_items > blockIdx.x ? (uint32_t)((num_items - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0u;
+  auto item_of = [&](uint32_t local, int& pb, int& f, int& kb) {
+    const unsigned it = blockIdx.x + local * gridDim.x;
+    pb = num_pb - 1 - (int)(it / per_pb);
+    const unsigned rem = it % per_pb;
+    f = (int)(rem / (unsigned)num_kb);
+    kb = (int)(rem % (unsigned)num_kb);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -94,8 +100,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   if (warp == 0) {
     // ---------------- TMA producer
     uint32_t stage = 0, phase = 0;
-    int kb = kb0, pb = pb0, f = f0;
-    for (long long it = it_begin; it < it_end && !timed_out; ++it) {
+    for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
+      int pb, f, kb;
+      item_of(local, pb, f, kb);
       for (int ks = 0; ks < num_ks; ++ks) {
         if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
         if (lane == 0) {
@@ -108,13 +115,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         __syncwarp();
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
-      if (++kb == num_kb) { kb = 0; if (++pb == num_pb) { pb = 0; ++f; } }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
     constexpr uint32_t idesc = umma_idesc_f16(BLOCK_M, BLOCK_N);
-    uint32_t stage = 0, phase = 0, local = 0;
-    for (long long it = it_begin; it < it_end && !timed_out; ++it, ++local) {
+    uint32_t stage = 0, phase = 0;
+    for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
       if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -145,9 +151,9 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
     const int half = (warp - 2) >> 2;                    // which half of the BLOCK_N columns
     constexpr int HALF_N = BLOCK_N / 2;
     const int k4 = K >> 2;
-    uint32_t local = 0;
-    int kb = kb0, pb = pb0, f = f0;
-    for (long long it = it_begin; it < it_end && !timed_out; ++it, ++local) {
+    for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
+      int pb, f, kb;
+      item_of(local, pb, f, kb);
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -170,7 +176,6 @@ const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
-      if (++kb == num_kb) { kb = 0; if (++pb == num_pb) { pb = 0; ++f; } }
     }
   }
 

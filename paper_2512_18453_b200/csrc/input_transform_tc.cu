@@ -108,9 +108,11 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int CB = (C + 127) / 128;
-  const long long num_units = (long long)pc * CB;
-  const long long u_begin = num_units * blockIdx.x / gridDim.x;
-  const uint32_t n_local = (uint32_t)(num_units * (blockIdx.x + 1) / gridDim.x - u_begin);
+  // Unit i of this CTA is unit blockIdx.x + i * gridDim.x of the chunk: the chunk's tiles are
+  // transformed in ascending order chip-wide, so that the rows of V written last - the ones
+  // still in L2 when the product kernel starts - are the highest tiles.
+  const unsigned num_units = (unsigned)pc * (unsigned)CB;
+  const uint32_t n_local = num_units > blockIdx.x ? (num_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -144,13 +146,12 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
       for (int b = 0; b < 2 * Cfg::KA; ++b)
         tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, &tmKron, kron_bar, 0, b * Cfg::NFP);
     }
-    // tile coordinates of this warp's first unit, then advanced kProdWarps units at a time
-    // without divisions
-    const long long ufirst = u_begin + warp;
-    int cblk = (int)(ufirst % CB);
-    const long long pfirst = p0 + ufirst / CB;
-    int tw = (int)(pfirst % Tw), th = (int)((pfirst / Tw) % Th), img = (int)(pfirst / ((long long)Tw * Th));
     for (uint32_t local = warp; local < n_local && !timed_out; local += kProdWarps) {
+      const unsigned u = blockIdx.x + local * gridDim.x;
+      const int cblk = (int)(u % (unsigned)CB);
+      const unsigned p = (unsigned)p0 + u / (unsigned)CB;
+      const int tw = (int)(p % (unsigned)Tw), th = (int)((p / (unsigned)Tw) % (unsigned)Th);
+      const int img = (int)(p / ((unsigned)Tw * (unsigned)Th));
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
       if (lane == 0) {
@@ -160,12 +161,6 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
         tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - 1, M * th - 1, img);
       }
       __syncwarp();
-#pragma unroll
-      for (int s = 0; s < kProdWarps; ++s)
-        if (++cblk == CB) {
-          cblk = 0;
-          if (++tw == Tw) { tw = 0; if (++th == Th) { th = 0; ++img; } }
-        }
     }
   } else if (warp < kProdWarps + kMmaWarps) {
     // ---------------- MMA issuers
@@ -201,9 +196,9 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
     const int quad = warp & 3;                    // the TMEM lane quadrant this warp may read
     const int group = (warp - kProdWarps - kMmaWarps) >> 2;
     const size_t f_stride = (size_t)pc_pad * C;
-    const long long ufirst = u_begin + group;
-    int cblk = (int)(ufirst % CB), pl = (int)(ufirst / CB);
     for (uint32_t local = group; local < n_local && !timed_out; local += kEpiGroups) {
+      const unsigned u = blockIdx.x + local * gridDim.x;
+      const int cblk = (int)(u % (unsigned)CB), pl = (int)(u / (unsigned)CB);
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
       const int c = cblk * 128 + quad * 32 + lane;
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
@@ -232,9 +227,6 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
             }
         }
       }
-#pragma unroll
-      for (int s = 0; s < kEpiGroups; ++s)
-        if (++cblk == CB) { cblk = 0; ++pl; }
     }
   }
 

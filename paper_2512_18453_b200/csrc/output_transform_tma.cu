@@ -60,9 +60,10 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
   const int lane = threadIdx.x & 31;
   const int KG = (K + 15) >> 4;                       // filter groups of 16
   const int TG = pc_pad >> 3;                         // tile groups of 8 (pc_pad is a multiple of 128)
-  const long long num_units = (long long)TG * KG;
-  const long long u_begin = num_units * blockIdx.x / gridDim.x;
-  const uint32_t n_local = (uint32_t)(num_units * (blockIdx.x + 1) / gridDim.x - u_begin);
+  // Unit i of this CTA is unit blockIdx.x + i * gridDim.x: ascending tiles chip-wide, i.e. the
+  // rows of M the product kernel wrote last (still in L2) first.
+  const unsigned num_units = (unsigned)TG * (unsigned)KG;
+  const uint32_t n_local = num_units > blockIdx.x ? (num_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 4); }
@@ -74,8 +75,9 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
 
   if (warp == 0) {
     // ---------------- TMA producer
-    int kg = (int)(u_begin % KG), tg = (int)(u_begin / KG);
     for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
+      const unsigned u = blockIdx.x + local * gridDim.x;
+      const int kg = (int)(u % (unsigned)KG), tg = (int)(u / (unsigned)KG);
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
       if (lane == 0) {
@@ -83,7 +85,6 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
         tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, &tmM, &full_bar[stage], tg * 32, kg * 4, 0);
       }
       __syncwarp();
-      if (++kg == KG) { kg = 0; ++tg; }
     }
   } else {
     // ---------------- consumers
@@ -95,9 +96,9 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
     // the 16-byte chunk index is XORed with the row index modulo 8)
     const uint32_t off_even = kq * 128 + ((t ^ kq) << 4) + kk * 4;
     const uint32_t off_odd = kq * 128 + ((t ^ (kq + 4)) << 4) + kk * 4;
-    const long long ufirst = u_begin + group;
-    int kg = (int)(ufirst % KG), tg = (int)(ufirst / KG);
     for (uint32_t local = group; local < n_local && !timed_out; local += kConsGroups) {
+      const unsigned u = blockIdx.x + local * gridDim.x;
+      const int kg = (int)(u % (unsigned)KG), tg = (int)(u / (unsigned)KG);
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
       const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
@@ -117,9 +118,6 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
         T* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
         store_tile<M, T>(Y, dst, (size_t)W * K, K, H - h0, W - w0, relu);
       }
-#pragma unroll
-      for (int s = 0; s < kConsGroups; ++s)
-        if (++kg == KG) { kg = 0; ++tg; }
     }
   }
 
