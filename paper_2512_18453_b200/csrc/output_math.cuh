@@ -1,8 +1,11 @@
 // Y = A^T M A for one (tile, filter) whose n*n transformed-domain values sit in a shared-memory
 // stage (Section 2.1 step 4, 2-D nested form of Appendix B.5), evaluated in float.
-// Frequency f = xi*n + nu is 512*f bytes into the stage; even and odd f differ in the
-// swizzled 16-byte chunk, hence two per-lane bases.  Every load is one ld.shared with an
-// immediate offset; the row and pair indices are template parameters for that reason.
+// A thread owns VEC consecutive filters of one tile.  VEC = 1: the stage holds 4 filter quads per
+// frequency, frequency f = xi*n + nu is 512*f bytes in, and even and odd f differ in the swizzled
+// 16-byte chunk (two per-lane bases).  VEC = 2: 8 quads per frequency, 1024*f bytes, one base;
+// the arithmetic then runs on packed fp32 pairs (two IEEE results per instruction).  Every load is
+// one ld.shared with an immediate offset; the row and pair indices are template parameters for
+// that reason.
 #pragma once
 #include "sm100.cuh"
 #include "transform_math.cuh"
@@ -10,71 +13,80 @@
 namespace nova {
 namespace xf {
 
-template <int M, bool SYM>
+__device__ __forceinline__ float vmax_lo(float v, float lo) { return v < lo ? lo : v; }
+__device__ __forceinline__ float2 vmax_lo(float2 v, float lo) {
+  return make_float2(v.x < lo ? lo : v.x, v.y < lo ? lo : v.y);
+}
+
+template <int M, bool SYM, int VEC = 1>
 struct OutputTile {
   static constexpr int N = M + 2;
+  using V = typename VecOf<VEC>::type;
   const Coefs& cf;
-  uint32_t sb_even, sb_odd;
+  uint32_t sb_even, sb_odd;      // VEC = 2 uses sb_even only
 
   template <int XI, int NU>
-  __device__ __forceinline__ void fill(float (&in)[N]) const {
+  __device__ __forceinline__ void fill(V (&in)[N]) const {
     if constexpr (NU < N) {
       constexpr int F = XI * N + NU;
-      in[NU] = (F & 1) ? sm100::lds_f32<F * 512>(sb_odd) : sm100::lds_f32<F * 512>(sb_even);
+      if constexpr (VEC == 1)
+        in[NU] = (F & 1) ? sm100::lds_f32<F * 512>(sb_odd) : sm100::lds_f32<F * 512>(sb_even);
+      else
+        in[NU] = sm100::lds_f32x2<F * 1024>(sb_even);
       fill<XI, NU + 1>(in);
     }
   }
   // z[j] = sum_nu A^T[j][nu] * M[xi][nu]
   template <int XI>
-  __device__ __forceinline__ void row(float (&z)[M]) const {
-    float in[N];
+  __device__ __forceinline__ void row(V (&z)[M]) const {
+    V in[N];
     fill<XI, 0>(in);
-    at_apply<M, SYM, float>(cf, in, z);
+    at_apply<M, SYM, V>(cf, in, z);
   }
   // dense: Y[i][j] += A^T[i][xi] * z_xi[j] for every xi
   template <int XI>
-  __device__ __forceinline__ void dense_from(float (&Y)[M][M]) const {
+  __device__ __forceinline__ void dense_from(V (&Y)[M][M]) const {
     if constexpr (XI < N) {
-      float z[M];
+      V z[M];
       row<XI>(z);
 #pragma unroll
       for (int i = 0; i < M; ++i)
 #pragma unroll
-        for (int j = 0; j < M; ++j) Y[i][j] = (XI == 0) ? cf.AT[i][0] * z[j] : fmaf(cf.AT[i][XI], z[j], Y[i][j]);
+        for (int j = 0; j < M; ++j) Y[i][j] = (XI == 0) ? vmul(cf.AT[i][0], z[j]) : vfma(cf.AT[i][XI], z[j], Y[i][j]);
       dense_from<XI + 1>(Y);
     }
   }
   // symmetric: rows +a / -a (Q, Q+1) share |coefficients|: even output rows take the sum of
   // the two row results, odd output rows the difference
   template <int Q>
-  __device__ __forceinline__ void pairs_from(float (&Y)[M][M]) const {
+  __device__ __forceinline__ void pairs_from(V (&Y)[M][M]) const {
     if constexpr (Q < N - 1) {
-      float zp[M], zm[M];
+      V zp[M], zm[M];
       row<Q>(zp);
       row<Q + 1>(zm);
 #pragma unroll
       for (int j = 0; j < M; ++j) {
-        const float s = zp[j] + zm[j], d = zp[j] - zm[j];
+        const V s = vadd(zp[j], zm[j]), d = vsub(zp[j], zm[j]);
 #pragma unroll
         for (int i = 0; i < M; ++i)
-          Y[i][j] = (Q == 1) ? cf.AT[i][1] * ((i & 1) ? d : s) : fmaf(cf.AT[i][Q], (i & 1) ? d : s, Y[i][j]);
+          Y[i][j] = (Q == 1) ? vmul(cf.AT[i][1], (i & 1) ? d : s) : vfma(cf.AT[i][Q], (i & 1) ? d : s, Y[i][j]);
       }
       pairs_from<Q + 2>(Y);
     }
   }
-  __device__ __forceinline__ void run(float (&Y)[M][M]) const {
+  __device__ __forceinline__ void run(V (&Y)[M][M]) const {
     if constexpr (!SYM) {
       dense_from<0>(Y);
     } else {
       pairs_from<1>(Y);
       // A^T column 0 is e_0 and column n-1 is e_{m-1}
-      float z0[M], zi[M];
+      V z0[M], zi[M];
       row<0>(z0);
       row<N - 1>(zi);
 #pragma unroll
       for (int j = 0; j < M; ++j) {
-        Y[0][j] += z0[j];
-        Y[M - 1][j] += zi[j];
+        Y[0][j] = vadd(Y[0][j], z0[j]);
+        Y[M - 1][j] = vadd(Y[M - 1][j], zi[j]);
       }
     }
   }
@@ -83,8 +95,8 @@ struct OutputTile {
 // Round Y to the storage type and store the m x m outputs of one (tile, filter): pixel (i, j)
 // goes to dst + (i * W + j) * K.  rows / cols = how many of the tile's rows / columns lie inside
 // the image (m for an interior tile: no per-store predicate then).  ReLU keeps NaN and +inf.
-template <int M, typename T>
-__device__ __forceinline__ void store_tile(const float (&Y)[M][M], T* dst, size_t row_stride, int K, int rows,
+template <int M, typename T, typename V>
+__device__ __forceinline__ void store_tile(const V (&Y)[M][M], T* dst, size_t row_stride, int K, int rows,
                                            int cols, int relu) {
   const float lo = relu ? 0.f : -__int_as_float(0x7f800000);
   if (rows >= M && cols >= M) {
@@ -93,8 +105,7 @@ __device__ __forceinline__ void store_tile(const float (&Y)[M][M], T* dst, size_
       T* p = dst;
 #pragma unroll
       for (int j = 0; j < M; ++j) {
-        const float v = Y[i][j];
-        vstore(p, v < lo ? lo : v);
+        vstore(p, vmax_lo(Y[i][j], lo));
         p += K;
       }
       dst += row_stride;
@@ -106,8 +117,7 @@ __device__ __forceinline__ void store_tile(const float (&Y)[M][M], T* dst, size_
         T* p = dst;
 #pragma unroll
         for (int j = 0; j < M; ++j) {
-          const float v = Y[i][j];
-          if (j < cols) vstore(p, v < lo ? lo : v);
+          if (j < cols) vstore(p, vmax_lo(Y[i][j], lo));
           p += K;
         }
       }

@@ -29,11 +29,12 @@ using namespace xf;
 constexpr int kConsGroups = 3;
 constexpr int kOtThreads = 32 * (1 + 4 * kConsGroups);
 
-template <int M>
+template <int M, int VEC>
 struct OtCfg {
   static constexpr int N = M + 2;
   static constexpr int NF = N * N;
-  static constexpr int kStageBytes = NF * 512;        // NF * 4 rows of 128 bytes; a multiple of 1024
+  static constexpr int kQuads = 4 * VEC;              // filter quads per unit: 16 * VEC filters
+  static constexpr int kStageBytes = NF * kQuads * 128;   // NF * kQuads rows of 128 bytes; a multiple of 1024
   // a multiple of the number of consumer groups: a stage is always read by the same group, so
   // no warp can get two phases ahead of a barrier it waits on by parity
   static constexpr int kStages = ((200 * 1024 / kStageBytes) >= 6 ? 6 : 3);
@@ -42,14 +43,14 @@ struct OtCfg {
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;
 };
 
-template <int M, typename T, bool SYM>
+template <int M, typename T, bool SYM, int VEC>
 __global__ void __launch_bounds__(kOtThreads, 1)
 output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
                             T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
                             int pc_pad, int relu, int* __restrict__ status) {
-  using Cfg = OtCfg<M>;
-  constexpr int N = Cfg::N;
+  using Cfg = OtCfg<M, VEC>;
   constexpr int kStages = Cfg::kStages;
+  constexpr int kUnitK = 16 * VEC;                    // filters per unit
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarrierOffset);
@@ -58,7 +59,7 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int KG = (K + 15) >> 4;                       // filter groups of 16
+  const int KG = (K + kUnitK - 1) / kUnitK;           // filter groups of 16 * VEC
   const int TG = pc_pad >> 3;                         // tile groups of 8 (pc_pad is a multiple of 128)
   // Unit i of this CTA is unit blockIdx.x + i * gridDim.x: ascending tiles chip-wide, i.e. the
   // rows of M the product kernel wrote last (still in L2) first.
@@ -82,7 +83,7 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
       if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
       if (lane == 0) {
         mbar_expect_tx(&full_bar[stage], Cfg::kStageBytes);
-        tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, &tmM, &full_bar[stage], tg * 32, kg * 4, 0);
+        tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, &tmM, &full_bar[stage], tg * 32, kg * Cfg::kQuads, 0);
       }
       __syncwarp();
     }
@@ -91,11 +92,13 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
     const int group = (warp - 1) >> 2;
     const int w = (warp - 1) & 3;
     const int t = w + 4 * (lane >> 4);                // tile within the unit's 8
-    const int kq = (lane & 15) >> 2, kk = lane & 3;   // filter quad within the unit's 4, filter in quad
-    // byte offsets of this lane's value inside an even / odd frequency's 4 rows (128B swizzle:
-    // the 16-byte chunk index is XORed with the row index modulo 8)
+    // filter quad within the unit, filter (pair) in the quad, and the byte offsets of this lane's
+    // value(s) inside a frequency's rows (128B swizzle: the 16-byte chunk index is XORed with the
+    // row index modulo 8; with 4 rows per frequency even and odd frequencies differ)
+    const int kq = (VEC == 1) ? (lane & 15) >> 2 : (lane & 15) >> 1;
+    const int kk = (VEC == 1) ? (lane & 3) : (lane & 1) * 2;
     const uint32_t off_even = kq * 128 + ((t ^ kq) << 4) + kk * 4;
-    const uint32_t off_odd = kq * 128 + ((t ^ (kq + 4)) << 4) + kk * 4;
+    const uint32_t off_odd = kq * 128 + ((t ^ ((kq + 4) & 7)) << 4) + kk * 4;
     for (uint32_t local = group; local < n_local && !timed_out; local += kConsGroups) {
       const unsigned u = blockIdx.x + local * gridDim.x;
       const int kg = (int)(u % (unsigned)KG), tg = (int)(u / (unsigned)KG);
@@ -103,13 +106,13 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
       if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
       const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
       const uint32_t sb_even = sb + off_even, sb_odd = sb + off_odd;
-      float Y[M][M];
-      OutputTile<M, SYM>{cf, sb_even, sb_odd}.run(Y);
+      typename VecOf<VEC>::type Y[M][M];
+      OutputTile<M, SYM, VEC>{cf, sb_even, sb_odd}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
 
       const int pl = tg * 8 + t;
-      const int k = kg * 16 + (lane & 15);
+      const int k = kg * kUnitK + (lane & 15) * VEC;
       if (pl < pc && k < K) {
         const unsigned p = (unsigned)(p0 + pl);
         const unsigned tw = p % (unsigned)Tw, q2 = p / (unsigned)Tw;
@@ -146,20 +149,20 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int M, typename T, bool SYM>
+template <int M, typename T, bool SYM, int VEC>
 int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
                int pc_pad, int relu, cudaStream_t stream) {
-  using Cfg = OtCfg<M>;
+  using Cfg = OtCfg<M, VEC>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM>,
+    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
-  const long long units = (long long)(pc_pad / 8) * ((g.K + 15) / 16);
+  const long long units = (long long)(pc_pad / 8) * ((g.K + 16 * VEC - 1) / (16 * VEC));
   const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
-  output_transform_tma_kernel<M, T, SYM><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
+  output_transform_tma_kernel<M, T, SYM, VEC><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
       tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev);
   return (int)cudaGetLastError();
 }
@@ -173,7 +176,8 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
   const int k4 = g.K / 4;
   cuuint64_t dims[3] = {(cuuint64_t)pc_pad * 4, (cuuint64_t)k4, (cuuint64_t)(g.n * g.n)};
   cuuint64_t strides[2] = {(cuuint64_t)pc_pad * 16, (cuuint64_t)k4 * pc_pad * 16};
-  cuuint32_t box[3] = {32, 4, (cuuint32_t)(g.n * g.n)};
+  constexpr int VEC = (M <= 6) ? 2 : 1;               // packed fp32 pairs where the registers allow
+  cuuint32_t box[3] = {32, 4 * VEC, (cuuint32_t)(g.n * g.n)};
   cuuint32_t estr[3] = {1, 1, 1};
   if (enc(&tmM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(Mb), dims, strides, box, estr,
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -181,10 +185,10 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
     return (int)cudaErrorUnknown;
   const bool f32 = plan->mode == NOVA_FP32;
   if (plan->symmetric)
-    return f32 ? launch_one<M, float, true>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
-               : launch_one<M, __half, true>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
-  return f32 ? launch_one<M, float, false>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
-             : launch_one<M, __half, false>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
+    return f32 ? launch_one<M, float, true, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
+               : launch_one<M, __half, true, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
+  return f32 ? launch_one<M, float, false, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
+             : launch_one<M, __half, false, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
 }
 
 }  // namespace

@@ -164,6 +164,12 @@ __device__ __forceinline__ float lds_f32(uint32_t saddr) {
   return v;
 }
 template <int OFF>
+__device__ __forceinline__ float2 lds_f32x2(uint32_t saddr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(saddr), "n"(OFF));
+  return v;
+}
+template <int OFF>
 __device__ __forceinline__ void sts_b16(uint32_t saddr, unsigned short v) {
   asm volatile("st.shared.b16 [%0+%1], %2;" ::"r"(saddr), "n"(OFF), "h"(v) : "memory");
 }

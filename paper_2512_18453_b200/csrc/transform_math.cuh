@@ -18,10 +18,12 @@ __device__ __forceinline__ void st2(__half* p, float2 v) {
   *reinterpret_cast<__half2*>(p) = __floats2half2_rn(v.x, v.y);
 }
 __device__ __forceinline__ void st2(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
+// The 2-vector forms use Blackwell's packed single-precision instructions (two IEEE fp32
+// results per instruction, each rounded exactly like the scalar operation).
 __device__ __forceinline__ float2 fma2(float a, float2 b, float2 c) {
-  return make_float2(fmaf(a, b.x, c.x), fmaf(a, b.y, c.y));
+  return __ffma2_rn(make_float2(a, a), b, c);
 }
-__device__ __forceinline__ float2 mul2(float a, float2 b) { return make_float2(a * b.x, a * b.y); }
+__device__ __forceinline__ float2 mul2(float a, float2 b) { return __fmul2_rn(make_float2(a, a), b); }
 
 // Scalar / 2-vector arithmetic used by the output transform (VEC filters per thread).
 template <int VEC> struct VecOf;
@@ -35,9 +37,9 @@ __device__ __forceinline__ float2 vmul(float a, float2 b) { return mul2(a, b); }
 __device__ __forceinline__ float vfma(float a, float b, float c) { return fmaf(a, b, c); }
 __device__ __forceinline__ float2 vfma(float a, float2 b, float2 c) { return fma2(a, b, c); }
 __device__ __forceinline__ float vadd(float a, float b) { return a + b; }
-__device__ __forceinline__ float2 vadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 vadd(float2 a, float2 b) { return __fadd2_rn(a, b); }
 __device__ __forceinline__ float vsub(float a, float b) { return a - b; }
-__device__ __forceinline__ float2 vsub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 vsub(float2 a, float2 b) { return __fadd2_rn(a, make_float2(-b.x, -b.y)); }
 __device__ __forceinline__ float vrelu(float v) { return v < 0.f ? 0.f : v; }
 __device__ __forceinline__ float2 vrelu(float2 v) { return make_float2(v.x < 0.f ? 0.f : v.x, v.y < 0.f ? 0.f : v.y); }
 __device__ __forceinline__ void vstore(__half* p, float v) { *p = __float2half_rn(v); }
