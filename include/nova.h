@@ -109,9 +109,10 @@ int nova_plan_get_device_tables(const nova_plan* plan, float* AT_host, float* G_
  * Any other set keeps the caller's order and dense transforms.  Either pointer may be null. */
 int nova_plan_frequency_order(const nova_plan* plan, int* perm_host, int* symmetric_host);
 
-/* Tuning: how many CTAs of the single-kernel path run the input transform and the
- * transformed-domain product (the remaining ones run the output transform); 0, 0 restores
- * the default split.  Not thread-safe against concurrent nova_conv2d_fwd on the same plan. */
+/* Tuning of the single-kernel path (NOVA_FUSED): how many CTAs run the input transform; the
+ * others run the transformed-domain product and the output transform side by side.  n_product
+ * is ignored (kept for ABI stability); n_input = 0 restores the default share.  Not thread-safe
+ * against concurrent nova_conv2d_fwd on the same plan. */
 int nova_plan_set_role_split(nova_plan* plan, int n_input, int n_product);
 
 /* kappa_2 = sigma_max/sigma_min of the Vandermonde matrix V_ij = a_i^j over the

@@ -37,8 +37,7 @@ namespace {
 using namespace sm100;
 using namespace xf;
 
-constexpr int kFusedThreads = 640;     // 20 warps (5 per scheduler x 96 registers fill its register file):
-                                       // 11 of role I or G, then 9 of role O
+constexpr int kFusedThreads = 512;     // 16 warps x 128 registers: 11 of role I or G, then 5 of role O
 constexpr int kGWarps = 11;
 constexpr int kOWarpBase = 11;
 constexpr int BLOCK_M = 128;
@@ -146,8 +145,10 @@ template <int M>
 struct OCfg {
   static constexpr int N = M + 2;
   static constexpr int NF = N * N;
-  static constexpr int kStageBytes = NF * 512;
-  static constexpr int kGroups = 2;
+  static constexpr int VEC = (M <= 6) ? 2 : 1;        // filters per thread: packed fp32 pairs where the registers allow
+  static constexpr int kQuads = 4 * VEC;              // filter quads per unit (16 * VEC filters, 8 tiles)
+  static constexpr int kStageBytes = NF * kQuads * 128;
+  static constexpr int kGroups = 1;                   // one consumer group of four warps
   static constexpr int kStages = 2;
   static constexpr int kBytes = kStages * kStageBytes;
   static_assert(kStages % kGroups == 0, "stage ring");
@@ -157,7 +158,7 @@ struct GCfg {
   static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
   static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (OCfg<M>::kBytes > 70 * 1024) ? 2 : 3;   // what role O leaves of the SM's shared memory
+  static constexpr int kStages = 2;                   // what role O leaves of the SM's shared memory
   static constexpr int kBytes = kStages * kStageBytes;
 };
 constexpr int cmax(int a, int b) { return a > b ? a : b; }
@@ -398,7 +399,7 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
   const unsigned n_local = (num_items > (unsigned)rank) ? (num_items - rank + rp.nGO - 1) / rp.nGO : 0u;
   const int RP = rp.R * 128;
   const unsigned CB = (unsigned)((C + 127) / 128);
-  const uint32_t o_target = 16u * (uint32_t)((K + 15) >> 4) * 4u;     // see role O
+  const uint32_t o_target = 16u * (uint32_t)((K + 16 * OCfg<M>::VEC - 1) / (16 * OCfg<M>::VEC)) * 4u;   // see role O
 
   if (warp == 0) {
     uint32_t stage = 0, phase = 0;
@@ -519,8 +520,8 @@ __device__ __forceinline__ void output_init(uint64_t* bars) {
   constexpr int kStages = OCfg<M>::kStages;
   for (int s = 0; s < kStages; ++s) { mbar_init(&bars[s], 1); mbar_init(&bars[kStages + s], 4); }
 }
-// Warps kGWarps .. kGWarps+8 of the CTA (`warp` is relative to kGWarps): one TMA producer and
-// two consumer groups of four warps.
+// Warps kOWarpBase .. kOWarpBase+4 of the CTA (`warp` is relative to kOWarpBase): one TMA producer
+// and one consumer group of four warps.
 template <int M, bool SYM>
 __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* bars, volatile int* abort_flag,
                                             const CUtensorMap* tmM, const Coefs& cf, __half* __restrict__ y,
@@ -534,7 +535,8 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
 
   const int lane = threadIdx.x & 31;
   const int K = cs.K, H = cs.H, W = cs.W;
-  const unsigned KG = (unsigned)((K + 15) >> 4);
+  constexpr int VEC = Cfg::VEC;
+  const unsigned KG = (unsigned)((K + 16 * VEC - 1) / (16 * VEC));
   const unsigned NB = (unsigned)((rp.P + 127) >> 7);
   const unsigned num_units = NB * 16u * KG;
   const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + size - 1) / size : 0u;
@@ -553,7 +555,7 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
       if (lane == 0) {
         mbar_expect_tx(&full_bar[stage], Cfg::kStageBytes);
         tma_load_3d(smem + (size_t)stage * Cfg::kStageBytes, tmM, &full_bar[stage],
-                    (int)((tg * 8u) % (unsigned)RP) * 4, (int)kg * 4, 0);
+                    (int)((tg * 8u) % (unsigned)RP) * 4, (int)kg * Cfg::kQuads, 0);
       }
       __syncwarp();
     }
@@ -561,9 +563,10 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
     const int group = (warp - 1) >> 2;
     const int w = (warp - 1) & 3;
     const int t = w + 4 * (lane >> 4);
-    const int kq = (lane & 15) >> 2, kk = lane & 3;
+    const int kq = (VEC == 1) ? (lane & 15) >> 2 : (lane & 15) >> 1;
+    const int kk = (VEC == 1) ? (lane & 3) : (lane & 1) * 2;
     const uint32_t off_even = kq * 128 + ((t ^ kq) << 4) + kk * 4;
-    const uint32_t off_odd = kq * 128 + ((t ^ (kq + 4)) << 4) + kk * 4;
+    const uint32_t off_odd = kq * 128 + ((t ^ ((kq + 4) & 7)) << 4) + kk * 4;
     for (unsigned local = group; local < n_local && !timed_out; local += Cfg::kGroups) {
       const unsigned u = rank + local * size;
       const unsigned tg = u / KG, kg = u % KG;
@@ -571,14 +574,14 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
       if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
       const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
       const uint32_t sb_even = sb + off_even, sb_odd = sb + off_odd;
-      float Y[M][M];
-      OutputTile<M, SYM>{cf, sb_even, sb_odd}.run(Y);
+      typename VecOf<VEC>::type Y[M][M];
+      OutputTile<M, SYM, VEC>{cf, sb_even, sb_odd}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
       ctr_signal_read(rp.o_done + (tg >> 4));
 
       const int pl = (int)tg * 8 + t;
-      const int k = (int)kg * 16 + (lane & 15);
+      const int k = (int)kg * 16 * VEC + (lane & 15) * VEC;
       if (pl < rp.P && k < K) {
         const unsigned p = (unsigned)pl;
         const unsigned tw = p % (unsigned)cs.Tw, q2 = p / (unsigned)cs.Tw;
@@ -725,7 +728,7 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     const int k4 = g.K / 4;
     cuuint64_t dims[3] = {(cuuint64_t)RP * 4, (cuuint64_t)k4, (cuuint64_t)NF};
     cuuint64_t strides[2] = {(cuuint64_t)RP * 16, (cuuint64_t)k4 * RP * 16};
-    cuuint32_t box[3] = {32, 4, (cuuint32_t)NF};
+    cuuint32_t box[3] = {32, (cuuint32_t)OCfg<M>::kQuads, (cuuint32_t)NF};
     if (!encode(&tmM, f32, 3, Mr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
   }
   const int NB = (int)((g.P + 127) / 128);
@@ -741,7 +744,7 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
   rp.P = (int)g.P;
   const int sms = plan->sm_count;
   int nI = plan->fused_nI;
-  if (nI <= 0 || nI >= sms) nI = sms * 30 / 100;      // default share of the SMs for role I
+  if (nI <= 0 || nI >= sms) nI = sms * 43 / 100;      // default share of the SMs for role I
   rp.nI = nI;
   rp.nGO = sms - nI;
   ConvShape cs{g.H, g.W, g.C, g.K, g.Th, g.Tw, relu};
