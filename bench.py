@@ -51,7 +51,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -138,6 +138,31 @@ def time_oracle(c, budget_s=20.0):
     return {"value": fl / best / 1e12, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
             "sample": "oracle.conv.direct_conv_fp64 (fp64, numpy) on %d of %d images of %s, best of 3"
                       % (n_img, c.N, c.name)}
+
+
+def accuracy_report(c, nv, torch, n_img=2):
+    """rel-L2 against the oracle's fp64 direct convolution, per point set of the workload, on the
+    first n_img images (images are independent): the GPU path, and the oracle's rounding
+    emulation of the same pipeline beside it.  Untimed."""
+    import numpy as np
+    from oracle import conv
+    from synth import make_conv_inputs, point_set
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    y1 = conv.direct_conv_fp64(x, g)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    rep = {}
+    for kind in c.point_kinds:
+        pts = point_set(kind, c.m)
+        plan = nv.Plan(c.m, pts, nv.FP16_F32ACC)
+        y = plan.conv2d(xd, plan.filter_transform(gd))
+        torch.cuda.synchronize()
+        yh = y.cpu().numpy().astype(np.float32)
+        e_gpu = conv.rel_l2(yh, y1)
+        e_emu = conv.rel_l2(conv.winograd_conv_emulated(x, g, c.m, pts, "fp16"), y1)
+        rep[kind] = {"kappa2_V": plan.kappa(), "rel_l2_gpu": e_gpu if np.isfinite(e_gpu) else None,
+                     "rel_l2_emulation": e_emu if np.isfinite(e_emu) else None,
+                     "nonfinite_outputs": int((~np.isfinite(yh)).sum())}
+    return {"sample": "first %d images of %s" % (n_img, c.name), "points": rep}
 
 
 def run_reference(args):
@@ -340,6 +365,11 @@ def run_ours(args):
         achieved, peak, runit = work / chunks / dur_launch / 1e12, peaks["tflops_burst"], "TFLOP/s"
     else:
         achieved, peak, runit = work / chunks / dur_launch / 1e9, peaks["hbm_gbs"], "GB/s"
+    traffic = None                 # DRAM bytes per launch of that kernel from the committed ncu capture
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath) and not fused and not args.images and chunks == 1:
+        with open(tpath) as f:
+            traffic = json.load(f).get(args.workload, {}).get(names[dom])
     roof_s = max(actual / (peaks["tflops_burst"] * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
     value = whole_job_value(world, direct, ms_per_step)
     out = {
@@ -362,7 +392,7 @@ def run_ours(args):
         "kernels_ms_per_step": {n_: v for n_, v in zip(names, kms) if n_ != "-"},
         "filter_transform_ms": filter_ms,
         "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
-                     "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"],
                      "launch_us": dur_launch * 1e6},
         "e2e": {"value": world * direct / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(x_np.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)},
@@ -372,6 +402,7 @@ def run_ours(args):
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
+        out["accuracy"] = accuracy_report(c, nv, torch)
         out["cpu_baseline"] = time_oracle(c)
     print(json.dumps(out))
     if dist is not None:
@@ -381,7 +412,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
