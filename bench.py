@@ -412,13 +412,120 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_vgg(args):
+    """cfg5: the 13 convolution layers of VGG-16 (ReLU in the epilogue, 2x2 max-pool between the
+    blocks) on a synthetic 224x224 batch, F(8,3) NOVA points unless --points says otherwise.
+    A step = the whole stack; reports images/s beside the direct-equivalent TFLOP/s."""
+    import numpy as np
+    import torch
+    import paper_2512_18453_b200 as nv
+    from synth import point_set, make_vgg_inputs, VGG16_LAYERS
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--workload cfg5 is a single-GPU report")
+    torch.cuda.set_device(0)
+    N = args.images or 32
+    m = args.tile
+    pts = point_set(args.points, m)
+    plan = nv.Plan(m, pts, nv.FP16_F32ACC)
+    x_np, weights = make_vgg_inputs(N)
+    x = torch.from_numpy(x_np).cuda()
+    Us = [plan.filter_transform(torch.from_numpy(w).cuda()) for w in weights]
+    flags = nv.RELU | (nv.FUSED if args.fused else 0)
+    # buffers: activations of every layer, one scratch sized for the largest layer
+    shapes, hw, c_in = [], 224, 8
+    for (ci, co, pool) in VGG16_LAYERS:
+        shapes.append((hw, max(ci, 8), co, pool))
+        hw = hw // 2 if pool else hw
+    ws_bytes = max(plan.workspace_bytes(N, h, h, ci, co) for (h, ci, co, _) in shapes) if args.workspace_mb is None \
+        else int(args.workspace_mb * (1 << 20))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    ys = [torch.empty(N, h, h, co, dtype=torch.float16, device="cuda") for (h, ci, co, _) in shapes]
+    ps = [torch.empty(N, h // 2, h // 2, co, dtype=torch.float16, device="cuda") if pool else None
+          for (h, ci, co, pool) in shapes]
+    L = nv.lib()
+
+    def step():
+        a = x
+        for i, (h, ci, co, pool) in enumerate(shapes):
+            plan.conv2d(a, Us[i], y=ys[i], workspace=ws, flags=flags)
+            a = ys[i]
+            if pool:
+                nv.binding._check(L.nova_maxpool2x2(a.data_ptr(), ps[i].data_ptr(), N, h, h, co, nv.FP16_F32ACC,
+                                                    nv.binding._stream()), "nova_maxpool2x2")
+                a = ps[i]
+        return a
+
+    out_t = step()
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(gr, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for _ in range(args.warmup):
+        gr.replay()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.1)
+    steps = min(args.steps, 200)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        gr.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.stop()
+    status = plan.device_status()
+    # per-layer durations (events around each convolution, direct launches, one extra pass)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in shapes]
+    a = x
+    for i, (h, ci, co, pool) in enumerate(shapes):
+        evs[i][0].record()
+        plan.conv2d(a, Us[i], y=ys[i], workspace=ws, flags=flags)
+        evs[i][1].record()
+        a = ys[i]
+        if pool:
+            nv.binding._check(L.nova_maxpool2x2(a.data_ptr(), ps[i].data_ptr(), N, h, h, co, nv.FP16_F32ACC,
+                                                nv.binding._stream()), "nova_maxpool2x2")
+            a = ps[i]
+    torch.cuda.synchronize()
+    layers_ms = ["%dx%d C%d K%d: %.3f" % (h, h, ci, co, e[0].elapsed_time(e[1])) for (h, ci, co, _), e in zip(shapes, evs)]
+    direct = sum(2.0 * N * h * h * co * ci_true * 9 for (h, _, co, _), (ci_true, _, _) in zip(shapes, VGG16_LAYERS))
+    launches = sum(plan.launch_count(N, h, h, ci, co, ws_bytes, flags) for (h, ci, co, _) in shapes) + 5
+    # accuracy on the first two images (images are independent), untimed
+    acc = None
+    if not args.no_cpu_baseline:
+        from oracle import conv
+        x2, _ = x_np[:2], None
+        ref = conv.vgg_stack_fp64(x2, weights, VGG16_LAYERS)
+        emu = conv.vgg_stack_emulated(x2, weights, VGG16_LAYERS, m, pts)
+        got = out_t[:2].cpu().numpy()
+        acc = {"sample": "first 2 images", "rel_l2_gpu": conv.rel_l2(got, ref), "rel_l2_emulation": conv.rel_l2(emu, ref)}
+    out = {
+        "metric": METRIC, "value": direct / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16 (f32 accumulate)", "data": "synthetic",
+        "config": {"workload": "cfg5: VGG-16 conv stack, 13 layers, N=%d, 224x224x3 (padded to 8 channels), F(%dx%d,3x3) %s points"
+                               % (N, m, m, args.points),
+                   "step": "13 x nova_conv2d_fwd (ReLU fused) + 5 x nova_maxpool2x2, CUDA graph replay",
+                   "workspace_mb": ws_bytes / (1 << 20), "fused": bool(args.fused)},
+        "images_per_s": N / (ms * 1e-3), "layers_ms": layers_ms, "gpu_launches": launches * steps, "device_status": status,
+        "accuracy": acc, "clocks": clocks,
+    }
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--tile", type=int, default=8, help="tile size m of the cfg5 stack")
     ap.add_argument("--points", default="nova")
     ap.add_argument("--gemm", default="auto", choices=["auto", "tcgen05", "simt"])
     ap.add_argument("--workspace-mb", type=float, default=None)
@@ -430,6 +537,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cfg5":
+        run_vgg(args)
     else:
         run_ours(args)
 
