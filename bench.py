@@ -257,6 +257,8 @@ def run_ours(args):
     flags = {"auto": 0, "tcgen05": nv.GEMM_TCGEN05, "simt": nv.GEMM_SIMT}[args.gemm]
     if args.fused:
         flags |= nv.FUSED
+    if args.two_kernel:
+        flags |= nv.FUSED_PRODUCT_OUTPUT
     if args.split:
         plan.set_role_split(*[int(v) for v in args.split.split(",")])
     launches = plan.launch_count(c.N, c.H, c.W, c.C, c.K, ws_bytes, flags)
@@ -347,7 +349,8 @@ def run_ours(args):
 
     peaks = read_peaks()
     fused = launches == 1
-    chunks = 1 if fused else launches // 3
+    two = launches == 2
+    chunks = 1 if (fused or two) else launches // 3
     names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
     n2 = (c.m + 2) ** 2
     elt = 2
@@ -371,7 +374,9 @@ def run_ours(args):
     else:
         achieved, peak, runit = work / chunks / dur_launch / 1e9, peaks["hbm_gbs"], "GB/s"
     traffic = None                 # DRAM bytes per launch of that kernel from the committed ncu capture
-    if not fused and not args.images and chunks == 1:
+    if two:
+        names = ["input_transform", "product+output (one kernel, M ring in L2)", "-"]
+    if not fused and not two and not args.images and chunks == 1:
         traffic = NCU_DRAM_BYTES.get(args.workload, {}).get(names[dom])
     roof_s = max(actual / (peaks["tflops_burst"] * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
     value = whole_job_value(world, direct, ms_per_step)
@@ -531,6 +536,7 @@ def main():
     ap.add_argument("--workspace-mb", type=float, default=None)
     ap.add_argument("--launch", default="graph", choices=["graph", "direct"])
     ap.add_argument("--fused", action="store_true", help="the single role-specialised kernel instead of one kernel per step")
+    ap.add_argument("--two-kernel", action="store_true", help="input transform, then product+output in one kernel")
     ap.add_argument("--split", default="", help="CTAs for the input-transform and product roles, e.g. 30,60")
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

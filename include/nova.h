@@ -53,6 +53,8 @@ enum {
   NOVA_FUSED = 1 << 11,     /* run the three steps as ONE persistent kernel whose CTAs are specialised
                                by role and exchange tiles through L2-resident rings (half mode, C >= 64;
                                otherwise ignored); the default is one kernel per step */
+  NOVA_FUSED_PRODUCT_OUTPUT = 1 << 12, /* two kernels: the input transform, then product and output transform
+                               in one kernel with the product M in an L2-resident ring (half mode, C >= 64) */
   NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
                                    where the tensor-core formulation applies, the output transform
                                    without TMA staging (testing) */

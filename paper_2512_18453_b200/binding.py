@@ -12,6 +12,7 @@ GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
 TRANSFORM_SIMT = 1 << 10
 FUSED = 1 << 11
+FUSED_PRODUCT_OUTPUT = 1 << 12
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",

@@ -68,6 +68,27 @@ bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, i
   return true;
 }
 
+// Two-kernel path: the input transform over all tiles, then ONE kernel for product and output
+// transform with M in an L2-resident ring of *R blocks.  The scratch holds V for all tiles
+// (padded to whole blocks) and the ring.
+bool two_kernel_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R, size_t* v_bytes) {
+  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev) return false;
+  if (!(flags & NOVA_FUSED_PRODUCT_OUTPUT) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT | NOVA_FUSED))) return false;
+  if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
+  const long long NB = (g.P + 127) / 128;
+  const size_t vb = round_up((size_t)g.n * g.n * NB * 128 * g.C * 2, kAlign);
+  const size_t mblock = (size_t)g.n * g.n * 128 * g.K * 4;
+  if (bytes < vb + 2 * kAlign) return false;
+  long long r = (long long)((bytes - vb - kAlign) / mblock);
+  if (r > NB) r = NB;
+  if (r > 8) r = 8;                                   // keep the ring well inside the L2
+  if (r < 2 && r < NB) return false;
+  if (r < 1) return false;
+  *R = (int)r;
+  *v_bytes = vb;
+  return true;
+}
+
 bool use_tcgen05(const nova_plan* p, int flags) {
   if (p->mode == NOVA_FP32) return false;
   return (flags & NOVA_GEMM_SIMT) == 0;
@@ -112,7 +133,9 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
   Geom g = make_geom(p, N, H, W, C, K);
   int R = 0;
+  size_t vb = 0;
   if (fused_applies(p, g, workspace_bytes, flags, &R)) return 1;
+  if (two_kernel_applies(p, g, workspace_bytes, flags, &R, &vb)) return 2;
   Chunking c;
   if (!choose_chunking(p, g, workspace_bytes, &c)) return NOVA_ERR_WORKSPACE;
   return 3 * c.chunks;
@@ -135,6 +158,20 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
     if (ev) cudaEventRecord(ev[1], s);
     const int e = launch_fused_conv(p, g, x, U, y, ws, R, (flags & NOVA_RELU) ? 1 : 0, stream);
     if (ev) cudaEventRecord(ev[2], s);
+    if (e) g_last_cuda_error = e;
+    return e ? NOVA_ERR_CUDA : NOVA_OK;
+  }
+  size_t vb = 0;
+  if (two_kernel_applies(p, g, ws_bytes, flags, &R, &vb)) {
+    cudaStream_t s = (cudaStream_t)stream;
+    const int pad = (int)((g.P + 127) / 128 * 128);
+    if (ev) cudaEventRecord(ev[0], s);
+    int e = launch_input_transform_tc(p, g, x, ws, 0, (int)g.P, pad, stream);
+    if (ev) cudaEventRecord(ev[1], s);
+    if (!e)
+      e = launch_fused_product_output(p, g, x, ws, U, y, reinterpret_cast<float*>(static_cast<char*>(ws) + vb), R,
+                                      (flags & NOVA_RELU) ? 1 : 0, stream);
+    if (ev) { cudaEventRecord(ev[2], s); cudaEventRecord(ev[3], s); }
     if (e) g_last_cuda_error = e;
     return e ? NOVA_ERR_CUDA : NOVA_OK;
   }
@@ -182,8 +219,8 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   if (!kernel_ms) return NOVA_ERR_INVALID_ARG;
   const int launches = nova_conv2d_launch_count(p, N, H, W, C, K, ws_bytes, flags);
   if (launches < 0) return launches;
-  const bool fused = launches == 1;
-  const int chunks = fused ? 1 : launches / 3;
+  const bool fused = launches == 1, two = launches == 2;
+  const int chunks = (fused || two) ? 1 : launches / 3;
   cudaEvent_t* ev = new cudaEvent_t[4 * chunks];
   for (int i = 0; i < 4 * chunks; ++i) cudaEventCreate(&ev[i]);
   int st = conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, ev);
@@ -191,6 +228,9 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
   if (st == NOVA_OK && fused) {
     cudaEventElapsedTime(&kernel_ms[1], ev[1], ev[2]);      // the one kernel does all three steps
+  } else if (st == NOVA_OK && two) {
+    cudaEventElapsedTime(&kernel_ms[0], ev[0], ev[1]);      // input transform
+    cudaEventElapsedTime(&kernel_ms[1], ev[1], ev[2]);      // product + output transform in one kernel
   } else if (st == NOVA_OK)
     for (int c = 0; c < chunks; ++c)
       for (int k = 0; k < 3; ++k) {

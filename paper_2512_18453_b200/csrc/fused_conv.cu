@@ -49,9 +49,11 @@ struct RingParams {
   uint32_t* g_done;      // [NB]
   uint32_t* o_done;      // [NB]
   int* abort_all;        // set by any CTA that gives up
-  int R;                 // ring length in 128-tile blocks
+  int R;                 // ring length of M in 128-tile blocks
+  int RV;                // ring length of V (all blocks when V was produced by an earlier kernel: nI == 0)
   int P;                 // tiles
   int nI, nGO;           // CTAs of role I; the others run roles G and O together
+  uint32_t g_target;     // g_done value of a finished block: n^2 * (filter blocks) * 4
 };
 
 struct ConvShape {
@@ -76,6 +78,30 @@ __device__ __forceinline__ bool ctr_wait_warp(const uint32_t* ctr, uint32_t targ
   if ((threadIdx.x & 31) == 0) ok = ctr_wait(ctr, target, abort_flag, abort_all) ? 1u : 0u;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
+// A counter check whose load was issued one work item ahead (the load is asynchronous until its
+// value is used), so that a dependency that is already satisfied costs no round trip to L2 on
+// the producer's critical path.  Lane 0 holds the state; gate() returns the verdict to all lanes.
+struct CtrGate {
+  uint32_t val;
+  int block;      // block the prefetched value belongs to (-1: none)
+  __device__ __forceinline__ void prefetch(const uint32_t* ctrs, int b) {
+    if ((threadIdx.x & 31) == 0) {
+      block = b;
+      val = 0;
+      if (b >= 0) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(val) : "l"(ctrs + b) : "memory");
+    }
+  }
+  __device__ __forceinline__ bool gate(const uint32_t* ctrs, int b, uint32_t target, volatile int* abort_flag,
+                                       const int* abort_all) {
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+      ok = (block == b && val >= target) ? 1u : 0u;
+      if (!ok) ok = ctr_wait(ctrs + b, target, abort_flag, abort_all) ? 1u : 0u;
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+  }
+};
+
 // Called by all lanes of a warp after their global stores (or shared-memory reads) of a unit.
 __device__ __forceinline__ void ctr_signal(uint32_t* ctr) {
   __syncwarp();
@@ -251,8 +277,8 @@ __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32
   const unsigned CB = (unsigned)((C + 127) / 128);
   const unsigned num_units = (unsigned)rp.P * CB;
   const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + rp.nI - 1) / rp.nI : 0u;
-  const int RP = rp.R * 128;
-  const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((cs.K + 255) / 256) * 4u;   // see role G
+  const int RP = rp.RV * 128;
+  const uint32_t g_target = rp.g_target;
 
   if (warp < Cfg::kProd) {
     if (warp == 0 && lane == 0) {
@@ -266,7 +292,7 @@ __device__ __forceinline__ void role_input(uint8_t* smem, uint64_t* bars, uint32
       const unsigned tw = p % (unsigned)cs.Tw, q2 = p / (unsigned)cs.Tw;
       const unsigned th = q2 % (unsigned)cs.Th, img = q2 / (unsigned)cs.Th;
       const int b = (int)(p >> 7);
-      if (b >= rp.R && !ctr_wait_warp(rp.g_done + (b - rp.R), g_target, abort_flag, rp.abort_all)) {
+      if (b >= rp.RV && !ctr_wait_warp(rp.g_done + (b - rp.RV), g_target, abort_flag, rp.abort_all)) {
         timed_out = true; break;
       }
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
@@ -403,20 +429,21 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
 
   if (warp == 0) {
     uint32_t stage = 0, phase = 0;
+    CtrGate gate_v{0, -1}, gate_o{0, -1};
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
       const unsigned it = rank + local * rp.nGO;
       const unsigned pb = it / per_block, rem = it % per_block;
       const unsigned f = rem / num_kb, kb = rem % num_kb;
       int tiles = rp.P - (int)pb * 128;
       tiles = tiles > 128 ? 128 : tiles;
-      if (!ctr_wait_warp(rp.v_ready + pb, (uint32_t)tiles * CB * 4u, abort_flag, rp.abort_all)) {
+      if (rp.nI > 0 && !gate_v.gate(rp.v_ready, (int)pb, (uint32_t)tiles * CB * 4u, abort_flag, rp.abort_all)) {
         timed_out = true; break;
       }
-      if ((int)pb >= rp.R && !ctr_wait_warp(rp.o_done + (pb - rp.R), o_target, abort_flag, rp.abort_all)) {
+      if ((int)pb >= rp.R && !gate_o.gate(rp.o_done, (int)pb - rp.R, o_target, abort_flag, rp.abort_all)) {
         timed_out = true; break;
       }
       async_proxy_acquire();
-      const int row0 = (int)(pb % (unsigned)rp.R) * 128;
+      const int row0 = (int)(pb % (unsigned)rp.RV) * 128;
       for (int ks = 0; ks < num_ks; ++ks) {
         if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
         if (lane == 0) {
@@ -428,6 +455,11 @@ __device__ __forceinline__ void role_gemm(uint8_t* smem, uint64_t* bars, uint32_
         }
         __syncwarp();
         if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+      if (local + 1 < n_local) {                       // look one item ahead
+        const int npb = (int)((rank + (local + 1) * rp.nGO) / per_block);
+        if (rp.nI > 0) gate_v.prefetch(rp.v_ready, npb);
+        gate_o.prefetch(rp.o_done, npb >= rp.R ? npb - rp.R : -1);
       }
     }
   } else if (warp == 1) {
@@ -541,14 +573,15 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
   const unsigned num_units = NB * 16u * KG;
   const unsigned n_local = (num_units > (unsigned)rank) ? (num_units - rank + size - 1) / size : 0u;
   const int RP = rp.R * 128;
-  const uint32_t g_target = (uint32_t)(Cfg::NF) * (uint32_t)((K + 255) / 256) * 4u;
+  const uint32_t g_target = rp.g_target;
 
   if (warp == 0) {
+    CtrGate gate_g{0, -1};
     for (unsigned local = 0; local < n_local && !timed_out; ++local) {
       const unsigned u = rank + local * size;
       const unsigned tg = u / KG, kg = u % KG;
       const unsigned b = tg >> 4;
-      if (!ctr_wait_warp(rp.g_done + b, g_target, abort_flag, rp.abort_all)) { timed_out = true; break; }
+      if (!gate_g.gate(rp.g_done, (int)b, g_target, abort_flag, rp.abort_all)) { timed_out = true; break; }
       async_proxy_acquire();
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
@@ -558,6 +591,7 @@ __device__ __forceinline__ void role_output(int warp, uint8_t* smem, uint64_t* b
                     (int)((tg * 8u) % (unsigned)RP) * 4, (int)kg * Cfg::kQuads, 0);
       }
       __syncwarp();
+      if (local + 1 < n_local) gate_g.prefetch(rp.g_done, (int)(((rank + (local + 1) * size) / KG) >> 4));
     }
   } else if (warp <= 4 * Cfg::kGroups) {
     const int group = (warp - 1) >> 2;
@@ -683,9 +717,11 @@ bool encode(CUtensorMap* map, CUtensorMapDataType dt, int rank, const void* base
              swz, promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// nI_req < 0: the plan's (or the default) share of CTAs runs role I and V is a ring of R blocks;
+// nI_req == 0: V (all tiles) was produced by an earlier kernel and every CTA runs roles G and O.
 template <int M, int BLOCK_N, bool SYM>
 int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* Vr,
-                   float* Mr, int R, int relu, cudaStream_t stream) {
+                   float* Mr, int R, int nI_req, int relu, cudaStream_t stream) {
   using F = FusedCfg<M, BLOCK_N>;
   constexpr int n = M + 2, NF = n * n;
   static bool attr_set = false;
@@ -695,7 +731,9 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
-  const int RP = R * 128;
+  const int NB = (int)((g.P + 127) / 128);
+  const int RV = (nI_req == 0) ? NB : R;
+  const int RP = R * 128, RPV = RV * 128;
   CUtensorMap tmX, tmK, tmV, tmU, tmM;
   const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
   const CUtensorMapL2promotion p256 = CU_TENSOR_MAP_L2_PROMOTION_L2_256B, p128 = CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
@@ -713,8 +751,8 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     if (!encode(&tmK, f16, 2, plan->kron_dev, dims, strides, box, p256)) return (int)cudaErrorUnknown;
   }
   {
-    cuuint64_t dims[3] = {(cuuint64_t)g.C, (cuuint64_t)RP, (cuuint64_t)NF};
-    cuuint64_t strides[2] = {(cuuint64_t)g.C * 2, (cuuint64_t)RP * g.C * 2};
+    cuuint64_t dims[3] = {(cuuint64_t)g.C, (cuuint64_t)RPV, (cuuint64_t)NF};
+    cuuint64_t strides[2] = {(cuuint64_t)g.C * 2, (cuuint64_t)RPV * g.C * 2};
     cuuint32_t box[3] = {BLOCK_K, BLOCK_M, 1};
     if (!encode(&tmV, f16, 3, Vr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
   }
@@ -731,7 +769,6 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
     cuuint32_t box[3] = {32, (cuuint32_t)OCfg<M>::kQuads, (cuuint32_t)NF};
     if (!encode(&tmM, f32, 3, Mr, dims, strides, box, p128)) return (int)cudaErrorUnknown;
   }
-  const int NB = (int)((g.P + 127) / 128);
   uint32_t* ctr = plan->fused_ctr_dev;
   if (cudaMemsetAsync(ctr, 0, (size_t)(3 * NB + 4) * sizeof(uint32_t), stream) != cudaSuccess)
     return (int)cudaErrorUnknown;
@@ -741,12 +778,15 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
   rp.o_done = ctr + 2 * NB;
   rp.abort_all = reinterpret_cast<int*>(ctr + 3 * NB);
   rp.R = R;
+  rp.RV = RV;
   rp.P = (int)g.P;
   const int sms = plan->sm_count;
   int nI = plan->fused_nI;
   if (nI <= 0 || nI >= sms) nI = sms * 43 / 100;      // default share of the SMs for role I
+  if (nI_req == 0) nI = 0;
   rp.nI = nI;
   rp.nGO = sms - nI;
+  rp.g_target = (uint32_t)NF * (uint32_t)((g.K + BLOCK_N - 1) / BLOCK_N) * 4u;
   ConvShape cs{g.H, g.W, g.C, g.K, g.Th, g.Tw, relu};
 
   cudaLaunchConfig_t cfg = {};
@@ -765,9 +805,9 @@ int launch_fused_t(const nova_plan* plan, const Geom& g, const void* x, const vo
 
 template <int M>
 int launch_fused_m(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* Vr,
-                   float* Mr, int R, int relu, cudaStream_t s) {
-  if (plan->symmetric) return launch_fused_t<M, 256, true>(plan, g, x, U, y, Vr, Mr, R, relu, s);
-  return launch_fused_t<M, 256, false>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+                   float* Mr, int R, int nI_req, int relu, cudaStream_t s) {
+  if (plan->symmetric) return launch_fused_t<M, 256, true>(plan, g, x, U, y, Vr, Mr, R, nI_req, relu, s);
+  return launch_fused_t<M, 256, false>(plan, g, x, U, y, Vr, Mr, R, nI_req, relu, s);
 }
 
 }  // namespace
@@ -783,10 +823,25 @@ int launch_fused_conv(const nova_plan* plan, const Geom& g, const void* x, const
   void* Vr = ws;
   float* Mr = reinterpret_cast<float*>(static_cast<char*>(ws) + v_bytes);
   switch (plan->m) {
-    case 2: return launch_fused_m<2>(plan, g, x, U, y, Vr, Mr, R, relu, s);
-    case 4: return launch_fused_m<4>(plan, g, x, U, y, Vr, Mr, R, relu, s);
-    case 6: return launch_fused_m<6>(plan, g, x, U, y, Vr, Mr, R, relu, s);
-    case 8: return launch_fused_m<8>(plan, g, x, U, y, Vr, Mr, R, relu, s);
+    case 2: return launch_fused_m<2>(plan, g, x, U, y, Vr, Mr, R, -1, relu, s);
+    case 4: return launch_fused_m<4>(plan, g, x, U, y, Vr, Mr, R, -1, relu, s);
+    case 6: return launch_fused_m<6>(plan, g, x, U, y, Vr, Mr, R, -1, relu, s);
+    case 8: return launch_fused_m<8>(plan, g, x, U, y, Vr, Mr, R, -1, relu, s);
+  }
+  return (int)cudaErrorInvalidValue;
+}
+
+// Product and output transform in one kernel over a V that holds all tiles ([n*n][P_pad][C], written by
+// the input-transform kernel before): every CTA runs roles G and O, M is a ring of R blocks.
+int launch_fused_product_output(const nova_plan* plan, const Geom& g, const void* x, const void* V, const void* U,
+                                void* y, float* Mring, int R, int relu, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  void* Vr = const_cast<void*>(V);
+  switch (plan->m) {
+    case 2: return launch_fused_m<2>(plan, g, x, U, y, Vr, Mring, R, 0, relu, s);
+    case 4: return launch_fused_m<4>(plan, g, x, U, y, Vr, Mring, R, 0, relu, s);
+    case 6: return launch_fused_m<6>(plan, g, x, U, y, Vr, Mring, R, 0, relu, s);
+    case 8: return launch_fused_m<8>(plan, g, x, U, y, Vr, Mring, R, 0, relu, s);
   }
   return (int)cudaErrorInvalidValue;
 }

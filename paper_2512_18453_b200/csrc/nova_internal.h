@@ -80,6 +80,8 @@ int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void
                                 long long p0, int pc, int pc_pad, int relu, void* stream);
 int launch_fused_conv(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* ws,
                       int R, int relu, void* stream);
+int launch_fused_product_output(const nova_plan* plan, const Geom& g, const void* x, const void* V, const void* U,
+                                void* y, float* Mring, int R, int relu, void* stream);
 size_t fused_block_bytes(const nova_plan* plan, int C, int K);
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,
                      int nfreq, int pc, int pc_pad, int C, int K, void* stream);

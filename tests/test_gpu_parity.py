@@ -187,6 +187,14 @@ def test_single_kernel_path_matches_three_kernel_path(kind, m, shape, ws_blocks)
     assert plan.device_status() == 0
     assert np.array_equal(ya.cpu().numpy(), yb.cpu().numpy())
     check_fp16(ya.cpu().numpy(), x, g, m, pts)
+    # the two-kernel variant: input transform, then product and output transform in one kernel
+    ws2 = torch.empty(plan.workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device="cuda")
+    assert plan.launch_count(N, H, W, C, K, ws2.numel(), nv.FUSED_PRODUCT_OUTPUT) == 2
+    yc = torch.full((N, H, W, K), float("nan"), dtype=torch.float16, device="cuda")
+    plan.conv2d(xd, U, y=yc, workspace=ws2, flags=nv.FUSED_PRODUCT_OUTPUT)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert np.array_equal(yc.cpu().numpy(), yb.cpu().numpy())
 
 
 @pytest.mark.parametrize("kind,m,shape", [("nova", 8, (16, 28, 28, 512, 64)), ("nova", 4, (8, 40, 40, 256, 64)),
@@ -204,6 +212,8 @@ def test_many_units_per_cta_in_every_ring(kind, m, shape):
     assert abs(ea - eb) <= 0.05 * eb and conv.rel_l2(ya, yb) < 0.3 * eb
     yc, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.FUSED)
     assert np.array_equal(ya, yc)
+    yd, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, nv.FUSED_PRODUCT_OUTPUT)
+    assert np.array_equal(ya, yd)
 
 
 def test_ragged_last_row_block_after_full_blocks():
