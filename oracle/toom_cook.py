@@ -42,7 +42,7 @@ def _poly_mul_linear(coeffs, root):
     return out
 
 
-def build_matrices(m, r, points):
+def build_matrices(m, r, points, scale_G=None, scale_B=None):
     """Exact A^T (m x n), G (n x r), B^T (n x n) as nested lists of Fraction.
 
     Algorithm 3, in its own order:
@@ -53,6 +53,12 @@ def build_matrices(m, r, points):
       B^T[p][:] = coefficients (ascending) of prod_{j != p} (t - alpha_j),
                   zero padded to n; infinity row = coefficients of
                   prod_j (t - alpha_j)
+
+    scale_G / scale_B (optional, one non-zero rational per point) apply the
+    diagonal rescaling of the comparison with learned-scale methods
+    (Appendix "Relation to complementary techniques"): D_G multiplies the rows
+    of G, D_B the rows of B^T, and D_A = (D_G D_B)^-1 the columns of A^T, so
+    that D_A D_G D_B = I and the bilinear identity is unchanged.
     """
     n = m + r - 1
     if len(points) != n:
@@ -89,7 +95,38 @@ def build_matrices(m, r, points):
         poly = _poly_mul_linear(poly, al[j])
     for j, c in enumerate(poly):
         BT[n - 1][j] = c
+    if scale_G is not None or scale_B is not None:
+        sg = [Fraction(1)] * n if scale_G is None else [Fraction(*v) if isinstance(v, tuple) else Fraction(v) for v in scale_G]
+        sb = [Fraction(1)] * n if scale_B is None else [Fraction(*v) if isinstance(v, tuple) else Fraction(v) for v in scale_B]
+        if len(sg) != n or len(sb) != n or any(v == 0 for v in sg + sb):
+            raise ValueError("need one non-zero scale per point")
+        for p in range(n):
+            G[p] = [sg[p] * v for v in G[p]]
+            BT[p] = [sb[p] * v for v in BT[p]]
+            for i in range(m):
+                AT[i][p] = AT[i][p] / (sg[p] * sb[p])
     return AT, G, BT
+
+
+def snap_to_rational(x, d_max=10):
+    """Nearest simple rational (Definition "Snap-to-Rational", Section "Snap-to-Rational";
+    Algorithm 2): argmin |x - a/b| over 1 <= b <= d_max, |a| <= 5 b.  Candidates are visited
+    by increasing denominator, then increasing numerator, and only a strictly smaller
+    distance replaces the incumbent, so ties keep the first (smallest-denominator) one."""
+    x = Fraction(x)
+    best, best_dist = None, None
+    for b in range(1, d_max + 1):
+        for a in range(-5 * b, 5 * b + 1):
+            f = Fraction(a, b)
+            dist = abs(x - f)
+            if best is None or dist < best_dist:
+                best, best_dist = f, dist
+    return best
+
+
+def norm2(M):
+    """Spectral norm (largest singular value)."""
+    return float(np.linalg.svd(np.asarray(M, dtype=np.float64), compute_uv=False)[0])
 
 
 def decomposition_residual(m, r, AT, G, BT):

@@ -33,6 +33,8 @@ POINT_SETS = {
     ("nova", 4): _sym((5, 6), (7, 6)),
     ("nova", 6): _sym((3, 5), (1, 1), (7, 6)),
     ("nova", 8): _sym((2, 5), (5, 6), (1, 1), (7, 6)),
+    # Table "Dtype-aware vs unconstrained discovery": dyadic points, exact in binary16
+    ("dyadic", 4): _sym((3, 4), (5, 4)),
 }
 
 
