@@ -155,18 +155,28 @@ def accuracy_report(c, nv, torch, n_img=2):
     x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
     y1 = conv.direct_conv_fp64(x, g)
     xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    from synth import pow2_range_scales
     rep = {}
     for kind in c.point_kinds:
         pts = point_set(kind, c.m)
-        plan = nv.Plan(c.m, pts, nv.FP16_F32ACC)
-        y = plan.conv2d(xd, plan.filter_transform(gd))
-        torch.cuda.synchronize()
-        yh = y.cpu().numpy().astype(np.float32)
-        e_gpu = conv.rel_l2(yh, y1)
-        e_emu = conv.rel_l2(conv.winograd_conv_emulated(x, g, c.m, pts, "fp16"), y1)
-        rep[kind] = {"kappa2_V": plan.kappa(), "rel_l2_gpu": e_gpu if np.isfinite(e_gpu) else None,
-                     "rel_l2_emulation": e_emu if np.isfinite(e_emu) else None,
-                     "nonfinite_outputs": int((~np.isfinite(yh)).sum())}
+        # each set as constructed, and with power-of-two row scales that normalise the range of
+        # U and V (diagonal rescaling D_A D_G D_B = I; conditioning unchanged)
+        for label, scaled in ((kind, False), (kind + "+pow2_rows", True)):
+            sc = (None, None)
+            if scaled:
+                _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC).matrices()
+                sc = pow2_range_scales(G, BT)
+            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, scale_G=sc[0], scale_B=sc[1])
+            y = plan.conv2d(xd, plan.filter_transform(gd))
+            torch.cuda.synchronize()
+            yh = y.cpu().numpy().astype(np.float32)
+            e_gpu = conv.rel_l2(yh, y1)
+            e_emu = conv.rel_l2(conv.winograd_conv_emulated(x, g, c.m, pts, "fp16", scales=sc), y1)
+            kap, nrm = plan.kappa_matrices()
+            rep[label] = {"kappa2_V": plan.kappa(), "kappa2_A_G_B": list(kap), "norm_product": nrm[0] * nrm[1] * nrm[2],
+                          "rel_l2_gpu": e_gpu if np.isfinite(e_gpu) else None,
+                          "rel_l2_emulation": e_emu if np.isfinite(e_emu) else None,
+                          "nonfinite_outputs": int((~np.isfinite(yh)).sum())}
     return {"sample": "first %d images of %s" % (n_img, c.name), "points": rep}
 
 
@@ -409,8 +419,9 @@ def run_ours(args):
         "kappa2_V": plan.kappa(),
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and (args.accuracy or not args.no_cpu_baseline):
         out["accuracy"] = accuracy_report(c, nv, torch)
+    if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = time_oracle(c)
     print(json.dumps(out))
     if dist is not None:
@@ -539,6 +550,8 @@ def main():
     ap.add_argument("--two-kernel", action="store_true", help="input transform, then product+output in one kernel")
     ap.add_argument("--split", default="", help="CTAs for the input-transform and product roles, e.g. 30,60")
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
+    ap.add_argument("--accuracy", action="store_true",
+                    help="report rel-L2 per point set (and per rescaled variant) even with --no-cpu-baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

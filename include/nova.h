@@ -94,6 +94,48 @@ int nova_plan_create(int m, int r, const nova_rat* points_host, int n,
                      int mode, int coef, nova_plan** out);
 void nova_plan_destroy(nova_plan* plan);
 
+/*
+ * The same construction with a diagonal rescaling (the form Y = D_A A^T [(D_G G g) (.) (D_B B^T d)]
+ * of the appendix comparing learned-scale methods): row p of G is multiplied by scale_G[p], row p of
+ * B^T by scale_B[p] and column p of A^T by 1 / (scale_G[p] scale_B[p]), so that D_A D_G D_B = I and
+ * the exact identity still holds (it is checked again).  Either scale array may be null (all ones);
+ * each holds n non-zero finite rationals, the last one for the point at infinity.  Scales that differ
+ * within a +-pair, or whose product scale_G scale_B is not 1 at the point 0 or at infinity, make the
+ * plan non-symmetric (dense transforms, same results).  Powers of two change no rounding,
+ * only the range of U and V - e.g. to keep a large tile inside binary16.
+ */
+int nova_plan_create_scaled(int m, int r, const nova_rat* points_host, int n,
+                            const nova_rat* scale_G_host, const nova_rat* scale_B_host,
+                            int mode, int coef, nova_plan** out);
+
+/*
+ * Snap-to-rational (Algorithm 2; definition in Section "Snap-to-Rational"): the a/b with
+ * 1 <= b <= max_den and |a| <= 5 b closest to x, compared exactly; of equally close candidates the
+ * one met first when b, then a, increase.  Returned in lowest terms.  1 <= max_den <= 4096.
+ */
+int nova_snap_to_rational(double x, int max_den, nova_rat* out);
+
+/* Snap n_finite continuous points (the paper uses max_den = 10), append infinity and build the
+ * plan; NOVA_ERR_DUPLICATE_POINT if two points snap to the same rational. */
+int nova_plan_create_f64(int m, int r, const double* finite_points_host, int n_finite, int max_den,
+                         int mode, int coef, nova_plan** out);
+
+/* The exact verifier of Section 2.4 on caller-supplied matrices (row-major AT [m*n], G [n*r],
+ * BT [n*n], n == m + r - 1 <= 64, denominators > 0): NOVA_OK iff
+ * sum_p AT[i][p] G[p][k] BT[p][j] == [j == i + k] for all i, k, j in exact arithmetic,
+ * NOVA_ERR_VERIFY_FAILED otherwise. */
+int nova_verify_decomposition(int m, int r, int n, const nova_rat* AT_host, const nova_rat* G_host,
+                              const nova_rat* BT_host);
+
+/* The exact matrices as reduced fractions (same shapes and order as nova_plan_get_matrices);
+ * NOVA_ERR_RATIONAL_OVERFLOW if an entry does not fit 64-bit numerator and denominator. */
+int nova_plan_get_matrices_rational(const nova_plan* plan, nova_rat* AT_host, nova_rat* G_host, nova_rat* BT_host);
+
+/* kappa_2 and spectral norm of A, G, B in that order (three doubles each; either may be null) -
+ * the per-matrix table of "Transform Matrix Analysis (A, B, G)" and the norm
+ * product of the forward error bound ("Norm Products" paragraph). */
+int nova_plan_kappa_matrices(const nova_plan* plan, double* kappa2_host, double* norm2_host);
+
 /* Copy the fp64 tables, row-major, in the caller's point order:
  * AT [m*n], G [n*r], BT [n*n].  Any pointer may be null. */
 int nova_plan_get_matrices(const nova_plan* plan, double* AT_host, double* G_host, double* BT_host);

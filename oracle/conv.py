@@ -97,10 +97,11 @@ def _two_sided(L, X, axes, dtype):
 # --------------------------------------------------------------------------
 # O3: Winograd in fp64 with the exact matrices
 # --------------------------------------------------------------------------
-def winograd_conv_fp64(x, g, m, points):
+def winograd_conv_fp64(x, g, m, points, scales=(None, None)):
     """Y = A^T [ (G g G^T) (.) (B^T d B) ] A per tile, summed over channels
-    (Section B.5 for the 2-D nesting, Section 2.1 for the four steps)."""
-    AT, G, BT = (tc.to_float(M_) for M_ in tc.build_matrices(m, 3, points))
+    (Section B.5 for the 2-D nesting, Section 2.1 for the four steps).
+    scales = (scale_G, scale_B): optional diagonal rescaling, see toom_cook.build_matrices."""
+    AT, G, BT = (tc.to_float(M_) for M_ in tc.build_matrices(m, 3, points, *scales))
     x = np.asarray(x, dtype=np.float64)
     g = np.asarray(g, dtype=np.float64)
     N, H, W, C = x.shape
@@ -155,14 +156,14 @@ def winograd_conv_exact(x, g, m, points):
 # --------------------------------------------------------------------------
 # O4: rounding emulation of the low-precision pipeline
 # --------------------------------------------------------------------------
-def coefficient_tables(m, points, mode, coef="mode"):
+def coefficient_tables(m, points, mode, coef="mode", scales=(None, None)):
     """Transform matrices as the device evaluates them, returned as float32.
 
     mode "fp16", coef "mode": exact rational -> float64 -> float16 (round to
     nearest even) -> widened (Section 5.1 "cast to FP16"; Section C.3 "matrices
     stored in float16").  coef "fp32" or mode "fp32": rounded to float32 only.
     """
-    mats = tc.build_matrices(m, 3, points)
+    mats = tc.build_matrices(m, 3, points, *scales)
     out = []
     for M_ in mats:
         a = tc.to_float(M_)
@@ -173,9 +174,9 @@ def coefficient_tables(m, points, mode, coef="mode"):
     return out  # AT, G, BT
 
 
-def filter_transform_emulated(g, m, points, mode, coef="mode"):
+def filter_transform_emulated(g, m, points, mode, coef="mode", scales=(None, None)):
     """U[K,n,n,C]: fp32-evaluated G g G^T, rounded once to the operand dtype."""
-    _, G, _ = coefficient_tables(m, points, mode, coef)
+    _, G, _ = coefficient_tables(m, points, mode, coef, scales)
     with np.errstate(all="ignore"):
         U = _two_sided(G, np.asarray(g), (1, 2), np.float32)
         if mode == "fp16":
@@ -183,7 +184,7 @@ def filter_transform_emulated(g, m, points, mode, coef="mode"):
     return U
 
 
-def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False):
+def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False, scales=(None, None)):
     """The four steps with the pipeline's rounding points:
 
     tables rounded as in coefficient_tables; U and V evaluated in float32 and
@@ -193,7 +194,7 @@ def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False)
     the storage dtype.  Mode "fp32" keeps every stage in float32.  Non-finite
     values propagate (Section C.4 "Saturation").
     """
-    AT, G, BT = coefficient_tables(m, points, mode, coef)
+    AT, G, BT = coefficient_tables(m, points, mode, coef, scales)
     x = np.asarray(x)
     N, H, W, C = x.shape
     st = np.float16 if mode == "fp16" else np.float32

@@ -20,6 +20,8 @@ EXPORTED_SYMBOLS = (
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
     "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
+    "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
+    "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices",
 )
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -49,6 +51,20 @@ def lib():
     vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
     L.nova_plan_create.argtypes = [i, i, ctypes.POINTER(_Rat), i, i, i, ctypes.POINTER(vp)]
     L.nova_plan_create.restype = i
+    rp = ctypes.POINTER(_Rat)
+    dp = ctypes.POINTER(ctypes.c_double)
+    L.nova_plan_create_scaled.argtypes = [i, i, rp, i, rp, rp, i, i, ctypes.POINTER(vp)]
+    L.nova_plan_create_scaled.restype = i
+    L.nova_plan_create_f64.argtypes = [i, i, dp, i, i, i, i, ctypes.POINTER(vp)]
+    L.nova_plan_create_f64.restype = i
+    L.nova_snap_to_rational.argtypes = [ctypes.c_double, i, rp]
+    L.nova_snap_to_rational.restype = i
+    L.nova_verify_decomposition.argtypes = [i, i, i, rp, rp, rp]
+    L.nova_verify_decomposition.restype = i
+    L.nova_plan_get_matrices_rational.argtypes = [vp, rp, rp, rp]
+    L.nova_plan_get_matrices_rational.restype = i
+    L.nova_plan_kappa_matrices.argtypes = [vp, dp, dp]
+    L.nova_plan_kappa_matrices.restype = i
     L.nova_plan_destroy.argtypes = [vp]
     L.nova_plan_destroy.restype = None
     dp, fp = ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_float)
@@ -110,6 +126,35 @@ def _torch_dtype(mode):
     return torch.float32 if mode == FP32 else torch.float16
 
 
+def _rat_array(vals):
+    out = []
+    for v in vals:
+        if isinstance(v, tuple):
+            out.append(_Rat(int(v[0]), int(v[1])))
+        else:                                   # int or fractions.Fraction
+            out.append(_Rat(int(v.numerator), int(v.denominator)))
+    return (_Rat * len(out))(*out)
+
+
+def snap_to_rational(x, max_den=10):
+    """Algorithm 2 through the C ABI; returns (num, den)."""
+    r = _Rat()
+    _check(lib().nova_snap_to_rational(float(x), int(max_den), ctypes.byref(r)), "nova_snap_to_rational")
+    return int(r.num), int(r.den)
+
+
+def verify_decomposition(m, r, AT, G, BT):
+    """Exact check of the bilinear identity on matrices of Fractions / (num, den) pairs; True iff it holds."""
+    n = m + r - 1
+    flat = lambda M: _rat_array([v for row in M for v in row])
+    st = lib().nova_verify_decomposition(m, r, n, flat(AT), flat(G), flat(BT))
+    if st == 0:
+        return True
+    if st == -6:
+        return False
+    _check(st, "nova_verify_decomposition")
+
+
 class Plan:
     """nova_plan: transform matrices for F(m x m, 3 x 3) from a point set.
 
@@ -117,12 +162,32 @@ class Plan:
     (the point at infinity).
     """
 
-    def __init__(self, m, points, mode=FP16_F32ACC, coef=COEF_ROUND_TO_MODE, r=3):
-        arr = (_Rat * len(points))(*[_Rat(int(a), int(b)) for a, b in points])
+    def __init__(self, m, points, mode=FP16_F32ACC, coef=COEF_ROUND_TO_MODE, r=3, scale_G=None, scale_B=None):
+        arr = _rat_array(points)
         h = ctypes.c_void_p()
-        _check(lib().nova_plan_create(m, r, arr, len(points), mode, coef, ctypes.byref(h)), "nova_plan_create")
+        if scale_G is None and scale_B is None:
+            _check(lib().nova_plan_create(m, r, arr, len(points), mode, coef, ctypes.byref(h)), "nova_plan_create")
+        else:
+            sg = _rat_array(scale_G) if scale_G is not None else None
+            sb = _rat_array(scale_B) if scale_B is not None else None
+            if any(a is not None and len(a) != len(points) for a in (sg, sb)):
+                raise ValueError("one scale per point")
+            _check(lib().nova_plan_create_scaled(m, r, arr, len(points), sg, sb, mode, coef, ctypes.byref(h)),
+                   "nova_plan_create_scaled")
         self._h = h
         self.m, self.r, self.n, self.mode, self.coef = m, r, m + r - 1, mode, coef
+
+    @classmethod
+    def from_floats(cls, m, finite_points, max_den=10, mode=FP16_F32ACC, coef=COEF_ROUND_TO_MODE, r=3):
+        """Snap continuous points to simple rationals (Algorithm 2), append infinity, build the plan."""
+        arr = (ctypes.c_double * len(finite_points))(*[float(v) for v in finite_points])
+        h = ctypes.c_void_p()
+        _check(lib().nova_plan_create_f64(m, r, arr, len(finite_points), max_den, mode, coef, ctypes.byref(h)),
+               "nova_plan_create_f64")
+        self = cls.__new__(cls)
+        self._h = h
+        self.m, self.r, self.n, self.mode, self.coef = m, r, m + r - 1, mode, coef
+        return self
 
     def close(self):
         if getattr(self, "_h", None):
@@ -143,6 +208,21 @@ class Plan:
         _check(lib().nova_plan_get_matrices(self._h, AT.ctypes.data_as(dp), G.ctypes.data_as(dp),
                                             BT.ctypes.data_as(dp)), "nova_plan_get_matrices")
         return AT, G, BT
+
+    def matrices_rational(self):
+        """Exact A^T, G, B^T as nested lists of fractions.Fraction."""
+        from fractions import Fraction
+        AT = (_Rat * (self.m * self.n))(); G = (_Rat * (self.n * self.r))(); BT = (_Rat * (self.n * self.n))()
+        _check(lib().nova_plan_get_matrices_rational(self._h, AT, G, BT), "nova_plan_get_matrices_rational")
+        shape = lambda a, rows, cols: [[Fraction(a[i * cols + j].num, a[i * cols + j].den) for j in range(cols)]
+                                       for i in range(rows)]
+        return shape(AT, self.m, self.n), shape(G, self.n, self.r), shape(BT, self.n, self.n)
+
+    def kappa_matrices(self):
+        """(kappa_2, spectral norm) of A, G, B: two 3-tuples."""
+        k = (ctypes.c_double * 3)(); nrm = (ctypes.c_double * 3)()
+        _check(lib().nova_plan_kappa_matrices(self._h, k, nrm), "nova_plan_kappa_matrices")
+        return tuple(k), tuple(nrm)
 
     def device_tables(self):
         import numpy as np

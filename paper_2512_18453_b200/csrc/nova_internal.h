@@ -29,6 +29,9 @@ struct nova_plan {
   double G[nova::kMaxN * nova::kR];       // n x r
   double BT[nova::kMaxN * nova::kMaxN];   // n x n
   double kappa2_V;
+  double kappa2_mat[3], norm2_mat[3];     // kappa_2 and spectral norm of A, G, B (as scaled)
+  nova_rat AT_rat[nova::kMaxM * nova::kMaxN], G_rat[nova::kMaxN * nova::kR], BT_rat[nova::kMaxN * nova::kMaxN];
+  int rat_fits;                           // every exact entry fits a 64-bit numerator / denominator
   nova::Coefs coefs;                      // rounded to the coefficient precision, caller's point order
   // The kernels index frequencies in an internal point order: perm[i] is the
   // caller's index of internal point i.  For a symmetric set {0, +-a_1, ..,

@@ -177,14 +177,16 @@ float round_through_half(double v) {
 }
 
 // ---------------------------------------------------------------- kappa_2
-// One-sided Jacobi SVD of a small square matrix; returns sigma_max/sigma_min.
-double cond2(std::vector<double> a, int n) {
+// One-sided Jacobi SVD of a small rows x n matrix (rows >= n, row-major, leading dimension n);
+// returns sigma_max/sigma_min and, if asked, sigma_max.
+double cond2(std::vector<double> a, int n, int rows = -1, double* sigma_max = nullptr) {
+  if (rows < 0) rows = n;
   for (int sweep = 0; sweep < 60; ++sweep) {
     double off = 0;
     for (int p = 0; p < n - 1; ++p)
       for (int q = p + 1; q < n; ++q) {
         double al = 0, be = 0, ga = 0;
-        for (int i = 0; i < n; ++i) {
+        for (int i = 0; i < rows; ++i) {
           al += a[i * n + p] * a[i * n + p];
           be += a[i * n + q] * a[i * n + q];
           ga += a[i * n + p] * a[i * n + q];
@@ -194,7 +196,7 @@ double cond2(std::vector<double> a, int n) {
         double zeta = (be - al) / (2 * ga);
         double t = (zeta >= 0 ? 1.0 : -1.0) / (std::fabs(zeta) + std::sqrt(1 + zeta * zeta));
         double c = 1 / std::sqrt(1 + t * t), s = c * t;
-        for (int i = 0; i < n; ++i) {
+        for (int i = 0; i < rows; ++i) {
           double x = a[i * n + p], y = a[i * n + q];
           a[i * n + p] = c * x - s * y;
           a[i * n + q] = s * x + c * y;
@@ -205,18 +207,50 @@ double cond2(std::vector<double> a, int n) {
   double smax = 0, smin = INFINITY;
   for (int j = 0; j < n; ++j) {
     double s = 0;
-    for (int i = 0; i < n; ++i) s += a[i * n + j] * a[i * n + j];
+    for (int i = 0; i < rows; ++i) s += a[i * n + j] * a[i * n + j];
     s = std::sqrt(s);
     smax = std::max(smax, s);
     smin = std::min(smin, s);
   }
+  if (sigma_max) *sigma_max = smax;
   return smax / smin;
 }
 
-}  // namespace
+// Exact check of the bilinear identity sum_p A^T[i][p] G[p][k] B^T[p][j] == [j == i + k]
+// (Section 2.4), over arbitrary-precision integers.
+bool identity_holds(int m, int r, int n, const std::vector<Rat>& AT, const std::vector<Rat>& G,
+                    const std::vector<Rat>& BT) {
+  for (int i = 0; i < m; ++i)
+    for (int k = 0; k < r; ++k)
+      for (int j = 0; j < n; ++j) {
+        Big num, den = big_from(1);
+        for (int p = 0; p < n; ++p) {
+          const Rat &a = AT[i * n + p], &g = G[p * r + k], &b = BT[p * n + j];
+          if (a.n == 0 || g.n == 0 || b.n == 0) continue;
+          Big tn = big_mul(big_mul(big_from(a.n), big_from(g.n)), big_from(b.n));
+          Big td = big_mul(big_mul(big_from(a.d), big_from(g.d)), big_from(b.d));
+          num = big_add(big_mul(num, td), big_mul(tn, den));
+          den = big_mul(den, td);
+        }
+        if (j == i + k) { Big md = den; md.neg = !md.neg; num = big_add(num, md); }
+        if (!num.zero()) return false;
+      }
+  return true;
+}
 
-extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int mode, int coef,
-                                nova_plan** out) {
+bool fits64(const Rat& v, nova_rat* out) {
+  const i128 lim = (i128)1 << 63;
+  if (v.n >= lim || v.n < -lim || v.d >= lim) return false;
+  out->num = (int64_t)v.n;
+  out->den = (int64_t)v.d;
+  return true;
+}
+
+int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* scale_G, const nova_rat* scale_B,
+                int mode, int coef, nova_plan** out);
+
+int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* scale_G, const nova_rat* scale_B,
+                int mode, int coef, nova_plan** out) {
   if (out) *out = nullptr;
   if (!points || !out) return NOVA_ERR_INVALID_ARG;
   if (m != 2 && m != 4 && m != 6 && m != 8) return NOVA_ERR_INVALID_ARG;
@@ -274,24 +308,21 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
     }
     for (size_t t = 0; t < poly.size(); ++t) BT[p * n + t] = poly[t];
   }
+  // Diagonal rescaling: rows of G by D_G, rows of B^T by D_B, columns of A^T by (D_G D_B)^-1.
+  if (scale_G || scale_B) {
+    for (int p = 0; p < n; ++p) {
+      Rat sg = one, sb = one;
+      if (scale_G) { if (scale_G[p].den <= 0 || scale_G[p].num == 0) return NOVA_ERR_INVALID_ARG; sg = ar.norm(scale_G[p].num, scale_G[p].den); }
+      if (scale_B) { if (scale_B[p].den <= 0 || scale_B[p].num == 0) return NOVA_ERR_INVALID_ARG; sb = ar.norm(scale_B[p].num, scale_B[p].den); }
+      const Rat both = ar.mul(sg, sb);
+      for (int k = 0; k < r; ++k) G[p * r + k] = ar.mul(G[p * r + k], sg);
+      for (int j = 0; j < n; ++j) BT[p * n + j] = ar.mul(BT[p * n + j], sb);
+      for (int i = 0; i < m; ++i) AT[i * n + p] = ar.div(AT[i * n + p], both);
+    }
+  }
   if (ar.bad) return NOVA_ERR_RATIONAL_OVERFLOW;
 
-  // Exact check: sum_p A^T[i][p] G[p][k] B^T[p][j] == [j == i + k]  (Section 2.4)
-  for (int i = 0; i < m; ++i)
-    for (int k = 0; k < r; ++k)
-      for (int j = 0; j < n; ++j) {
-        Big num, den = big_from(1);
-        for (int p = 0; p < n; ++p) {
-          const Rat &a = AT[i * n + p], &g = G[p * r + k], &b = BT[p * n + j];
-          if (a.n == 0 || g.n == 0 || b.n == 0) continue;
-          Big tn = big_mul(big_mul(big_from(a.n), big_from(g.n)), big_from(b.n));
-          Big td = big_mul(big_mul(big_from(a.d), big_from(g.d)), big_from(b.d));
-          num = big_add(big_mul(num, td), big_mul(tn, den));
-          den = big_mul(den, td);
-        }
-        if (j == i + k) { Big md = den; md.neg = !md.neg; num = big_add(num, md); }
-        if (!num.zero()) return NOVA_ERR_VERIFY_FAILED;
-      }
+  if (!identity_holds(m, r, n, AT, G, BT)) return NOVA_ERR_VERIFY_FAILED;
 
   nova_plan* pl = new (std::nothrow) nova_plan();
   if (!pl) return NOVA_ERR_INVALID_ARG;
@@ -301,6 +332,20 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
   for (int i = 0; i < m * n; ++i) pl->AT[i] = rat_to_double(AT[i]);
   for (int i = 0; i < n * r; ++i) pl->G[i] = rat_to_double(G[i]);
   for (int i = 0; i < n * n; ++i) pl->BT[i] = rat_to_double(BT[i]);
+  pl->rat_fits = 1;
+  for (int i = 0; i < m * n; ++i) if (!fits64(AT[i], &pl->AT_rat[i])) pl->rat_fits = 0;
+  for (int i = 0; i < n * r; ++i) if (!fits64(G[i], &pl->G_rat[i])) pl->rat_fits = 0;
+  for (int i = 0; i < n * n; ++i) if (!fits64(BT[i], &pl->BT_rat[i])) pl->rat_fits = 0;
+  {
+    std::vector<double> A(n * m), Gd(pl->G, pl->G + n * r), Bd(n * n);
+    for (int i = 0; i < m; ++i)
+      for (int p = 0; p < n; ++p) A[p * m + i] = pl->AT[i * n + p];          // A = (A^T)^T, n x m
+    for (int p = 0; p < n; ++p)
+      for (int j = 0; j < n; ++j) Bd[j * n + p] = pl->BT[p * n + j];
+    pl->kappa2_mat[0] = cond2(A, m, n, &pl->norm2_mat[0]);
+    pl->kappa2_mat[1] = cond2(Gd, r, n, &pl->norm2_mat[1]);
+    pl->kappa2_mat[2] = cond2(Bd, n, n, &pl->norm2_mat[2]);
+  }
 
   const bool through_half = (mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE);
   auto rnd = [&](double v) { return through_half ? round_through_half(v) : (float)v; };
@@ -411,6 +456,94 @@ extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int
   }
   (void)cudaGetLastError();
   *out = pl;
+  return NOVA_OK;
+}
+
+}  // namespace
+
+extern "C" int nova_plan_create(int m, int r, const nova_rat* points, int n, int mode, int coef,
+                                nova_plan** out) {
+  return create_impl(m, r, points, n, nullptr, nullptr, mode, coef, out);
+}
+
+extern "C" int nova_plan_create_scaled(int m, int r, const nova_rat* points, int n, const nova_rat* scale_G,
+                                       const nova_rat* scale_B, int mode, int coef, nova_plan** out) {
+  return create_impl(m, r, points, n, scale_G, scale_B, mode, coef, out);
+}
+
+extern "C" int nova_snap_to_rational(double x, int max_den, nova_rat* out) {
+  if (!out || max_den < 1 || max_den > 4096 || !std::isfinite(x)) return NOVA_ERR_INVALID_ARG;
+  // Candidates lie in [-5, 5], so clamping x to [-6, 6] changes no answer; and an |x| below
+  // 2^-30 is closer to 0 than to the smallest non-zero candidate (>= 2^-12) with no tie possible.
+  if (x > 6) x = 6;
+  if (x < -6) x = -6;
+  if (std::fabs(x) < std::ldexp(1.0, -30)) { out->num = 0; out->den = 1; return NOVA_OK; }
+  // x = X / 2^s exactly, |X| < 2^53, s <= 83.  |x - a/b| = |X b - a 2^s| / (b 2^s); two
+  // candidates compare by cross-multiplication, which stays below 2^111.
+  int e;
+  const double fr = std::frexp(x, &e);
+  i128 X = (i128)(long long)std::ldexp(fr, 53);
+  int s = 53 - e;
+  while (s < 0) { X *= 2; ++s; }
+  long long best_a = 0, best_b = 1;
+  i128 best_num = -1;
+  for (long long b = 1; b <= max_den; ++b)          // Algorithm 2's scan order; strict "<" keeps the first of a tie
+    for (long long a = -5 * b; a <= 5 * b; ++a) {
+      i128 num = X * b - ((i128)a << s);
+      if (num < 0) num = -num;
+      if (best_num < 0 || num * best_b < best_num * b) { best_num = num; best_a = a; best_b = b; }
+    }
+  const long long g = (long long)gcd128(best_a, best_b);
+  out->num = best_a / (g ? g : 1);
+  out->den = best_b / (g ? g : 1);
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_create_f64(int m, int r, const double* finite_points, int n_finite, int max_den,
+                                    int mode, int coef, nova_plan** out) {
+  if (out) *out = nullptr;
+  if (!finite_points || !out || n_finite < 1 || n_finite >= nova::kMaxN) return NOVA_ERR_INVALID_ARG;
+  nova_rat pts[nova::kMaxN];
+  for (int i = 0; i < n_finite; ++i) {
+    const int st = nova_snap_to_rational(finite_points[i], max_den, &pts[i]);
+    if (st != NOVA_OK) return st;
+  }
+  pts[n_finite].num = 1;
+  pts[n_finite].den = 0;
+  return create_impl(m, r, pts, n_finite + 1, nullptr, nullptr, mode, coef, out);
+}
+
+extern "C" int nova_verify_decomposition(int m, int r, int n, const nova_rat* AT, const nova_rat* G,
+                                         const nova_rat* BT) {
+  if (!AT || !G || !BT || m < 1 || r < 1 || n != m + r - 1 || n > 64) return NOVA_ERR_INVALID_ARG;
+  Arith ar;
+  std::vector<Rat> a(m * n), g(n * r), b(n * n);
+  auto conv = [&](const nova_rat* src, std::vector<Rat>& dst) {
+    for (size_t i = 0; i < dst.size(); ++i) {
+      if (src[i].den <= 0) return false;
+      dst[i] = ar.norm(src[i].num, src[i].den);
+    }
+    return true;
+  };
+  if (!conv(AT, a) || !conv(G, g) || !conv(BT, b)) return NOVA_ERR_INVALID_ARG;
+  return identity_holds(m, r, n, a, g, b) ? NOVA_OK : NOVA_ERR_VERIFY_FAILED;
+}
+
+extern "C" int nova_plan_get_matrices_rational(const nova_plan* p, nova_rat* AT, nova_rat* G, nova_rat* BT) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  if (!p->rat_fits) return NOVA_ERR_RATIONAL_OVERFLOW;
+  if (AT) std::memcpy(AT, p->AT_rat, sizeof(nova_rat) * p->m * p->n);
+  if (G) std::memcpy(G, p->G_rat, sizeof(nova_rat) * p->n * p->r);
+  if (BT) std::memcpy(BT, p->BT_rat, sizeof(nova_rat) * p->n * p->n);
+  return NOVA_OK;
+}
+
+extern "C" int nova_plan_kappa_matrices(const nova_plan* p, double* kappa2, double* norm2) {
+  if (!p) return NOVA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) {
+    if (kappa2) kappa2[i] = p->kappa2_mat[i];
+    if (norm2) norm2[i] = p->norm2_mat[i];
+  }
   return NOVA_OK;
 }
 

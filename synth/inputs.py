@@ -29,7 +29,7 @@ class ConvCase:
 
 CONFIGS = {
     "cfg1": ConvCase("cfg1", 2, 1, 16, 16, 8, 8, "fp32", False, False, 1001, ("std",)),
-    "cfg2": ConvCase("cfg2", 4, 8, 56, 56, 64, 64, "fp16", True, True, 1002, ("std", "nova")),
+    "cfg2": ConvCase("cfg2", 4, 8, 56, 56, 64, 64, "fp16", True, True, 1002, ("std", "nova", "dyadic")),
     "cfg3": ConvCase("cfg3", 6, 32, 56, 56, 256, 256, "fp16", True, True, 1003, ("half", "nova", "std")),
     "cfg4": ConvCase("cfg4", 8, 32, 28, 28, 512, 512, "fp16", True, True, 1004, ("std", "nova")),
 }

@@ -41,3 +41,19 @@ POINT_SETS = {
 def point_set(kind, m):
     """Return a fresh list of (num, den) pairs; the last entry is infinity."""
     return list(POINT_SETS[(kind, m)])
+
+
+def pow2_range_scales(G, BT):
+    """Power-of-two row scales (scale_G, scale_B), as (num, den) pairs, that bring the largest
+    magnitude of every row of G and of B^T into [1, 2).  G, BT: nested lists / arrays of numbers
+    (the unscaled matrices).  Powers of two change no rounding of the transforms, only the range
+    of the transformed filter and input - the hardware-friendly form of the per-tap scales in the
+    appendix on complementary techniques.  The same scale serves both points of a +- pair because
+    their rows differ by signs only."""
+    import math
+
+    def scale(row):
+        mx = max(abs(float(v)) for v in row)
+        e = math.floor(math.log2(mx))
+        return (1, 2 ** e) if e >= 0 else (2 ** (-e), 1)
+    return [scale(r) for r in G], [scale(r) for r in BT]

@@ -27,8 +27,8 @@ def _need_cuda():
         pytest.fail("the GPU tests need a CUDA device; there is no CPU fallback")
 
 
-def gpu_conv(x, g, m, pts, mode, flags=0, ws="default", coef=nv.COEF_ROUND_TO_MODE):
-    plan = nv.Plan(m, pts, mode, coef)
+def gpu_conv(x, g, m, pts, mode, flags=0, ws="default", coef=nv.COEF_ROUND_TO_MODE, scales=(None, None)):
+    plan = nv.Plan(m, pts, mode, coef, scale_G=scales[0], scale_B=scales[1])
     xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
     U = plan.filter_transform(gd)
     N, H, W, C = x.shape
@@ -42,9 +42,9 @@ def gpu_conv(x, g, m, pts, mode, flags=0, ws="default", coef=nv.COEF_ROUND_TO_MO
     return y.cpu().numpy(), U.cpu().numpy(), plan
 
 
-def check_fp16(y, x, g, m, pts, coef="mode"):
+def check_fp16(y, x, g, m, pts, coef="mode", scales=(None, None)):
     y1 = conv.direct_conv_fp64(x, g)
-    ye = conv.winograd_conv_emulated(x, g, m, pts, "fp16", coef)
+    ye = conv.winograd_conv_emulated(x, g, m, pts, "fp16", coef, scales=scales)
     e_gpu, e_emu = conv.rel_l2(y, y1), conv.rel_l2(ye, y1)
     if not np.isfinite(e_emu) or e_emu >= 1.0:
         assert (not np.isfinite(e_gpu)) or e_gpu >= 0.5, (e_gpu, e_emu)
@@ -395,3 +395,64 @@ def test_cfg5_vgg16_stack_f8_nova_two_images():
         assert (not np.isfinite(e_gpu)) or e_gpu >= 0.5
     else:
         assert e_gpu <= 2.0 * e_emu
+
+
+# ---------------------------------------------------------------- diagonal rescaling (D_A D_G D_B = I)
+def _pow2_scales(m, pts):
+    from oracle import toom_cook as tc
+    from synth import pow2_range_scales
+    _, G, BT = tc.build_matrices(m, 3, pts)
+    return pow2_range_scales(G, BT)
+
+
+@pytest.mark.parametrize("kind,m", [("std", 4), ("dyadic", 4), ("nova", 6), ("half", 6), ("nova", 8), ("std", 8)])
+@pytest.mark.parametrize("shape", [(2, 19, 23, 64, 72), (1, 30, 30, 128, 256)])
+def test_rescaled_plans_match_the_rescaled_emulation(kind, m, shape):
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", seed=300 + m)
+    pts = point_set(kind, m)
+    sc = _pow2_scales(m, pts)
+    y, _, plan = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, scales=sc)
+    e_gpu, e_emu = check_fp16(y, x, g, m, pts, scales=sc)
+    # the range-normalised integer F(8,3) set no longer overflows binary16 (Section C.4)
+    if (kind, m) == ("std", 8):
+        assert np.isfinite(y.astype(np.float32)).all()
+    y32, _, _ = gpu_conv(x.astype(np.float32), g.astype(np.float32), m, pts, nv.FP32, scales=sc)
+    y1 = conv.direct_conv_fp64(x, g)
+    e32 = conv.rel_l2(y32, y1)
+    e32_emu = conv.rel_l2(conv.winograd_conv_emulated(x.astype(np.float32), g.astype(np.float32), m, pts, "fp32",
+                                                      scales=sc), y1)
+    # fp32 mode: the stated absolute bounds, and no worse than 3x the emulation (whose sums over the
+    # channels run in another order)
+    assert e32 <= {4: 1e-5, 6: 1e-4, 8: 1e-1 if kind == "std" else 5e-4}[m], e32
+    assert e32 <= 3.0 * e32_emu + 1e-7, (e32, e32_emu)
+
+
+def test_power_of_two_rescaling_changes_no_bit_on_the_device():
+    # in range, a power of two commutes with every rounding, with the hi/lo split of the
+    # tensor-core input transform and with the fp32 accumulation: the output is bit-identical
+    x, g = make_conv_inputs(2, 24, 24, 64, 64, "fp16", seed=77, he_weights=False)
+    pts = point_set("nova", 4)
+    a, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC)
+    sg, sb = _pow2_scales(4, pts)
+    for p in (0, len(pts) - 1):                      # unit columns of A^T at 0 and infinity keep the
+        sb[p] = (sg[p][1], sg[p][0])                 # even/odd transforms, i.e. the same summation order
+    b, _, plan = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC, scales=(sg, sb))
+    assert plan.frequency_order()[1] is True
+    # bit-identical wherever no entry of U or V was subnormal in either run (binary16 subnormals do
+    # not scale); such entries are rare and tiny, so the few outputs they touch move by one ulp
+    ia, ib = a.view(np.int16).astype(np.int32), b.view(np.int16).astype(np.int32)
+    differ = ia != ib
+    assert differ.mean() < 2e-3, differ.mean()
+    assert np.abs(ia - ib).max() <= 1
+
+
+def test_unpaired_scales_take_the_dense_transforms_and_stay_correct():
+    from fractions import Fraction
+    x, g = make_conv_inputs(1, 26, 18, 64, 64, "fp16", seed=78)
+    pts = point_set("nova", 6)
+    sg = [Fraction(1), Fraction(2), Fraction(3), Fraction(1, 2), Fraction(1, 4), Fraction(5, 4), Fraction(1), Fraction(3, 2)]
+    sb = [Fraction(2), Fraction(1), Fraction(1, 3), Fraction(2), Fraction(4), Fraction(1), Fraction(7, 8), Fraction(1)]
+    y, _, plan = gpu_conv(x, g, 6, pts, nv.FP16_F32ACC, scales=(sg, sb))
+    assert plan.frequency_order()[1] is False
+    check_fp16(y, x, g, 6, pts, scales=(sg, sb))

@@ -99,3 +99,75 @@ def test_size_queries_and_argument_checks_without_a_device():
     assert L.nova_filter_transform(plan._h, None, 8, 8, None, None) == -1
     assert L.nova_maxpool2x2(None, None, 1, 8, 8, 8, 1, None) == -1
     assert nv.status_string(-9) == "a bounded device-side wait expired"
+
+
+# ---------------------------------------------------------------- discovery helpers and rescaling
+def test_snap_through_the_abi_equals_the_oracle():
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    xs = list(rng.uniform(-6, 6, size=300)) + [0.0, 0.25, 0.75, -0.75, 5.0, -5.0, 7.3, -100.0, 1e-12, 5 / 6, 7 / 6]
+    for d_max in (1, 2, 6, 10, 20):
+        for x in xs:
+            want = tc.snap_to_rational(float(x), d_max)
+            assert nv.snap_to_rational(x, d_max) == (want.numerator, want.denominator), (x, d_max)
+    for bad in (0, 5000):
+        with pytest.raises(nv.NovaError):
+            nv.snap_to_rational(0.5, bad)
+    with pytest.raises(nv.NovaError):
+        nv.snap_to_rational(float("nan"), 10)
+
+
+def test_plan_from_floats_recovers_the_discovered_sets():
+    # continuous optima near the printed fractions snap onto them (Section "Snap-to-Rational")
+    plan = nv.Plan.from_floats(4, [0.0004, 0.8329, -0.8338, 1.1671, -1.1660])
+    want = nv.Plan(4, point_set("nova", 4))
+    for a, b in zip(plan.matrices(), want.matrices()):
+        assert np.array_equal(a, b)
+    assert abs(plan.kappa() - 14.5) < 0.05
+    with pytest.raises(nv.NovaError) as e:           # two points snapping to the same rational
+        nv.Plan.from_floats(4, [0.0, 0.83, 0.834, 1.0, -1.0])
+    assert e.value.status == -4
+
+
+@pytest.mark.parametrize("kind,m", sorted(POINT_SETS))
+def test_exact_matrices_and_per_matrix_conditioning_match_the_oracle(kind, m):
+    pts = point_set(kind, m)
+    plan = nv.Plan(m, pts)
+    oAT, oG, oBT = tc.build_matrices(m, 3, pts)
+    AT, G, BT = plan.matrices_rational()
+    assert AT == oAT and G == oG and BT == oBT                    # exact, entry by entry
+    kap, nrm = plan.kappa_matrices()
+    for got, M in zip(kap, (oAT, oG, oBT)):
+        assert abs(got / tc.kappa2(tc.to_float(M)) - 1) < 1e-9
+    for got, M in zip(nrm, (oAT, oG, oBT)):
+        assert abs(got / tc.norm2(tc.to_float(M)) - 1) < 1e-12
+
+
+def test_verifier_accepts_valid_and_rejects_planted_mistakes():
+    from fractions import Fraction
+    AT, G, BT = tc.build_matrices(6, 3, point_set("nova", 6))
+    assert nv.verify_decomposition(6, 3, AT, G, BT)
+    bad = [row[:] for row in G]; bad[3][1] = -bad[3][1]
+    assert not nv.verify_decomposition(6, 3, AT, bad, BT)
+    bad = [row[:] for row in BT]; bad[2][4] += Fraction(1, 10 ** 9)
+    assert not nv.verify_decomposition(6, 3, AT, G, bad)
+    BTt = [[BT[j][i] for j in range(8)] for i in range(8)]         # transposed operand
+    assert not nv.verify_decomposition(6, 3, AT, G, BTt)
+
+
+def test_scaled_plan_matches_the_oracle_and_keeps_symmetry_only_for_paired_scales():
+    # the even/odd fast path needs equal scales within a +- pair and unit columns of A^T at 0 and infinity
+    from fractions import Fraction
+    pts = point_set("nova", 6)
+    sg = [Fraction(1, 4), Fraction(2), Fraction(2), Fraction(1, 4), Fraction(1, 4), Fraction(3), Fraction(3), Fraction(1, 2)]
+    sb = [Fraction(4), Fraction(1, 2), Fraction(1, 2), Fraction(8), Fraction(8), Fraction(1), Fraction(1), Fraction(2)]
+    plan = nv.Plan(6, pts, scale_G=sg, scale_B=sb)
+    assert plan.matrices_rational() == tc.build_matrices(6, 3, pts, scale_G=sg, scale_B=sb)
+    assert plan.frequency_order()[1] is True
+    assert plan.kappa() == nv.Plan(6, pts).kappa()                 # rescaling does not touch kappa(V)
+    sg[2] = Fraction(5)                                            # different scales within a +- pair
+    plan = nv.Plan(6, pts, scale_G=sg, scale_B=sb)
+    assert plan.matrices_rational() == tc.build_matrices(6, 3, pts, scale_G=sg, scale_B=sb)
+    assert plan.frequency_order()[1] is False
+    with pytest.raises(nv.NovaError):
+        nv.Plan(6, pts, scale_G=[0] * 8)

@@ -154,3 +154,43 @@ def test_filter_transform_matches_pipeline_stage():
     U0 = conv.filter_transform_emulated(g0, 4, point_set("nova", 4), "fp16")
     want = (G[:, 1][:, None] * G[:, 1][None, :]).astype(np.float16)
     assert np.array_equal(U0[0, :, :, 0], want)
+
+
+# ---------------------------------------------------------------- diagonal rescaling
+def _pow2_scales(m, kind):
+    from oracle import toom_cook as tc
+    from synth import pow2_range_scales
+    _, G, BT = tc.build_matrices(m, 3, point_set(kind, m))
+    return pow2_range_scales(G, BT)
+
+
+@pytest.mark.parametrize("kind,m", [("std", 4), ("nova", 6), ("std", 8)])
+def test_rescaled_winograd_fp64_still_equals_direct(kind, m):
+    x, g = make_conv_inputs(1, 11, 9, 4, 3, dtype="fp32", seed=5)
+    y1 = conv.direct_conv_fp64(x, g)
+    y3 = conv.winograd_conv_fp64(x, g, m, point_set(kind, m), scales=_pow2_scales(m, kind))
+    assert conv.rel_l2(y3, y1) < (1e-12 if kind == "nova" or m < 8 else 1e-8)
+
+
+def test_power_of_two_rescaling_changes_no_bit_while_in_range():
+    # a power of two commutes with every rounding of the pipeline as long as nothing leaves the
+    # normal range, so the emulated output is bit-identical with and without it
+    x, g = make_conv_inputs(2, 12, 12, 8, 8, dtype="fp16", seed=9)
+    pts = point_set("nova", 4)
+    a = conv.winograd_conv_emulated(x, g, 4, pts, "fp16")
+    b = conv.winograd_conv_emulated(x, g, 4, pts, "fp16", scales=_pow2_scales(4, "nova"))
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+
+
+def test_range_scaling_rescues_the_integer_points_of_the_largest_tile():
+    # Section C.4 "Saturation": F(8,3) on integer points leaves the binary16 range.  Row scales that
+    # are powers of two remove the overflow (finite output) without touching the conditioning,
+    # so the error stays far above that of the well-conditioned set.
+    x, g = make_conv_inputs(1, 16, 16, 64, 8, dtype="fp16", seed=13)
+    y1 = conv.direct_conv_fp64(x, g)
+    plain = conv.winograd_conv_emulated(x, g, 8, point_set("std", 8), "fp16")
+    scaled = conv.winograd_conv_emulated(x, g, 8, point_set("std", 8), "fp16", scales=_pow2_scales(8, "std"))
+    nova = conv.winograd_conv_emulated(x, g, 8, point_set("nova", 8), "fp16")
+    assert not np.isfinite(plain.astype(np.float64)).all()
+    assert np.isfinite(scaled.astype(np.float64)).all()
+    assert conv.rel_l2(nova, y1) < conv.rel_l2(scaled, y1)
