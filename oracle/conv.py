@@ -218,6 +218,78 @@ def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False,
 
 
 # --------------------------------------------------------------------------
+# INT8 Winograd-domain pipeline (Section 5.1 "INT8 Setup"; Appendix "INT8 Convolution Error
+# Validation"; Section "Rational Coefficients in Practice")
+# --------------------------------------------------------------------------
+def quantize_int8(v, scale):
+    """Symmetric quantiser: round(v / scale) to nearest, ties to even, saturated to [-128, 127].
+    The division is one float32 operation (the decision is taken in float32).  scale may be an
+    array broadcastable against v; a zero scale (an all-zero tensor) is treated as 1."""
+    v = np.asarray(v, dtype=np.float32)
+    s = np.asarray(scale, dtype=np.float32)
+    s = np.where(s == 0, np.float32(1), s)
+    q = np.rint(v / s)                                  # float32 / float32 -> float32; rint = ties to even
+    return np.clip(q, -128, 127).astype(np.int8)
+
+
+def int8_scale(absmax):
+    """s = max|.| / 127 in float32 (Section 5.1: "s = max(|w|)/127")."""
+    return (np.asarray(absmax, dtype=np.float32) / np.float32(127)).astype(np.float32)
+
+
+def winograd_conv_int8_emulated(x, g, m, points, per_channel=False, scale_U=None, scale_V=None,
+                                coef="fp32", apply_relu=False, scales=(None, None), return_parts=False):
+    """The four steps with the Winograd-domain tensors quantised to int8.
+
+    The transform matrices stay in floating point (float32 tables by default, as the paper's
+    note on rational coefficients states; coef="mode" rounds them through float16 like the
+    half pipeline).  U = G g G^T and V = B^T d B are evaluated in float32 and quantised
+    symmetrically: U with one scale per tensor, or one per output channel k when per_channel
+    (s = max|.|/127 over the tensor / the channel's slice); V with one scale for the whole batch.
+    scale_U (array of K) / scale_V (number) override the data-derived scales ("static" scales).
+    The product over input channels is exact integer arithmetic (int32 on the device); it is
+    converted to float32, multiplied by the float32 product s_U[k] * s_V, and the output
+    transform is evaluated in float32 and rounded once to float16.
+    """
+    AT, G, BT = coefficient_tables(m, points, "fp16", coef, scales)
+    x = np.asarray(x)
+    N, H, W, C = x.shape
+    with np.errstate(all="ignore"):
+        U = _two_sided(G, np.asarray(g), (1, 2), np.float32)                  # [K,n,n,C]
+        K = U.shape[0]
+        if scale_U is None:
+            amax = np.abs(U).max(axis=(1, 2, 3)) if per_channel else np.full(K, np.abs(U).max(), np.float32)
+            sU = int8_scale(amax)
+        else:
+            sU = np.broadcast_to(np.asarray(scale_U, dtype=np.float32), (K,)).copy()
+        sU = np.where(sU == 0, np.float32(1), sU).astype(np.float32)
+        Uq = quantize_int8(U, sU[:, None, None, None])
+        d = _gather_tiles(x.astype(np.float32), m)
+        V = _two_sided(BT, d, (3, 4), np.float32)                              # [N,Th,Tw,n,n,C]
+        sV = int8_scale(np.abs(V).max()) if scale_V is None else np.float32(scale_V)
+        if sV == 0:
+            sV = np.float32(1)
+        Vq = quantize_int8(V, sV)
+        n = m + 2
+        Th, Tw = d.shape[1], d.shape[2]
+        Mi = np.empty((N, Th, Tw, n, n, K), dtype=np.int64)
+        for p in range(n):
+            for q in range(n):
+                # exact: |sum| <= C * 128 * 128 < 2^53
+                Mi[:, :, :, p, q, :] = np.rint(Vq[:, :, :, p, q, :].astype(np.float64) @ Uq[:, p, q, :].astype(np.float64).T)
+        s = (sU * sV).astype(np.float32)                                        # one float32 product per filter
+        Mf = Mi.astype(np.float32) * s                                          # int -> float32 (RNE), then one multiply
+        Y = _two_sided(AT, Mf, (3, 4), np.float32)
+        y = _scatter_tiles(Y, H, W)
+        if apply_relu:
+            y = np.where(y < 0, np.float32(0), y)
+        y = y.astype(np.float16)
+    if return_parts:
+        return y, {"Uq": Uq, "scale_U": sU, "Vq": Vq, "scale_V": sV, "M": Mi}
+    return y
+
+
+# --------------------------------------------------------------------------
 # VGG-16 convolution stack
 # --------------------------------------------------------------------------
 def vgg_stack_fp64(x, weights, layers):
