@@ -60,6 +60,13 @@ enum {
                                    without TMA staging (testing) */
 };
 
+/* How nova_filter_transform_int8 obtains the scales of the transformed filter. */
+enum {
+  NOVA_QUANT_PER_TENSOR = 0,   /* one scale, max|U| / 127 over the whole tensor (written to all K entries) */
+  NOVA_QUANT_PER_CHANNEL = 1,  /* one scale per output channel k, max over that channel's slice / 127 */
+  NOVA_QUANT_GIVEN = 2         /* scale_U_dev already holds K scales chosen by the caller */
+};
+
 enum {
   NOVA_OK = 0,
   NOVA_ERR_INVALID_ARG = -1,        /* null / misaligned pointer, bad shape, m not in {2,4,6,8}, n != m+r-1 */
@@ -257,6 +264,46 @@ int nova_conv2d_fwd_static(const nova_plan* plan, const void* x_dev, const void*
  * and workspace size (negative = error). */
 int nova_conv2d_launch_count(const nova_plan* plan, int N, int H, int W, int C, int K,
                              size_t workspace_bytes, int flags);
+
+/*
+ * INT8 Winograd-domain pipeline (Section 5.1 "INT8 Setup"; appendix "INT8 Convolution Error
+ * Validation"; Section "Snap-to-Rational", paragraph "Rational Coefficients in Practice").  The
+ * transform matrices stay in floating point (create the plan with NOVA_FP16_F32ACC and, as the
+ * paper does, NOVA_COEF_FP32); the transformed filter U and the transformed input V are
+ * quantised symmetrically to signed 8 bit - code = round-to-nearest-even(value / s) saturated to
+ * [-128, 127], s = max|value| / 127, one float division each - the product over the input
+ * channels is exact int32 arithmetic on the tensor cores (tcgen05 kind::i8), and the output
+ * transform runs in float on float(M) * (s_U[k] * s_V), rounded once to half.  x, g and y are
+ * half tensors as in nova_conv2d_fwd.  C and K must be multiples of 16.
+ *
+ * nova_filter_transform_int8: g [K,3,3,C] half -> Uq (nova_filter_transform_int8_bytes() bytes,
+ * opaque layout) and scale_U_dev[K] floats (device).  quant: one of NOVA_QUANT_*.
+ */
+size_t nova_filter_transform_int8_bytes(const nova_plan* plan, int K, int C);
+int nova_filter_transform_int8(const nova_plan* plan, const void* g_dev, int K, int C, int quant,
+                               void* Uq_dev, float* scale_U_dev, nova_stream stream);
+
+/*
+ * nova_conv2d_fwd_int8: scale_V > 0 is a static (calibrated) scale for the transformed input;
+ * scale_V == 0 derives it from the data, max|V| / 127 over the whole batch, which costs a second
+ * pass of the input transform.  The workspace (nova_conv2d_int8_workspace_bytes(), 256-byte
+ * aligned) holds Vq, the int32 product and the scale; the whole batch is processed in one piece
+ * (NOVA_ERR_WORKSPACE if it does not fit).  flags: NOVA_RELU; NOVA_GEMM_SIMT selects an exact
+ * CUDA-core product (cross-check).  The scale used is left in the first float of the workspace.
+ * Asynchronous on `stream`; allocates nothing.
+ */
+size_t nova_conv2d_int8_workspace_bytes(const nova_plan* plan, int N, int H, int W, int C, int K);
+int nova_conv2d_fwd_int8(const nova_plan* plan, const void* x_dev, const void* Uq_dev,
+                         const float* scale_U_dev, float scale_V, void* y_dev,
+                         int N, int H, int W, int C, int K,
+                         void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream);
+/* The same with one CUDA event pair per kernel; ms_host[4] receives the input transform (all its
+ * passes), the product, the output transform and the total, in milliseconds.  Synchronises. */
+int nova_conv2d_fwd_int8_timed(const nova_plan* plan, const void* x_dev, const void* Uq_dev,
+                               const float* scale_U_dev, float scale_V, void* y_dev,
+                               int N, int H, int W, int C, int K,
+                               void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream,
+                               float* ms_host);
 
 /* 2x2 max pooling, stride 2, NHWC, H and W even, C % 8 == 0 (used between the
  * blocks of a VGG-style stack; not part of the paper's method).  `mode`

@@ -22,7 +22,10 @@ EXPORTED_SYMBOLS = (
     "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
     "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
     "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices",
+    "nova_filter_transform_int8_bytes", "nova_filter_transform_int8", "nova_conv2d_int8_workspace_bytes",
+    "nova_conv2d_fwd_int8", "nova_conv2d_fwd_int8_timed",
 )
+QUANT_PER_TENSOR, QUANT_PER_CHANNEL, QUANT_GIVEN = 0, 1, 2
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -95,6 +98,17 @@ def lib():
     L.nova_conv2d_fwd_host.restype = i
     L.nova_conv2d_fwd_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
     L.nova_conv2d_fwd_static.restype = i
+    cf = ctypes.c_float
+    L.nova_filter_transform_int8_bytes.argtypes = [vp, i, i]
+    L.nova_filter_transform_int8_bytes.restype = sz
+    L.nova_filter_transform_int8.argtypes = [vp, vp, i, i, i, vp, vp, vp]
+    L.nova_filter_transform_int8.restype = i
+    L.nova_conv2d_int8_workspace_bytes.argtypes = [vp, i, i, i, i, i]
+    L.nova_conv2d_int8_workspace_bytes.restype = sz
+    L.nova_conv2d_fwd_int8.argtypes = [vp, vp, vp, vp, cf, vp, i, i, i, i, i, vp, sz, i, vp]
+    L.nova_conv2d_fwd_int8.restype = i
+    L.nova_conv2d_fwd_int8_timed.argtypes = [vp, vp, vp, vp, cf, vp, i, i, i, i, i, vp, sz, i, vp, fp]
+    L.nova_conv2d_fwd_int8_timed.restype = i
     L.nova_conv2d_launch_count.argtypes = [vp, i, i, i, i, i, sz, i]
     L.nova_conv2d_launch_count.restype = i
     L.nova_maxpool2x2.argtypes = [vp, vp, i, i, i, i, i, vp]
@@ -317,6 +331,45 @@ class Plan:
                                           workspace.data_ptr(), workspace.numel(), flags, _stream()),
                "nova_conv2d_fwd_host")
         return y_host
+
+    # ---- INT8 Winograd-domain pipeline
+    def filter_transform_int8(self, g, quant=QUANT_PER_TENSOR, scale_U=None):
+        """g [K,3,3,C] half -> (Uq int8 [n*n, K, C], scale_U float32 [K])."""
+        import torch
+        K, _, _, C = g.shape
+        assert g.is_cuda and g.is_contiguous() and g.dtype == torch.float16
+        Uq = torch.empty(lib().nova_filter_transform_int8_bytes(self._h, K, C), dtype=torch.int8, device=g.device)
+        if quant == QUANT_GIVEN:
+            sc = scale_U.to(device=g.device, dtype=torch.float32).contiguous()
+            assert sc.numel() == K
+        else:
+            sc = torch.empty(K, dtype=torch.float32, device=g.device)
+        _check(lib().nova_filter_transform_int8(self._h, g.data_ptr(), K, C, quant, Uq.data_ptr(), sc.data_ptr(),
+                                                _stream()), "nova_filter_transform_int8")
+        return Uq.view(self.n * self.n, K, C), sc
+
+    def int8_workspace_bytes(self, N, H, W, C, K):
+        return lib().nova_conv2d_int8_workspace_bytes(self._h, N, H, W, C, K)
+
+    def conv2d_int8(self, x, Uq, scale_U, scale_V=0.0, y=None, workspace=None, flags=0, timed=False):
+        """x [N,H,W,C] half -> y [N,H,W,K] half.  scale_V = 0 derives the input scale from the data.
+        timed=True returns (y, [input ms, product ms, output ms, total ms])."""
+        import torch
+        N, H, W, C = x.shape
+        K = Uq.shape[1]
+        assert x.is_cuda and x.is_contiguous() and x.dtype == torch.float16 and Uq.dtype == torch.int8
+        if y is None:
+            y = torch.empty((N, H, W, K), dtype=torch.float16, device=x.device)
+        if workspace is None:
+            workspace = torch.empty(self.int8_workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device=x.device)
+        args = (self._h, x.data_ptr(), Uq.data_ptr(), scale_U.data_ptr(), float(scale_V), y.data_ptr(),
+                N, H, W, C, K, workspace.data_ptr(), workspace.numel(), flags, _stream())
+        if timed:
+            ms = (ctypes.c_float * 4)()
+            _check(lib().nova_conv2d_fwd_int8_timed(*args, ms), "nova_conv2d_fwd_int8_timed")
+            return y, list(ms)
+        _check(lib().nova_conv2d_fwd_int8(*args), "nova_conv2d_fwd_int8")
+        return y
 
     def device_status(self):
         return lib().nova_last_device_status(self._h, _stream())

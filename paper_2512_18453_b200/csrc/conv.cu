@@ -294,6 +294,111 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
   return conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, NOVA_STATIC_SCRATCH_BYTES, flags, stream, nullptr);
 }
 
+// ---------------------------------------------------------------------------
+// INT8 Winograd-domain pipeline.
+namespace {
+bool int8_shape_ok(const nova_plan* p, int N, int H, int W, int C, int K) {
+  return p && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
+}
+struct Int8Layout {
+  int pad;                  // tiles rounded up to whole 128-row blocks
+  size_t v_off, m_off, total;
+};
+Int8Layout int8_layout(const Geom& g) {
+  Int8Layout l;
+  l.pad = (int)round_up_ll(g.P, 128);
+  l.v_off = kAlign;                                   // the first block holds the scale of V
+  l.m_off = l.v_off + round_up((size_t)g.n * g.n * l.pad * g.C, kAlign);
+  l.total = l.m_off + round_up((size_t)g.n * g.n * l.pad * g.K * 4, kAlign);
+  return l;
+}
+
+int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const float* scale_U, float scale_V,
+                     void* y, int N, int H, int W, int C, int K, void* ws, size_t ws_bytes, int flags,
+                     nova_stream stream, cudaEvent_t* ev) {
+  if (!int8_shape_ok(p, N, H, W, C, K) || !aligned16(x) || !aligned16(Uq) || !aligned16(y) || !scale_U ||
+      !(scale_V >= 0.f))
+    return p && p->mode != NOVA_FP16_F32ACC ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
+  if (!p->status_dev) return NOVA_ERR_CUDA;
+  const Geom g = make_geom(p, N, H, W, C, K);
+  if (g.P >= (1ll << 24)) return NOVA_ERR_UNSUPPORTED;
+  const Int8Layout l = int8_layout(g);
+  if (ws_bytes < l.total) return NOVA_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  float* slot = reinterpret_cast<float*>(base);
+  void* Vq = base + l.v_off;
+  int32_t* Mb = reinterpret_cast<int32_t*>(base + l.m_off);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int pc = (int)g.P, nfreq = g.n * g.n;
+  int e = 0;
+  if (ev) cudaEventRecord(ev[0], s);
+  if (scale_V > 0.f) {
+    e = launch_scale_slot(slot, scale_V, 0, stream);
+  } else {                                            // s_V = max|V| / 127 over the batch: one more pass
+    if (cudaMemsetAsync(slot, 0, sizeof(float), s) != cudaSuccess) return NOVA_ERR_CUDA;
+    e = launch_input_transform_int8(p, g, x, Vq, slot, 0, 0, pc, l.pad, stream);
+    if (!e) e = launch_scale_slot(slot, 0.f, 1, stream);
+  }
+  if (!e) e = launch_input_transform_int8(p, g, x, Vq, slot, 1, 0, pc, l.pad, stream);
+  if (ev) cudaEventRecord(ev[1], s);
+  if (!e)
+    e = (flags & NOVA_GEMM_SIMT) ? launch_gemm_simt_i8(Vq, Uq, Mb, nfreq, pc, l.pad, C, K, stream)
+                                 : launch_gemm_tcgen05_i8(p, Vq, Uq, Mb, nfreq, pc, l.pad, C, K, p->status_dev, stream);
+  if (ev) cudaEventRecord(ev[2], s);
+  if (!e)
+    e = launch_output_transform_tma(p, g, Mb, y, 0, pc, l.pad, (flags & NOVA_RELU) ? 1 : 0, stream, scale_U, slot);
+  if (ev) cudaEventRecord(ev[3], s);
+  if (e) g_last_cuda_error = e;
+  return e ? NOVA_ERR_CUDA : NOVA_OK;
+}
+}  // namespace
+
+extern "C" size_t nova_filter_transform_int8_bytes(const nova_plan* p, int K, int C) {
+  if (!p || K <= 0 || C <= 0) return 0;
+  return (size_t)p->n * p->n * K * C;
+}
+
+extern "C" int nova_filter_transform_int8(const nova_plan* p, const void* g, int K, int C, int quant, void* Uq,
+                                          float* scale_U, nova_stream stream) {
+  if (!p || !aligned16(g) || !aligned16(Uq) || !scale_U || K <= 0 || C <= 0 || (K % 16) || (C % 16))
+    return NOVA_ERR_INVALID_ARG;
+  if (quant != NOVA_QUANT_PER_TENSOR && quant != NOVA_QUANT_PER_CHANNEL && quant != NOVA_QUANT_GIVEN)
+    return NOVA_ERR_INVALID_ARG;
+  if (p->mode != NOVA_FP16_F32ACC) return NOVA_ERR_UNSUPPORTED;
+  const int e = launch_filter_transform_int8(p, g, K, C, Uq, scale_U, quant, stream);
+  if (e) g_last_cuda_error = e;
+  return e ? NOVA_ERR_CUDA : NOVA_OK;
+}
+
+extern "C" size_t nova_conv2d_int8_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
+  if (!int8_shape_ok(p, N, H, W, C, K)) return 0;
+  return int8_layout(make_geom(p, N, H, W, C, K)).total;
+}
+
+extern "C" int nova_conv2d_fwd_int8(const nova_plan* p, const void* x, const void* Uq, const float* scale_U,
+                                    float scale_V, void* y, int N, int H, int W, int C, int K, void* ws,
+                                    size_t ws_bytes, int flags, nova_stream stream) {
+  return conv2d_int8_impl(p, x, Uq, scale_U, scale_V, y, N, H, W, C, K, ws, ws_bytes, flags, stream, nullptr);
+}
+
+extern "C" int nova_conv2d_fwd_int8_timed(const nova_plan* p, const void* x, const void* Uq, const float* scale_U,
+                                          float scale_V, void* y, int N, int H, int W, int C, int K, void* ws,
+                                          size_t ws_bytes, int flags, nova_stream stream, float* ms) {
+  if (!ms) return NOVA_ERR_INVALID_ARG;
+  cudaEvent_t ev[4];
+  for (auto& e : ev) cudaEventCreate(&e);
+  int st = conv2d_int8_impl(p, x, Uq, scale_U, scale_V, y, N, H, W, C, K, ws, ws_bytes, flags, stream, ev);
+  if (st == NOVA_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st = NOVA_ERR_CUDA;
+  ms[0] = ms[1] = ms[2] = ms[3] = 0.f;
+  if (st == NOVA_OK) {
+    for (int k = 0; k < 3; ++k) cudaEventElapsedTime(&ms[k], ev[k], ev[k + 1]);
+    cudaEventElapsedTime(&ms[3], ev[0], ev[3]);
+  }
+  for (auto& e : ev) cudaEventDestroy(e);
+  return st;
+}
+
 extern "C" int nova_last_cuda_error(void) { return g_last_cuda_error; }
 
 extern "C" int nova_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode,

@@ -68,7 +68,36 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
   }
 }
 
+// The int8 product on CUDA cores (cross-check of the kind::i8 tensor-core kernel): one thread per
+// (tile, filter quad), four dp4a-free integer dot products over the channels.  Exact.
+__global__ void __launch_bounds__(256)
+gemm_simt_i8_kernel(const int8_t* __restrict__ V, const int8_t* __restrict__ U, int32_t* __restrict__ Mo,
+                    int pc, int pc_pad, int C, int K) {
+  const int f = blockIdx.z;
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  const int k = blockIdx.y * 4;
+  if (p >= pc || k >= K) return;
+  const int8_t* v = V + ((size_t)f * pc_pad + p) * C;
+  const int8_t* u = U + ((size_t)f * K + k) * C;
+  int acc[4] = {0, 0, 0, 0};
+  for (int c = 0; c < C; ++c) {
+    const int a = v[c];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] += a * (int)u[(size_t)j * C + c];
+  }
+  *reinterpret_cast<int4*>(Mo + (((size_t)f * (K >> 2) + (k >> 2)) * pc_pad + p) * 4) =
+      make_int4(acc[0], acc[1], acc[2], acc[3]);
+}
+
 }  // namespace
+
+int launch_gemm_simt_i8(const void* V, const void* U, int32_t* M, int nfreq, int pc, int pc_pad, int C, int K,
+                        void* stream) {
+  dim3 grid((pc + 255) / 256, K / 4, nfreq);
+  gemm_simt_i8_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const int8_t*)V, (const int8_t*)U, M, pc, pc_pad,
+                                                              C, K);
+  return (int)cudaGetLastError();
+}
 
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M, int nfreq, int pc,
                      int pc_pad, int C, int K, void* stream) {

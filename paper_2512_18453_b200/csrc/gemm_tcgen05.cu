@@ -1,6 +1,7 @@
 // Transformed-domain product on the sm_100a tensor cores (Section 2.1 step 3
 // summed over input channels): for every frequency f,
-//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c],   half x half -> float.
+//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c],   half x half -> float,
+// or, for the int8 pipeline (I8), signed 8-bit x signed 8-bit -> int32 (exact).
 //
 // Persistent, warp-specialised kernel.  One CTA per SM walks a list of work
 // items (f, 128-row block of tiles p, BLOCK_N-wide block of filters k):
@@ -28,26 +29,27 @@ namespace {
 using namespace sm100;
 
 constexpr int BLOCK_M = 128;
-constexpr int BLOCK_K = 64;            // 64 halves = 128 bytes = one swizzle row
-constexpr int UMMA_K = 16;
+constexpr int kRowBytes = 128;         // one swizzle row of K per stage: 64 halves or 128 int8
+constexpr int kUmmaBytes = 32;         // K bytes one tcgen05.mma contracts (16 halves / 32 int8)
 constexpr int kStages = 4;
 constexpr int kThreads = 320;          // producer, MMA issuer, 2 x 4 epilogue warps
 
 template <int BLOCK_N>
 struct SmemLayout {
-  static constexpr int kABytes = BLOCK_M * BLOCK_K * 2;
-  static constexpr int kBBytes = BLOCK_N * BLOCK_K * 2;
+  static constexpr int kABytes = BLOCK_M * kRowBytes;
+  static constexpr int kBBytes = BLOCK_N * kRowBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarrierOffset = kStages * kStageBytes;
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;     // barriers + alignment slack
 };
 
-template <int BLOCK_N>
+template <int BLOCK_N, bool I8>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
                     float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
                     int* __restrict__ status) {
   using L = SmemLayout<BLOCK_N>;
+  constexpr int BLOCK_K = I8 ? kRowBytes : kRowBytes / 2;   // elements of K per stage
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -118,7 +120,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
-    constexpr uint32_t idesc = umma_idesc_f16(BLOCK_M, BLOCK_N);
+    constexpr uint32_t idesc = I8 ? umma_idesc_i8(BLOCK_M, BLOCK_N) : umma_idesc_f16(BLOCK_M, BLOCK_N);
     uint32_t stage = 0, phase = 0;
     for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
@@ -131,11 +133,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         if (lane == 0) {
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
-const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
-          umma_f16(tmem_d, ad0, bd0, idesc, ks > 0 ? 1u : 0u);
+          const uint64_t ad0 = umma_desc_sw128(sa), bd0 = umma_desc_sw128(sb);
+          if constexpr (I8) {
+            umma_i8(tmem_d, ad0, bd0, idesc, ks > 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 1; k < BLOCK_K / 16; ++k)
-            umma_f16_c<true>(tmem_d, umma_desc_advance(ad0, k * 32), umma_desc_advance(bd0, k * 32), idesc);
+            for (int k = 1; k < kRowBytes / kUmmaBytes; ++k)
+              umma_i8(tmem_d, umma_desc_advance(ad0, k * kUmmaBytes), umma_desc_advance(bd0, k * kUmmaBytes), idesc, 1u);
+          } else {
+            umma_f16(tmem_d, ad0, bd0, idesc, ks > 0 ? 1u : 0u);
+#pragma unroll
+            for (int k = 1; k < kRowBytes / kUmmaBytes; ++k)
+              umma_f16_c<true>(tmem_d, umma_desc_advance(ad0, k * kUmmaBytes), umma_desc_advance(bd0, k * kUmmaBytes), idesc);
+          }
           umma_commit(&empty_bar[stage]);                 // frees the smem stage when the MMAs retire
           if (ks == num_ks - 1) umma_commit(&tmem_full[acc]);
         }
@@ -226,25 +235,27 @@ bool make_map_3d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BLOCK_N>
+template <int BLOCK_N, bool I8>
 int launch_n(int sms, const void* V, const void* U, float* M, int nfreq, int pc, int pc_pad, int C, int K,
              int* status, cudaStream_t stream) {
   using L = SmemLayout<BLOCK_N>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BLOCK_N>,
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BLOCK_N, I8>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
   CUtensorMap tmV, tmU;
-  const CUtensorMapDataType f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-  if (!make_map_3d(&tmV, f16, 2, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
-      !make_map_3d(&tmU, f16, 2, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N))
+  const CUtensorMapDataType dt = I8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+  constexpr int esize = I8 ? 1 : 2;
+  constexpr int BLOCK_K = kRowBytes / esize;
+  if (!make_map_3d(&tmV, dt, esize, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
+      !make_map_3d(&tmU, dt, esize, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N))
     return (int)cudaErrorUnknown;
   const long long items = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M) * ((K + BLOCK_N - 1) / BLOCK_N);
   const int grid = (int)(items < sms ? items : sms);
-  gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K, status);
+  gemm_tcgen05_kernel<BLOCK_N, I8><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K, status);
   return (int)cudaGetLastError();
 }
 
@@ -254,9 +265,21 @@ int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, flo
                         int pc_pad, int C, int K, int* status_dev, void* stream) {
   cudaStream_t s = (cudaStream_t)stream;
   const int sms = plan->sm_count;
-  if (K > 128) return launch_n<256>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
-  if (K > 64) return launch_n<128>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
-  return launch_n<64>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  if (K > 128) return launch_n<256, false>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  if (K > 64) return launch_n<128, false>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  return launch_n<64, false>(sms, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+}
+
+// The int8 product: V [nfreq][pc_pad][C] and U [nfreq][K][C] signed bytes (C a multiple of 16),
+// M as int32 in the same [f][K/4][pc_pad][4] layout.
+int launch_gemm_tcgen05_i8(const nova_plan* plan, const void* V, const void* U, int32_t* M, int nfreq, int pc,
+                           int pc_pad, int C, int K, int* status_dev, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  const int sms = plan->sm_count;
+  float* Mf = reinterpret_cast<float*>(M);            // the epilogue moves 32-bit words
+  if (K > 128) return launch_n<256, true>(sms, V, U, Mf, nfreq, pc, pc_pad, C, K, status_dev, s);
+  if (K > 64) return launch_n<128, true>(sms, V, U, Mf, nfreq, pc, pc_pad, C, K, status_dev, s);
+  return launch_n<64, true>(sms, V, U, Mf, nfreq, pc, pc_pad, C, K, status_dev, s);
 }
 
 }  // namespace nova

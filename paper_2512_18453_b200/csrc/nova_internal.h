@@ -79,8 +79,19 @@ size_t kron_table_halves(int m);
 void build_kron_table(const nova_plan* plan, unsigned short* out);
 int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y,
                             long long p0, int pc, int pc_pad, int relu, void* stream);
+// scale_U / scale_V non-null: M holds int32 sums of the int8 pipeline, dequantised on load
 int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void* M, void* y,
-                                long long p0, int pc, int pc_pad, int relu, void* stream);
+                                long long p0, int pc, int pc_pad, int relu, void* stream,
+                                const float* scale_U = nullptr, const float* scale_V = nullptr);
+int launch_filter_transform_int8(const nova_plan* plan, const void* g, int K, int C, void* Uq, float* scales,
+                                 int quant, void* stream);
+int launch_input_transform_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot,
+                                int pass, long long p0, int pc, int pc_pad, void* stream);
+int launch_scale_slot(float* slot, float value, int from_absmax, void* stream);
+int launch_gemm_tcgen05_i8(const nova_plan* plan, const void* V, const void* U, int32_t* M, int nfreq, int pc,
+                           int pc_pad, int C, int K, int* status_dev, void* stream);
+int launch_gemm_simt_i8(const void* V, const void* U, int32_t* M, int nfreq, int pc, int pc_pad, int C, int K,
+                        void* stream);
 int launch_fused_conv(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* ws,
                       int R, int relu, void* stream);
 int launch_fused_product_output(const nova_plan* plan, const Geom& g, const void* x, const void* V, const void* U,

@@ -18,12 +18,22 @@ __device__ __forceinline__ float2 vmax_lo(float2 v, float lo) {
   return make_float2(v.x < lo ? lo : v.x, v.y < lo ? lo : v.y);
 }
 
-template <int M, bool SYM, int VEC = 1>
+// int32 accumulator bits -> float (round to nearest even), times the dequantisation scale
+// (__fmul_rn: the product is rounded on its own, never contracted into a following add)
+__device__ __forceinline__ float dequant(float bits, float s) { return __fmul_rn(__int2float_rn(__float_as_int(bits)), s); }
+__device__ __forceinline__ float2 dequant(float2 bits, float2 s) {
+  return make_float2(__fmul_rn(__int2float_rn(__float_as_int(bits.x)), s.x), __fmul_rn(__int2float_rn(__float_as_int(bits.y)), s.y));
+}
+
+// QUANT: the stage holds the int32 sums of the int8 pipeline; every value is converted to float
+// and multiplied by qscale (this thread's filters' s_U[k] * s_V) as it is loaded.
+template <int M, bool SYM, int VEC = 1, bool QUANT = false>
 struct OutputTile {
   static constexpr int N = M + 2;
   using V = typename VecOf<VEC>::type;
   const Coefs& cf;
   uint32_t sb_even, sb_odd;      // VEC = 2 uses sb_even only
+  V qscale;
 
   template <int XI, int NU>
   __device__ __forceinline__ void fill(V (&in)[N]) const {
@@ -33,6 +43,7 @@ struct OutputTile {
         in[NU] = (F & 1) ? sm100::lds_f32<F * 512>(sb_odd) : sm100::lds_f32<F * 512>(sb_even);
       else
         in[NU] = sm100::lds_f32x2<F * 1024>(sb_even);
+      if constexpr (QUANT) in[NU] = dequant(in[NU], qscale);
       fill<XI, NU + 1>(in);
     }
   }

@@ -43,11 +43,13 @@ struct OtCfg {
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;
 };
 
-template <int M, typename T, bool SYM, int VEC>
+// QUANT: M holds the int32 sums of the int8 pipeline; scale_U[k] * *scale_V dequantises filter k.
+template <int M, typename T, bool SYM, int VEC, bool QUANT>
 __global__ void __launch_bounds__(kOtThreads, 1)
 output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
                             T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
-                            int pc_pad, int relu, int* __restrict__ status) {
+                            int pc_pad, int relu, int* __restrict__ status, const float* __restrict__ scale_U,
+                            const float* __restrict__ scale_V) {
   using Cfg = OtCfg<M, VEC>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kUnitK = 16 * VEC;                    // filters per unit
@@ -107,12 +109,18 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
       const uint32_t sb = smem_u32(smem) + stage * Cfg::kStageBytes;
       const uint32_t sb_even = sb + off_even, sb_odd = sb + off_odd;
       typename VecOf<VEC>::type Y[M][M];
-      OutputTile<M, SYM, VEC>{cf, sb_even, sb_odd}.run(Y);
+      const int k = kg * kUnitK + (lane & 15) * VEC;
+      typename VecOf<VEC>::type qs = {};
+      if constexpr (QUANT) {
+        const float sv = *scale_V;
+        if constexpr (VEC == 1) qs = __fmul_rn(k < K ? scale_U[k] : 0.f, sv);
+        else qs = make_float2(__fmul_rn(k < K ? scale_U[k] : 0.f, sv), __fmul_rn(k + 1 < K ? scale_U[k + 1] : 0.f, sv));
+      }
+      OutputTile<M, SYM, VEC, QUANT>{cf, sb_even, sb_odd, qs}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
 
       const int pl = tg * 8 + t;
-      const int k = kg * kUnitK + (lane & 15) * VEC;
       if (pl < pc && k < K) {
         const unsigned p = (unsigned)(p0 + pl);
         const unsigned tw = p % (unsigned)Tw, q2 = p / (unsigned)Tw;
@@ -149,27 +157,27 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int M, typename T, bool SYM, int VEC>
+template <int M, typename T, bool SYM, int VEC, bool QUANT>
 int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
-               int pc_pad, int relu, cudaStream_t stream) {
+               int pc_pad, int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
   using Cfg = OtCfg<M, VEC>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC>,
+    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC, QUANT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
   const long long units = (long long)(pc_pad / 8) * ((g.K + 16 * VEC - 1) / (16 * VEC));
   const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
-  output_transform_tma_kernel<M, T, SYM, VEC><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
-      tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev);
+  output_transform_tma_kernel<M, T, SYM, VEC, QUANT><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
+      tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev, scale_U, scale_V);
   return (int)cudaGetLastError();
 }
 
 template <int M>
 int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0, int pc, int pc_pad,
-             int relu, cudaStream_t stream) {
+             int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return (int)cudaErrorUnknown;
   CUtensorMap tmM;
@@ -184,23 +192,27 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return (int)cudaErrorUnknown;
   const bool f32 = plan->mode == NOVA_FP32;
-  if (plan->symmetric)
-    return f32 ? launch_one<M, float, true, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
-               : launch_one<M, __half, true, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
-  return f32 ? launch_one<M, float, false, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream)
-             : launch_one<M, __half, false, VEC>(plan, g, tmM, y, p0, pc, pc_pad, relu, stream);
+#define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
+  if (scale_U) {                                      // int8 pipeline (half storage only)
+    if (f32) return (int)cudaErrorInvalidValue;
+    return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
+  }
+  if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
+  return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
+#undef NOVA_OT
 }
 
 }  // namespace
 
 int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0,
-                                int pc, int pc_pad, int relu, void* stream) {
+                                int pc, int pc_pad, int relu, void* stream, const float* scale_U,
+                                const float* scale_V) {
   cudaStream_t s = (cudaStream_t)stream;
   switch (plan->m) {
-    case 2: return launch_m<2>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
-    case 4: return launch_m<4>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
-    case 6: return launch_m<6>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
-    case 8: return launch_m<8>(plan, g, Mb, y, p0, pc, pc_pad, relu, s);
+    case 2: return launch_m<2>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+    case 4: return launch_m<4>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+    case 6: return launch_m<6>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+    case 8: return launch_m<8>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
   }
   return (int)cudaErrorInvalidValue;
 }

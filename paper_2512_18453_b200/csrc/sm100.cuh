@@ -213,6 +213,20 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t 
   d |= (uint64_t)2 << 61;
   return d;
 }
+// Instruction descriptor, kind::i8: D int32 (format 2), A and B signed 8-bit (format 1), both
+// K-major; one instruction contracts 32 bytes of K.
+__host__ __device__ constexpr uint32_t umma_idesc_i8(int M, int N) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // Instruction descriptor, kind::f16, D float, A half MN-major, B half K-major.
 __host__ __device__ constexpr uint32_t umma_idesc_f16_amn(int M, int N) {
   return umma_idesc_f16(M, N) | (1u << 15);

@@ -13,11 +13,74 @@ namespace {
 
 using namespace xf;
 
+// Where the float results of a transform go.  StoreSink rounds them to the operand type;
+// AbsmaxSink only reduces them to their largest magnitude (first pass of a data-derived int8
+// scale s = max|.| / 127); QuantSink divides by a scale read from device memory, rounds to
+// nearest even and saturates to [-128, 127] (the symmetric quantiser of the INT8 set-up,
+// Section 5.1).  Offsets are in elements of the destination.
+template <typename T>
+struct StoreSink {
+  T* out;
+  __device__ __forceinline__ void begin(int) {}
+  __device__ __forceinline__ void put(size_t off, float2 v) { st2(out + off, v); }
+  __device__ __forceinline__ void finish() {}
+};
+struct AbsmaxSink {
+  unsigned* slots;     // non-negative floats order like their bit patterns
+  int per_channel;
+  float mx;
+  unsigned* slot;
+  __device__ __forceinline__ void begin(int channel) { mx = 0.f; slot = slots + (per_channel ? channel : 0); }
+  __device__ __forceinline__ void put(size_t, float2 v) { mx = fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y))); }
+  __device__ __forceinline__ void finish() {
+    if (per_channel) {
+      atomicMax(slot, __float_as_uint(mx));
+    } else {
+      const unsigned act = __activemask();
+      const unsigned m = __reduce_max_sync(act, __float_as_uint(mx));
+      if ((threadIdx.x & 31) == (unsigned)(__ffs(act) - 1)) atomicMax(slot, m);
+    }
+  }
+};
+__device__ __forceinline__ int quant_code(float v, float s) {
+  const int q = __float2int_rn(__fdiv_rn(v, s));       // one float division, ties to even
+  return max(-128, min(127, q));
+}
+struct QuantSink {
+  int8_t* out;
+  const float* scales;
+  int per_channel;
+  float s;
+  __device__ __forceinline__ void begin(int channel) {
+    s = scales[per_channel ? channel : 0];
+    if (s == 0.f) s = 1.f;
+  }
+  __device__ __forceinline__ void put(size_t off, float2 v) {
+    char2 q;
+    q.x = (signed char)quant_code(v.x, s);
+    q.y = (signed char)quant_code(v.y, s);
+    *reinterpret_cast<char2*>(out + off) = q;
+  }
+  __device__ __forceinline__ void finish() {}
+};
+
+// absmax slots -> scales, in place: s = max / 127 (float division); per tensor, slot 0 is
+// copied to all `count` entries.  One block.
+__global__ void scales_from_absmax_kernel(float* slots, int count, int per_channel) {
+  const float m0 = slots[0];
+  __syncthreads();
+  for (int i = threadIdx.x; i < count; i += blockDim.x) {
+    const float m = per_channel ? slots[i] : m0;
+    slots[i] = __fdiv_rn(m, 127.f);
+  }
+}
+__global__ void set_scale_kernel(float* slot, float value) { *slot = value; }
+
 // ---------------------------------------------------------------- U = G g G^T
 // One thread per (filter k, channel pair).  g [K,3,3,C] -> U [n*n][K][C].
-template <int M, typename T>
+template <int M, typename T, typename Sink>
 __global__ void __launch_bounds__(256)
-filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ g, T* __restrict__ U,
+filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ g, Sink sink,
                         int K, int C) {
   constexpr int N = M + 2;
   const int c2 = C >> 1;
@@ -25,6 +88,7 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
   if (idx >= (long long)K * c2) return;
   const int k = (int)(idx / c2);
   const int c = (int)(idx % c2) * 2;
+  sink.begin(k);
   float2 gg[3][3];
 #pragma unroll
   for (int a = 0; a < 3; ++a)
@@ -47,8 +111,9 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
       float2 s = mul2(cf.G[q][0], t[p][0]);
       s = fma2(cf.G[q][1], t[p][1], s);
       s = fma2(cf.G[q][2], t[p][2], s);
-      st2(U + ((size_t)(p * N + q) * K + k) * C + c, s);
+      sink.put(((size_t)(p * N + q) * K + k) * C + c, s);
     }
+  sink.finish();
 }
 
 // ---------------------------------------------------------------- V = B^T d B
@@ -57,9 +122,9 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
 // patch's columns (nu), keeps the n x 2 intermediate in registers, applies all n rows along
 // the patch's rows (xi) and stores the 2n frequencies (xi, nu in its group).  The n/2 groups
 // of a patch sit in one block, so the patch is read from DRAM once and from L1 afterwards.
-template <int M, typename T, bool SYM, int G>
+template <int M, typename T, bool SYM, int G, typename Sink>
 __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* __restrict__ x,
-                                                      T* __restrict__ V, int H, int W, int C, int h0,
+                                                      Sink& V, int H, int W, int C, int h0,
                                                       int w0, long long img, size_t out_off,
                                                       size_t f_stride) {
   constexpr int N = M + 2;
@@ -96,14 +161,14 @@ __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* 
   bt_all_rows<N, SYM>(cf, tb, ob);
 #pragma unroll
   for (int xi = 0; xi < N; ++xi) {
-    st2(V + out_off + (size_t)(xi * N + RA) * f_stride, oa[xi]);
-    st2(V + out_off + (size_t)(xi * N + RB) * f_stride, ob[xi]);
+    V.put(out_off + (size_t)(xi * N + RA) * f_stride, oa[xi]);
+    V.put(out_off + (size_t)(xi * N + RB) * f_stride, ob[xi]);
   }
 }
 
-template <int M, typename T, bool SYM>
+template <int M, typename T, bool SYM, typename Sink>
 __global__ void __launch_bounds__(32 * (M + 2) * 2)
-input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, T* __restrict__ V,
+input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, Sink V,
                        int H, int W, int C, int Th, int Tw, long long p0, int pc, int pc_pad) {
   constexpr int N = M + 2;
   constexpr int WORK = 128;                       // (tile, channel pair) items per block
@@ -122,6 +187,7 @@ input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x
   const size_t out_off = (size_t)pl * C + c;
   const size_t f_stride = (size_t)pc_pad * C;
   const T* xc = x + c;
+  V.begin(0);
   switch (g) {
     case 0: input_transform_group<M, T, SYM, 0>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
     case 1: input_transform_group<M, T, SYM, 1>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
@@ -129,6 +195,7 @@ input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x
     case 3: if constexpr (N >= 8) input_transform_group<M, T, SYM, 3>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
     case 4: if constexpr (N >= 10) input_transform_group<M, T, SYM, 4>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
   }
+  V.finish();
 }
 
 // ---------------------------------------------------------------- Y = A^T M A
@@ -270,7 +337,46 @@ inline unsigned blocks_for(long long work, int threads) {
 template <int M, typename T>
 int filter_launch(const nova_plan* plan, const void* g, int K, int C, void* U, cudaStream_t s) {
   const long long work = (long long)K * (C / 2);
-  filter_transform_kernel<M, T><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, (T*)U, K, C);
+  filter_transform_kernel<M, T, StoreSink<T>><<<blocks_for(work, 256), 256, 0, s>>>(
+      plan->kcoefs, (const T*)g, StoreSink<T>{(T*)U}, K, C);
+  return (int)cudaGetLastError();
+}
+// int8 filter transform: absmax pass (unless the scales are given), scales, quantising pass.
+template <int M, typename T>
+int filter_launch_int8(const nova_plan* plan, const void* g, int K, int C, void* Uq, float* scales, int quant,
+                       cudaStream_t s) {
+  const long long work = (long long)K * (C / 2);
+  const int per_channel = (quant & NOVA_QUANT_PER_CHANNEL) ? 1 : 0;
+  if (!(quant & NOVA_QUANT_GIVEN)) {
+    cudaError_t e = cudaMemsetAsync(scales, 0, sizeof(float) * K, s);
+    if (e != cudaSuccess) return (int)e;
+    filter_transform_kernel<M, T, AbsmaxSink><<<blocks_for(work, 256), 256, 0, s>>>(
+        plan->kcoefs, (const T*)g, AbsmaxSink{(unsigned*)scales, per_channel, 0.f, nullptr}, K, C);
+    scales_from_absmax_kernel<<<1, 256, 0, s>>>(scales, K, per_channel);
+  }
+  filter_transform_kernel<M, T, QuantSink><<<blocks_for(work, 256), 256, 0, s>>>(
+      plan->kcoefs, (const T*)g, QuantSink{(int8_t*)Uq, scales, 1, 0.f}, K, C);
+  return (int)cudaGetLastError();
+}
+// int8 input transform over tiles p0 .. p0+pc-1.  pass 0: absmax into *slot (zeroed by the caller);
+// pass 1: quantise with the scale at *slot.
+template <int M, typename T>
+int input_launch_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot, int pass,
+                      long long p0, int pc, int pc_pad, cudaStream_t s) {
+  constexpr int THREADS = 32 * (M + 2) * 2;
+  const long long work = (long long)pc * (g.C / 2);
+  const unsigned grid = blocks_for(work, 128);
+#define NOVA_IT8(SYMV, SINK, ...)                                                                         \
+  input_transform_kernel<M, T, SYMV, SINK><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, __VA_ARGS__, g.H, \
+                                                                   g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad)
+  if (pass == 0) {
+    if (plan->symmetric) NOVA_IT8(true, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
+    else NOVA_IT8(false, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
+  } else {
+    if (plan->symmetric) NOVA_IT8(true, QuantSink, QuantSink{(int8_t*)Vq, slot, 0, 0.f});
+    else NOVA_IT8(false, QuantSink, QuantSink{(int8_t*)Vq, slot, 0, 0.f});
+  }
+#undef NOVA_IT8
   return (int)cudaGetLastError();
 }
 template <int M, typename T>
@@ -280,11 +386,11 @@ int input_launch(const nova_plan* plan, const Geom& g, const void* x, void* V, l
   const long long work = (long long)pc * (g.C / 2);
   const unsigned grid = blocks_for(work, 128);
   if (plan->symmetric)
-    input_transform_kernel<M, T, true><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, (T*)V, g.H, g.W,
-                                                                g.C, g.Th, g.Tw, p0, pc, pc_pad);
+    input_transform_kernel<M, T, true, StoreSink<T>><<<grid, THREADS, 0, s>>>(
+        plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
   else
-    input_transform_kernel<M, T, false><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, (T*)V, g.H, g.W,
-                                                                 g.C, g.Th, g.Tw, p0, pc, pc_pad);
+    input_transform_kernel<M, T, false, StoreSink<T>><<<grid, THREADS, 0, s>>>(
+        plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
   return (int)cudaGetLastError();
 }
 template <int M, typename T>
@@ -325,6 +431,19 @@ int launch_input_transform(const nova_plan* plan, const Geom& g, const void* x, 
 int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y, long long p0,
                             int pc, int pc_pad, int relu, void* stream) {
   NOVA_DISPATCH_M_T(output_launch, plan, g, M, y, p0, pc, pc_pad, relu, (cudaStream_t)stream);
+}
+int launch_filter_transform_int8(const nova_plan* plan, const void* g, int K, int C, void* Uq, float* scales,
+                                 int quant, void* stream) {
+  NOVA_DISPATCH_M_T(filter_launch_int8, plan, g, K, C, Uq, scales, quant, (cudaStream_t)stream);
+}
+int launch_input_transform_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot,
+                                int pass, long long p0, int pc, int pc_pad, void* stream) {
+  NOVA_DISPATCH_M_T(input_launch_int8, plan, g, x, Vq, slot, pass, p0, pc, pc_pad, (cudaStream_t)stream);
+}
+int launch_scale_slot(float* slot, float value, int from_absmax, void* stream) {
+  if (from_absmax) scales_from_absmax_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(slot, 1, 0);
+  else set_scale_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(slot, value);
+  return (int)cudaGetLastError();
 }
 int launch_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode, void* stream) {
   const bool f32 = mode == NOVA_FP32;

@@ -456,3 +456,102 @@ def test_unpaired_scales_take_the_dense_transforms_and_stay_correct():
     y, _, plan = gpu_conv(x, g, 6, pts, nv.FP16_F32ACC, scales=(sg, sb))
     assert plan.frequency_order()[1] is False
     check_fp16(y, x, g, 6, pts, scales=(sg, sb))
+
+
+# ---------------------------------------------------------------- INT8 Winograd-domain pipeline
+def gpu_conv_int8(x, g, m, pts, quant=nv.QUANT_PER_TENSOR, scale_U=None, scale_V=0.0, flags=0, coef=nv.COEF_FP32,
+                  scales=(None, None)):
+    plan = nv.Plan(m, pts, nv.FP16_F32ACC, coef, scale_G=scales[0], scale_B=scales[1])
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    su = None if scale_U is None else torch.from_numpy(np.asarray(scale_U, dtype=np.float32))
+    Uq, sU = plan.filter_transform_int8(gd, quant, su)
+    N, H, W, C = x.shape
+    K = g.shape[0]
+    ws = torch.empty(plan.int8_workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device="cuda")
+    y = torch.full((N, H, W, K), float("nan"), dtype=torch.float16, device="cuda")
+    plan.conv2d_int8(xd, Uq, sU, scale_V, y=y, workspace=ws, flags=flags)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    sV = float(ws[:4].view(torch.float32).item())
+    return y.cpu().numpy(), Uq.cpu().numpy(), sU.cpu().numpy(), sV
+
+
+def test_int8_path_is_exact_when_the_codes_are_the_values():
+    # same construction as the oracle's pin: integer U and V inside +-127, unit scales
+    rng = np.random.default_rng(21)
+    x = rng.integers(-2, 3, size=(2, 7, 9, 16)).astype(np.float16)
+    g = (4 * rng.integers(-1, 2, size=(16, 3, 3, 16))).astype(np.float16)
+    y1 = conv.direct_conv_fp64(x, g)
+    for flags in (0, nv.GEMM_SIMT):
+        y, Uq, sU, sV = gpu_conv_int8(x, g, 2, point_set("std", 2), nv.QUANT_GIVEN, np.ones(16), 1.0, flags)
+        assert sV == 1.0 and np.all(sU == 1.0)
+        assert np.array_equal(y.astype(np.float64), y1)
+    ye, parts = conv.winograd_conv_int8_emulated(x, g, 2, point_set("std", 2), scale_U=1.0, scale_V=1.0, return_parts=True)
+    assert np.array_equal(Uq, parts["Uq"].transpose(1, 2, 0, 3).reshape(16, 16, 16))
+
+
+@pytest.mark.parametrize("kind,m", [("std", 2), ("std", 4), ("nova", 4), ("dyadic", 4), ("nova", 6), ("half", 6), ("nova", 8)])
+@pytest.mark.parametrize("quant", [nv.QUANT_PER_TENSOR, nv.QUANT_PER_CHANNEL])
+@pytest.mark.parametrize("shape", [(2, 13, 11, 16, 16), (2, 30, 30, 64, 80), (1, 17, 23, 144, 272)])
+def test_int8_path_matches_the_emulation(kind, m, quant, shape):
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", seed=500 + m)
+    pts = point_set(kind, m)
+    per_channel = quant == nv.QUANT_PER_CHANNEL
+    y, Uq, sU, sV = gpu_conv_int8(x, g, m, pts, quant)
+    ye, parts = conv.winograd_conv_int8_emulated(x, g, m, pts, per_channel=per_channel, return_parts=True)
+    n = m + 2
+    # scales: the same float32 division of maxima that may differ in the last bit (other summation order)
+    np.testing.assert_allclose(sU, parts["scale_U"], rtol=3e-7)
+    np.testing.assert_allclose(sV, float(parts["scale_V"]), rtol=3e-7)
+    # codes: identical except where value / scale sits on a rounding boundary
+    Ue = parts["Uq"].transpose(1, 2, 0, 3).reshape(n * n, K, C).astype(np.int32)
+    dU = np.abs(Uq.astype(np.int32) - Ue)
+    assert dU.max() <= 1 and (dU > 0).mean() < 2e-3
+    assert np.abs(Uq).max() == 127 if not per_channel else np.array_equal(np.abs(Uq).max(axis=(0, 2)), np.full(K, 127))
+    # result: against the fp64 direct convolution, no worse than 2x the emulation (collapse rule as in half mode)
+    y1 = conv.direct_conv_fp64(x, g)
+    e_gpu, e_emu = conv.rel_l2(y, y1), conv.rel_l2(ye, y1)
+    if not np.isfinite(e_emu) or e_emu >= 1.0:
+        assert (not np.isfinite(e_gpu)) or e_gpu >= 0.5, (e_gpu, e_emu)
+    else:
+        assert e_gpu <= 2.0 * e_emu, (e_gpu, e_emu)
+        # and close to the emulation itself, element by element, up to the few codes that flipped
+        assert conv.rel_l2(y, ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3
+
+
+def test_int8_tensor_core_product_equals_the_cuda_core_product_bit_for_bit():
+    # integer arithmetic: both product kernels must give the same int32 sums, hence the same bits of y
+    x, g = make_conv_inputs(2, 29, 31, 208, 272, "fp16", seed=91)
+    pts = point_set("nova", 6)
+    a = gpu_conv_int8(x, g, 6, pts)[0]
+    b = gpu_conv_int8(x, g, 6, pts, flags=nv.GEMM_SIMT)[0]
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+
+
+def test_int8_static_scale_relu_and_rescaled_plan():
+    x, g = make_conv_inputs(1, 20, 20, 64, 64, "fp16", seed=92)
+    pts = point_set("nova", 4)
+    y0, _, _, sV = gpu_conv_int8(x, g, 4, pts)
+    y1, _, _, sV1 = gpu_conv_int8(x, g, 4, pts, scale_V=sV)              # the data-derived scale given back
+    assert sV1 == sV and np.array_equal(y0.view(np.uint16), y1.view(np.uint16))
+    yr, _, _, _ = gpu_conv_int8(x, g, 4, pts, flags=nv.RELU)
+    assert np.array_equal(yr.view(np.uint16), np.maximum(y0, 0).astype(np.float16).view(np.uint16))
+    sc = _pow2_scales(4, pts)
+    ys, _, _, _ = gpu_conv_int8(x, g, 4, pts, scales=sc)
+    ref = conv.direct_conv_fp64(x, g)
+    e = conv.rel_l2(ys, ref)
+    e_emu = conv.rel_l2(conv.winograd_conv_int8_emulated(x, g, 4, pts, scales=sc), ref)
+    assert e <= 2.0 * e_emu
+
+
+def test_int8_argument_checks():
+    plan = nv.Plan(4, point_set("nova", 4), nv.FP16_F32ACC, nv.COEF_FP32)
+    g = torch.zeros((16, 3, 3, 24), dtype=torch.float16, device="cuda")     # C not a multiple of 16
+    with pytest.raises(nv.NovaError):
+        plan.filter_transform_int8(g)
+    assert plan.int8_workspace_bytes(1, 8, 8, 24, 16) == 0
+    plan32 = nv.Plan(4, point_set("nova", 4), nv.FP32)
+    with pytest.raises(nv.NovaError) as e:
+        plan32.filter_transform_int8(torch.zeros((16, 3, 3, 16), dtype=torch.float16, device="cuda"))
+    assert e.value.status == -7
