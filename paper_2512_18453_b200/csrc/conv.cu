@@ -332,15 +332,22 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
   cudaStream_t s = (cudaStream_t)stream;
   const int pc = (int)g.P, nfreq = g.n * g.n;
   int e = 0;
+  // The tensor-core transform needs the exact hi + lo table of half-rounded coefficients; plans
+  // with float32 coefficients (and narrow layers) use the CUDA-core transform.
+  const bool tc_in = p->kron_dev && C >= 64 && !(flags & NOVA_TRANSFORM_SIMT);
+  auto transform = [&](int pass) {
+    return tc_in ? launch_input_transform_tc_int8(p, g, x, Vq, slot, pass, 0, pc, l.pad, stream)
+                 : launch_input_transform_int8(p, g, x, Vq, slot, pass, 0, pc, l.pad, stream);
+  };
   if (ev) cudaEventRecord(ev[0], s);
   if (scale_V > 0.f) {
     e = launch_scale_slot(slot, scale_V, 0, stream);
   } else {                                            // s_V = max|V| / 127 over the batch: one more pass
     if (cudaMemsetAsync(slot, 0, sizeof(float), s) != cudaSuccess) return NOVA_ERR_CUDA;
-    e = launch_input_transform_int8(p, g, x, Vq, slot, 0, 0, pc, l.pad, stream);
+    e = transform(0);
     if (!e) e = launch_scale_slot(slot, 0.f, 1, stream);
   }
-  if (!e) e = launch_input_transform_int8(p, g, x, Vq, slot, 1, 0, pc, l.pad, stream);
+  if (!e) e = transform(1);
   if (ev) cudaEventRecord(ev[1], s);
   if (!e)
     e = (flags & NOVA_GEMM_SIMT) ? launch_gemm_simt_i8(Vq, Uq, Mb, nfreq, pc, l.pad, C, K, stream)

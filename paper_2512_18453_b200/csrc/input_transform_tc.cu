@@ -83,11 +83,15 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
       : "memory");
 }
 
-template <int M>
+// QMODE 0: V rounded to half.  QMODE 1: nothing is stored; the largest |V| is reduced into *qslot
+// (as float bits; first pass of the int8 pipeline's data-derived scale).  QMODE 2: V / *qslot
+// rounded to nearest even and saturated to signed 8 bit (the quantiser of the INT8 set-up,
+// Section 5.1), one float division per value.
+template <int M, int QMODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
-                          __half* __restrict__ V, int C, int Th, int Tw, long long p0, int pc, int pc_pad,
-                          int* __restrict__ status) {
+                          void* __restrict__ Vout, int C, int Th, int Tw, long long p0, int pc, int pc_pad,
+                          int* __restrict__ status, float* __restrict__ qslot) {
   using Cfg = TcCfg<M>;
   static_assert(TcCfgCheck<M>::ok, "");
   constexpr int kStages = Cfg::kStages;
@@ -196,6 +200,11 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
     const int quad = warp & 3;                    // the TMEM lane quadrant this warp may read
     const int group = (warp - kProdWarps - kMmaWarps) >> 2;
     const size_t f_stride = (size_t)pc_pad * C;
+    float qs = 1.f, amax = 0.f;
+    if constexpr (QMODE == 2) {
+      qs = *qslot;
+      if (qs == 0.f) qs = 1.f;
+    }
     for (uint32_t local = group; local < n_local && !timed_out; local += kEpiGroups) {
       const unsigned u = blockIdx.x + local * gridDim.x;
       const int cblk = (int)(u % (unsigned)CB), pl = (int)(u / (unsigned)CB);
@@ -204,7 +213,8 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
-      __half* dst = V + (size_t)pl * C + c;
+      __half* dst = reinterpret_cast<__half*>(Vout) + (size_t)pl * C + c;
+      int8_t* dst8 = reinterpret_cast<int8_t*>(Vout) + (size_t)pl * C + c;
 #pragma unroll
       for (int col0 = 0; col0 < Cfg::NFP; col0 += 64) {
         constexpr int kMaxCols = 64;
@@ -222,11 +232,24 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
 #pragma unroll
           for (int cc = 0; cc < kMaxCols; ++cc)
             if (col0 + cc < Cfg::NF) {
-              *dst = __float2half_rn(__uint_as_float(r[cc]));
-              dst += f_stride;
+              const float v = __uint_as_float(r[cc]);
+              if constexpr (QMODE == 0) {
+                *dst = __float2half_rn(v);
+                dst += f_stride;
+              } else if constexpr (QMODE == 1) {
+                amax = fmaxf(amax, fabsf(v));
+              } else {
+                const int q = __float2int_rn(__fdiv_rn(v, qs));
+                *dst8 = (int8_t)max(-128, min(127, q));
+                dst8 += f_stride;
+              }
             }
         }
       }
+    }
+    if constexpr (QMODE == 1) {                   // non-negative floats order like their bit patterns
+      const unsigned mx = __reduce_max_sync(0xffffffffu, __float_as_uint(amax));
+      if (lane == 0) atomicMax(reinterpret_cast<unsigned*>(qslot), mx);
     }
   }
 
@@ -261,13 +284,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int M>
+template <int M, int QMODE>
 int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc, int pc_pad,
-             cudaStream_t stream) {
+             float* qslot, cudaStream_t stream) {
   using Cfg = TcCfg<M>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M>,
+    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M, QMODE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
@@ -298,8 +321,8 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long 
   const int sms = plan->sm_count;
   const long long units = (long long)pc * ((g.C + 127) / 128);
   const int grid = (int)(units < sms ? units : sms);
-  input_transform_tc_kernel<M><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
-      tmX, tmK, (__half*)V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev);
+  input_transform_tc_kernel<M, QMODE><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
+      tmX, tmK, V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev, qslot);
   return (int)cudaGetLastError();
 }
 
@@ -334,11 +357,29 @@ int launch_input_transform_tc(const nova_plan* plan, const Geom& g, const void* 
                               int pc, int pc_pad, void* stream) {
   cudaStream_t s = (cudaStream_t)stream;
   switch (plan->m) {
-    case 2: return launch_m<2>(plan, g, x, V, p0, pc, pc_pad, s);
-    case 4: return launch_m<4>(plan, g, x, V, p0, pc, pc_pad, s);
-    case 6: return launch_m<6>(plan, g, x, V, p0, pc, pc_pad, s);
-    case 8: return launch_m<8>(plan, g, x, V, p0, pc, pc_pad, s);
+    case 2: return launch_m<2, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+    case 4: return launch_m<4, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+    case 6: return launch_m<6, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+    case 8: return launch_m<8, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
   }
+  return (int)cudaErrorInvalidValue;
+}
+
+// int8 pipeline: pass 0 reduces max|V| into *slot (zeroed by the caller), pass 1 quantises with
+// the scale at *slot into Vq [n*n][pc_pad][C] signed bytes.
+int launch_input_transform_tc_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot,
+                                   int pass, long long p0, int pc, int pc_pad, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+#define NOVA_TC8(MM) \
+  return pass == 0 ? launch_m<MM, 1>(plan, g, x, Vq, p0, pc, pc_pad, slot, s) \
+                   : launch_m<MM, 2>(plan, g, x, Vq, p0, pc, pc_pad, slot, s)
+  switch (plan->m) {
+    case 2: NOVA_TC8(2);
+    case 4: NOVA_TC8(4);
+    case 6: NOVA_TC8(6);
+    case 8: NOVA_TC8(8);
+  }
+#undef NOVA_TC8
   return (int)cudaErrorInvalidValue;
 }
 

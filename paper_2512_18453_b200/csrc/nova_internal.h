@@ -87,6 +87,8 @@ int launch_filter_transform_int8(const nova_plan* plan, const void* g, int K, in
                                  int quant, void* stream);
 int launch_input_transform_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot,
                                 int pass, long long p0, int pc, int pc_pad, void* stream);
+int launch_input_transform_tc_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot,
+                                   int pass, long long p0, int pc, int pc_pad, void* stream);
 int launch_scale_slot(float* slot, float value, int from_absmax, void* stream);
 int launch_gemm_tcgen05_i8(const nova_plan* plan, const void* V, const void* U, int32_t* M, int nfreq, int pc,
                            int pc_pad, int C, int K, int* status_dev, void* stream);

@@ -502,8 +502,8 @@ def test_int8_path_matches_the_emulation(kind, m, quant, shape):
     ye, parts = conv.winograd_conv_int8_emulated(x, g, m, pts, per_channel=per_channel, return_parts=True)
     n = m + 2
     # scales: the same float32 division of maxima that may differ in the last bit (other summation order)
-    np.testing.assert_allclose(sU, parts["scale_U"], rtol=3e-7)
-    np.testing.assert_allclose(sV, float(parts["scale_V"]), rtol=3e-7)
+    np.testing.assert_allclose(sU, parts["scale_U"], rtol=2e-6)
+    np.testing.assert_allclose(sV, float(parts["scale_V"]), rtol=2e-6)
     # codes: identical except where value / scale sits on a rounding boundary
     Ue = parts["Uq"].transpose(1, 2, 0, 3).reshape(n * n, K, C).astype(np.int32)
     dU = np.abs(Uq.astype(np.int32) - Ue)
@@ -555,3 +555,27 @@ def test_int8_argument_checks():
     with pytest.raises(nv.NovaError) as e:
         plan32.filter_transform_int8(torch.zeros((16, 3, 3, 16), dtype=torch.float16, device="cuda"))
     assert e.value.status == -7
+
+
+@pytest.mark.parametrize("kind,m", [("std", 4), ("nova", 4), ("nova", 6), ("half", 6), ("nova", 8)])
+@pytest.mark.parametrize("shape", [(2, 30, 30, 64, 80), (1, 17, 23, 144, 272), (3, 40, 36, 256, 64)])
+def test_int8_path_with_tensor_core_input_transform(kind, m, shape):
+    # half-rounded coefficient tables: the quantising input transform runs on the tensor cores
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", seed=600 + m)
+    pts = point_set(kind, m)
+    y, Uq, sU, sV = gpu_conv_int8(x, g, m, pts, coef=nv.COEF_ROUND_TO_MODE)
+    ye, parts = conv.winograd_conv_int8_emulated(x, g, m, pts, coef="mode", return_parts=True)
+    np.testing.assert_allclose(sV, float(parts["scale_V"]), rtol=2e-6)
+    y1 = conv.direct_conv_fp64(x, g)
+    e_gpu, e_emu = conv.rel_l2(y, y1), conv.rel_l2(ye, y1)
+    if not np.isfinite(e_emu) or e_emu >= 1.0:
+        assert (not np.isfinite(e_gpu)) or e_gpu >= 0.5, (e_gpu, e_emu)
+    else:
+        assert e_gpu <= 2.0 * e_emu, (e_gpu, e_emu)
+        assert conv.rel_l2(y, ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3
+    # the CUDA-core transform of the same plan: the same codes up to rounding-boundary flips
+    y2, _, _, sV2 = gpu_conv_int8(x, g, m, pts, coef=nv.COEF_ROUND_TO_MODE, flags=nv.TRANSFORM_SIMT)
+    np.testing.assert_allclose(sV2, sV, rtol=2e-6)
+    if np.isfinite(e_emu) and e_emu < 1.0:
+        assert conv.rel_l2(y2, y.astype(np.float64)) <= 0.25 * e_emu + 1e-3
