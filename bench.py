@@ -428,6 +428,212 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_int8(args):
+    """The INT8 Winograd-domain pipeline on the same workloads: one step = one
+    nova_conv2d_fwd_int8 call (quantising input transform - two passes when the scale of V is
+    derived from the data -, kind::i8 tensor-core product, dequantising output transform)."""
+    import numpy as np
+    import torch
+    import paper_2512_18453_b200 as nv
+    from synth import point_set, make_conv_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    c = workload(args.workload)
+    if args.images:
+        import dataclasses
+        c = dataclasses.replace(c, N=args.images, name="%s[N=%d]" % (c.name, args.images))
+    direct, actual, _, P = flops(c)
+    n2 = (c.m + 2) ** 2
+    min_bytes = 2.0 * c.N * c.H * c.W * (c.C + c.K) + 1.0 * n2 * c.K * c.C
+    pts = point_set(args.points, c.m)
+    coef = nv.COEF_FP32 if args.int8_coef == "fp32" else nv.COEF_ROUND_TO_MODE
+    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef)
+    quant = nv.QUANT_PER_CHANNEL if args.int8_quant == "per_channel" else nv.QUANT_PER_TENSOR
+    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, rank_seed(c.seed, rank))
+    g = torch.from_numpy(g_np).cuda()
+    n_sets = 3
+    xs = [torch.from_numpy(np.roll(x_np, i, axis=0)).cuda() for i in range(n_sets)]
+    ys = [torch.empty(c.N, c.H, c.W, c.K, dtype=torch.float16, device="cuda") for _ in range(n_sets)]
+    ws = torch.empty(plan.int8_workspace_bytes(c.N, c.H, c.W, c.C, c.K), dtype=torch.uint8, device="cuda")
+    Uq, sU = plan.filter_transform_int8(g, quant)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        Uq, sU = plan.filter_transform_int8(g, quant)
+    e1.record()
+    torch.cuda.synchronize()
+    filter_ms = e0.elapsed_time(e1) / 5
+    scale_V = 0.0
+    if args.int8_static_scale:                      # calibrate once on the first buffer set
+        plan.conv2d_int8(xs[0], Uq, sU, 0.0, y=ys[0], workspace=ws)
+        torch.cuda.synchronize()
+        scale_V = float(ws[:4].view(torch.float32).item())
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_direct(i):
+        plan.conv2d_int8(xs[i % n_sets], Uq, sU, scale_V, y=ys[i % n_sets], workspace=ws)
+
+    step = step_direct
+    step_direct(0)
+    torch.cuda.synchronize()
+    if args.launch == "graph":
+        graphs = []
+        side = torch.cuda.Stream()
+        for i in range(n_sets):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gr, stream=side):
+                    step_direct(i)
+            graphs.append(gr)
+        torch.cuda.synchronize()
+
+        def step(i):
+            graphs[i % n_sets].replay()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_per_step = max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / args.steps
+    status = plan.device_status()
+    kms = [0.0] * 4
+    prof_steps = min(args.steps, 20)
+    for i in range(prof_steps):
+        _, t = plan.conv2d_int8(xs[i % n_sets], Uq, sU, scale_V, y=ys[i % n_sets], workspace=ws, timed=True)
+        kms = [a + b for a, b in zip(kms, t)]
+    kms = [v / prof_steps for v in kms]
+    clocks = sampler.stop() if rank == 0 else None
+
+    # end to end: pinned host input in, host output back, around the C-ABI call
+    xh = torch.from_numpy(x_np).pin_memory()
+    yh = torch.empty(c.N, c.H, c.W, c.K, dtype=torch.float16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step(i):
+        xs[i % n_sets].copy_(xh, non_blocking=True)
+        plan.conv2d_int8(xs[i % n_sets], Uq, sU, scale_V, y=ys[i % n_sets], workspace=ws)
+        yh.copy_(ys[i % n_sets], non_blocking=True)
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / e2e_steps
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = read_peaks()
+    passes = 1 if scale_V > 0 else 2
+    names = ["input_transform_int8 (%d pass%s)" % (passes, "" if passes == 1 else "es"), "product_tcgen05_i8",
+             "output_transform_dequant"]
+    # algorithmic work per step of each kernel class; the int8 tensor peak is twice the measured
+    # bf16 one (nominal ratio of the dense peaks)
+    alg = [("hbm", passes * 2.0 * c.N * c.H * c.W * c.C + 1.0 * n2 * P * c.C),
+           ("tensor", actual),
+           ("hbm", 4.0 * n2 * P * c.K + 2.0 * c.N * c.H * c.W * c.K)]
+    dom = max(range(3), key=lambda i: kms[i])
+    bound, work = alg[dom]
+    dur = kms[dom] * 1e-3
+    i8_peak = 2.0 * peaks["tflops_burst"]
+    if bound == "tensor":
+        achieved, peak, runit = work / dur / 1e12, i8_peak, "TOP/s"
+    else:
+        achieved, peak, runit = work / dur / 1e9, peaks["hbm_gbs"], "GB/s"
+    roof_s = max(actual / (i8_peak * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
+    out = {
+        "metric": METRIC.replace("fp16", "int8"), "value": whole_job_value(world, direct, ms_per_step), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8 (s32 accumulate)",
+        "data": "synthetic",
+        "config": {
+            "workload": "%s: F(%dx%d,3x3) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
+                        % (c.name, c.m, c.m, args.points, c.N, c.C, c.K, c.H),
+            "step": "nova_conv2d_fwd_int8 (%s scale of U, %s scale of V, %s coefficient tables)"
+                    % (args.int8_quant, "static" if scale_V > 0 else "data-derived", args.int8_coef),
+            "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 126 MB L2)"
+                  % (n_sets, n_sets * (x_np.nbytes + ys[0].numel() * 2) / 1e6),
+            "launch": "CUDA graph replay of the step's kernels" if args.launch == "graph" else "direct launches",
+        },
+        "tops_actual": world * actual / (ms_per_step * 1e-3) / 1e12,
+        "path_roofline": {"roofline_us": roof_s * 1e6, "achieved_us": ms_per_step * 1e3,
+                          "frac": roof_s / (ms_per_step * 1e-3), "peaks": peaks["source"] + "; int8 tensor peak = 2 x bf16"},
+        "kernels_ms_per_step": dict(zip(names, kms[:3])),
+        "filter_transform_ms": filter_ms,
+        "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
+                     "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"], "launch_us": dur * 1e6},
+        "e2e": {"value": world * direct / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(x_np.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)},
+        "gpu_launches": (3 + 2 * passes) * args.steps if scale_V == 0 else 4 * args.steps,
+        "device_status": status, "kappa2_V": plan.kappa(), "clocks": clocks,
+    }
+    if world == 1 and (args.accuracy or not args.no_cpu_baseline):
+        out["accuracy"] = accuracy_report_int8(c, nv, torch, coef, args.int8_coef)
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = time_oracle(c)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def accuracy_report_int8(c, nv, torch, coef, coef_name, n_img=2):
+    """rel-L2 of the INT8 pipeline against the fp64 direct convolution per point set, per-tensor and
+    per-channel, with and without power-of-two range scaling; the oracle's emulation beside it."""
+    import numpy as np
+    from oracle import conv
+    from synth import make_conv_inputs, point_set, pow2_range_scales
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    y1 = conv.direct_conv_fp64(x, g)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    rep = {}
+    for kind in c.point_kinds:
+        pts = point_set(kind, c.m)
+        _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC).matrices()
+        for label, sc in ((kind, (None, None)), (kind + "+pow2_rows", pow2_range_scales(G, BT))):
+            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef, scale_G=sc[0], scale_B=sc[1])
+            for qname, quant in (("per_tensor", nv.QUANT_PER_TENSOR), ("per_channel", nv.QUANT_PER_CHANNEL)):
+                Uq, sU = plan.filter_transform_int8(gd, quant)
+                y = plan.conv2d_int8(xd, Uq, sU, 0.0)
+                torch.cuda.synchronize()
+                yh = y.cpu().numpy().astype(np.float32)
+                e_gpu = conv.rel_l2(yh, y1)
+                e_emu = conv.rel_l2(conv.winograd_conv_int8_emulated(
+                    x, g, c.m, pts, per_channel=(qname == "per_channel"),
+                    coef="fp32" if coef_name == "fp32" else "mode", scales=sc), y1)
+                rep["%s/%s" % (label, qname)] = {
+                    "kappa2_V": plan.kappa(), "rel_l2_gpu": e_gpu if np.isfinite(e_gpu) else None,
+                    "rel_l2_emulation": e_emu if np.isfinite(e_emu) else None,
+                    "nonfinite_outputs": int((~np.isfinite(yh)).sum())}
+    return {"sample": "first %d images of %s" % (n_img, c.name), "points": rep}
+
+
 def run_vgg(args):
     """cfg5: the 13 convolution layers of VGG-16 (ReLU in the epilogue, 2x2 max-pool between the
     blocks) on a synthetic 224x224 batch, F(8,3) NOVA points unless --points says otherwise.
@@ -552,12 +758,20 @@ def main():
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--accuracy", action="store_true",
                     help="report rel-L2 per point set (and per rescaled variant) even with --no-cpu-baseline")
+    ap.add_argument("--int8", action="store_true", help="time the INT8 Winograd-domain pipeline instead")
+    ap.add_argument("--int8-quant", default="per_tensor", choices=["per_tensor", "per_channel"])
+    ap.add_argument("--int8-coef", default="half", choices=["half", "fp32"],
+                    help="coefficient tables: half-rounded (tensor-core input transform) or float32 (CUDA cores)")
+    ap.add_argument("--int8-static-scale", action="store_true",
+                    help="calibrate the scale of V once instead of deriving it from every batch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg5":
         run_vgg(args)
+    elif args.int8:
+        run_int8(args)
     else:
         run_ours(args)
 

@@ -270,8 +270,9 @@ int nova_conv2d_launch_count(const nova_plan* plan, int N, int H, int W, int C, 
  * Validation"; Section "Snap-to-Rational", paragraph "Rational Coefficients in Practice").  The
  * transform matrices stay in floating point (create the plan with NOVA_FP16_F32ACC and, as the
  * paper does, NOVA_COEF_FP32); the transformed filter U and the transformed input V are
- * quantised symmetrically to signed 8 bit - code = round-to-nearest-even(value / s) saturated to
- * [-128, 127], s = max|value| / 127, one float division each - the product over the input
+ * quantised symmetrically to signed 8 bit - code = round-to-nearest-even(value * (1 / s))
+ * saturated to [-128, 127], s = max|value| / 127, the reciprocal taken once per scale in float -
+ * the product over the input
  * channels is exact int32 arithmetic on the tensor cores (tcgen05 kind::i8), and the output
  * transform runs in float on float(M) * (s_U[k] * s_V), rounded once to half.  x, g and y are
  * half tensors as in nova_conv2d_fwd.  C and K must be multiples of 16.

@@ -223,12 +223,15 @@ def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False,
 # --------------------------------------------------------------------------
 def quantize_int8(v, scale):
     """Symmetric quantiser: round(v / scale) to nearest, ties to even, saturated to [-128, 127].
-    The division is one float32 operation (the decision is taken in float32).  scale may be an
-    array broadcastable against v; a zero scale (an all-zero tensor) is treated as 1."""
+    As is customary in quantised inference the division is carried out as one float32
+    multiplication by the reciprocal scale r = 1 / scale, itself one float32 division per scale
+    (the decision is taken in float32).  scale may be an array broadcastable against v; a zero
+    scale (an all-zero tensor) is treated as 1."""
     v = np.asarray(v, dtype=np.float32)
     s = np.asarray(scale, dtype=np.float32)
     s = np.where(s == 0, np.float32(1), s)
-    q = np.rint(v / s)                                  # float32 / float32 -> float32; rint = ties to even
+    r = (np.float32(1) / s).astype(np.float32)
+    q = np.rint(v * r)                                  # float32 product; rint = ties to even
     return np.clip(q, -128, 127).astype(np.int8)
 
 

@@ -86,7 +86,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
 // QMODE 0: V rounded to half.  QMODE 1: nothing is stored; the largest |V| is reduced into *qslot
 // (as float bits; first pass of the int8 pipeline's data-derived scale).  QMODE 2: V / *qslot
 // rounded to nearest even and saturated to signed 8 bit (the quantiser of the INT8 set-up,
-// Section 5.1), one float division per value.
+// Section 5.1), as one float multiplication by the reciprocal scale per value.
 template <int M, int QMODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
@@ -204,6 +204,7 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
     if constexpr (QMODE == 2) {
       qs = *qslot;
       if (qs == 0.f) qs = 1.f;
+      qs = __fdiv_rn(1.f, qs);                    // the quantiser multiplies by the reciprocal scale
     }
     for (uint32_t local = group; local < n_local && !timed_out; local += kEpiGroups) {
       const unsigned u = blockIdx.x + local * gridDim.x;
@@ -228,7 +229,32 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
           __syncwarp();
           if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
-        if (c < C) {
+        if constexpr (QMODE == 2) {
+          // Four frequencies at a time: a lane packs its channel's four codes into a word, the
+          // four lanes of a group transpose the 4 x 4 bytes with two shuffles, and lane i of the
+          // group stores frequency i's four consecutive channels as one word (C % 16 == 0, so a
+          // group of four channels is inside or outside the tensor as a whole).
+          const int li = lane & 3;
+          int8_t* d4 = dst8 - li + (size_t)li * f_stride;
+#pragma unroll
+          for (int cc = 0; cc < kMaxCols; cc += 4)
+            if (col0 + cc < Cfg::NF) {
+              uint32_t w = 0;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                int q;
+                asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(q) : "f"(__fmul_rn(__uint_as_float(r[cc + j]), qs)));
+                w |= (uint32_t)(q & 0xff) << (8 * j);
+              }
+              const uint32_t p1 = __shfl_xor_sync(0xffffffffu, w, 1);
+              const uint32_t t = __byte_perm(w, p1, (li & 1) ? 0x3715 : 0x6240);
+              const uint32_t p2 = __shfl_xor_sync(0xffffffffu, t, 2);
+              const uint32_t o = __byte_perm(t, p2, (li & 2) ? 0x3276 : 0x5410);
+              if (c < C) *reinterpret_cast<uint32_t*>(d4) = o;
+              d4 += 4 * f_stride;
+            }
+          dst8 += (size_t)((Cfg::NF - col0 < kMaxCols) ? (Cfg::NF - col0) : kMaxCols) * f_stride;
+        } else if (c < C) {
 #pragma unroll
           for (int cc = 0; cc < kMaxCols; ++cc)
             if (col0 + cc < Cfg::NF) {
@@ -236,12 +262,8 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
               if constexpr (QMODE == 0) {
                 *dst = __float2half_rn(v);
                 dst += f_stride;
-              } else if constexpr (QMODE == 1) {
-                amax = fmaxf(amax, fabsf(v));
               } else {
-                const int q = __float2int_rn(__fdiv_rn(v, qs));
-                *dst8 = (int8_t)max(-128, min(127, q));
-                dst8 += f_stride;
+                amax = fmaxf(amax, fabsf(v));
               }
             }
         }

@@ -15,8 +15,8 @@ using namespace xf;
 
 // Where the float results of a transform go.  StoreSink rounds them to the operand type;
 // AbsmaxSink only reduces them to their largest magnitude (first pass of a data-derived int8
-// scale s = max|.| / 127); QuantSink divides by a scale read from device memory, rounds to
-// nearest even and saturates to [-128, 127] (the symmetric quantiser of the INT8 set-up,
+// scale s = max|.| / 127); QuantSink multiplies by the reciprocal of a scale read from device
+// memory, rounds to nearest even and saturates to [-128, 127] (the symmetric quantiser of the INT8 set-up,
 // Section 5.1).  Offsets are in elements of the destination.
 template <typename T>
 struct StoreSink {
@@ -42,9 +42,11 @@ struct AbsmaxSink {
     }
   }
 };
-__device__ __forceinline__ int quant_code(float v, float s) {
-  const int q = __float2int_rn(__fdiv_rn(v, s));       // one float division, ties to even
-  return max(-128, min(127, q));
+// v times the reciprocal scale, rounded to nearest even and saturated to [-128, 127]
+__device__ __forceinline__ int quant_code(float v, float r) {
+  int q;
+  asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(q) : "f"(__fmul_rn(v, r)));
+  return q;
 }
 struct QuantSink {
   int8_t* out;
@@ -54,6 +56,7 @@ struct QuantSink {
   __device__ __forceinline__ void begin(int channel) {
     s = scales[per_channel ? channel : 0];
     if (s == 0.f) s = 1.f;
+    s = __fdiv_rn(1.f, s);                              // the quantiser multiplies by the reciprocal
   }
   __device__ __forceinline__ void put(size_t off, float2 v) {
     char2 q;
