@@ -95,6 +95,9 @@ typedef void* nova_stream;            /* a cudaStream_t */
  * rationals, the decomposition identity of Section 2.4 is checked to be
  * exactly zero, and the tables are then rounded (rational -> double -> float
  * or half, round to nearest even).  Host only: works without a CUDA device.
+ * r = 3 plans drive the device path.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
+ * extension) builds a host-only plan - exact and fp64 matrices, verification, conditioning -
+ * which every device entry point refuses with NOVA_ERR_UNSUPPORTED.
  * On success *out must be released with nova_plan_destroy.
  */
 int nova_plan_create(int m, int r, const nova_rat* points_host, int n,

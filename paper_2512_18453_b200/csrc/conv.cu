@@ -46,6 +46,8 @@ bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* 
   return c->v_bytes + c->m_bytes <= bytes;
 }
 
+// The device path is written for 3 x 3 filters; plans for other filter sizes are host-only.
+bool device_plan(const nova_plan* p) { return p && p->r == kR; }
 bool shape_ok(int N, int H, int W, int C, int K) {
   return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
 }
@@ -100,7 +102,7 @@ bool use_tcgen05(const nova_plan* p, int flags) {
 using namespace nova;
 
 extern "C" size_t nova_filter_transform_bytes(const nova_plan* p, int K, int C) {
-  if (!p || K <= 0 || C <= 0) return 0;
+  if (!device_plan(p) || K <= 0 || C <= 0) return 0;
   return (size_t)p->n * p->n * K * C * elt_bytes(p->mode);
 }
 
@@ -108,17 +110,18 @@ extern "C" int nova_filter_transform(const nova_plan* p, const void* g, int K, i
                                      nova_stream stream) {
   if (!p || !aligned16(g) || !aligned16(U) || K <= 0 || C <= 0 || (K % 8) || (C % 8))
     return NOVA_ERR_INVALID_ARG;
+  if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   return launch_filter_transform(p, g, K, C, U, stream) == 0 ? NOVA_OK : NOVA_ERR_CUDA;
 }
 
 extern "C" size_t nova_conv2d_min_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
-  if (!p || !shape_ok(N, H, W, C, K)) return 0;
+  if (!device_plan(p) || !shape_ok(N, H, W, C, K)) return 0;
   Geom g = make_geom(p, N, H, W, C, K);
   return (size_t)128 * per_tile_bytes(p, g) + 4 * kAlign;
 }
 
 extern "C" size_t nova_conv2d_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
-  if (!p || !shape_ok(N, H, W, C, K)) return 0;
+  if (!device_plan(p) || !shape_ok(N, H, W, C, K)) return 0;
   Geom g = make_geom(p, N, H, W, C, K);
   const size_t pt = per_tile_bytes(p, g);
   long long pc = (long long)(kTargetChunkBytes / pt) / 128 * 128;
@@ -131,6 +134,7 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
                                         size_t workspace_bytes, int flags) {
   (void)flags;
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   Geom g = make_geom(p, N, H, W, C, K);
   int R = 0;
   size_t vb = 0;
@@ -149,6 +153,7 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
                     int K, void* ws, size_t ws_bytes, int flags, nova_stream stream, cudaEvent_t* ev) {
   if (!p || !aligned16(x) || !aligned16(U) || !aligned16(y) || !shape_ok(N, H, W, C, K))
     return NOVA_ERR_INVALID_ARG;
+  if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if ((flags & NOVA_GEMM_TCGEN05) && p->mode == NOVA_FP32) return NOVA_ERR_UNSUPPORTED;
   Geom g = make_geom(p, N, H, W, C, K);
@@ -286,6 +291,7 @@ int static_scratch_address(void** out) {
 extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const void* U, void* y, int N,
                                       int H, int W, int C, int K, int flags, nova_stream stream) {
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   if (nova_conv2d_min_workspace_bytes(p, N, H, W, C, K) > NOVA_STATIC_SCRATCH_BYTES)
     return NOVA_ERR_STATIC_LIMIT;
   void* ws = nullptr;
@@ -298,7 +304,7 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
 // INT8 Winograd-domain pipeline.
 namespace {
 bool int8_shape_ok(const nova_plan* p, int N, int H, int W, int C, int K) {
-  return p && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
+  return device_plan(p) && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
 }
 struct Int8Layout {
   int pad;                  // tiles rounded up to whole 128-row blocks
@@ -318,7 +324,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
                      nova_stream stream, cudaEvent_t* ev) {
   if (!int8_shape_ok(p, N, H, W, C, K) || !aligned16(x) || !aligned16(Uq) || !aligned16(y) || !scale_U ||
       !(scale_V >= 0.f))
-    return p && p->mode != NOVA_FP16_F32ACC ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
+    return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if (!p->status_dev) return NOVA_ERR_CUDA;
   const Geom g = make_geom(p, N, H, W, C, K);
@@ -362,7 +368,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
 }  // namespace
 
 extern "C" size_t nova_filter_transform_int8_bytes(const nova_plan* p, int K, int C) {
-  if (!p || K <= 0 || C <= 0) return 0;
+  if (!device_plan(p) || K <= 0 || C <= 0) return 0;
   return (size_t)p->n * p->n * K * C;
 }
 
@@ -372,7 +378,7 @@ extern "C" int nova_filter_transform_int8(const nova_plan* p, const void* g, int
     return NOVA_ERR_INVALID_ARG;
   if (quant != NOVA_QUANT_PER_TENSOR && quant != NOVA_QUANT_PER_CHANNEL && quant != NOVA_QUANT_GIVEN)
     return NOVA_ERR_INVALID_ARG;
-  if (p->mode != NOVA_FP16_F32ACC) return NOVA_ERR_UNSUPPORTED;
+  if (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   const int e = launch_filter_transform_int8(p, g, K, C, Uq, scale_U, quant, stream);
   if (e) g_last_cuda_error = e;
   return e ? NOVA_ERR_CUDA : NOVA_OK;

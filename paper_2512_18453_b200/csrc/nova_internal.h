@@ -8,7 +8,8 @@ namespace nova {
 
 constexpr int kMaxN = 10;   // n = m + 2 for m = 8
 constexpr int kMaxM = 8;
-constexpr int kR = 3;
+constexpr int kR = 3;        // filter taps of the device path
+constexpr int kMaxR = 5;     // filter taps a host-only plan may have
 
 // Coefficient tables as the kernels evaluate them.  Passed by value as a
 // __grid_constant__ kernel parameter, i.e. they live in the constant bank and
@@ -26,11 +27,11 @@ struct nova_plan {
   int mode, coef;
   nova_rat points[nova::kMaxN];
   double AT[nova::kMaxM * nova::kMaxN];   // m x n row-major
-  double G[nova::kMaxN * nova::kR];       // n x r
+  double G[nova::kMaxN * nova::kMaxR];    // n x r
   double BT[nova::kMaxN * nova::kMaxN];   // n x n
   double kappa2_V;
   double kappa2_mat[3], norm2_mat[3];     // kappa_2 and spectral norm of A, G, B (as scaled)
-  nova_rat AT_rat[nova::kMaxM * nova::kMaxN], G_rat[nova::kMaxN * nova::kR], BT_rat[nova::kMaxN * nova::kMaxN];
+  nova_rat AT_rat[nova::kMaxM * nova::kMaxN], G_rat[nova::kMaxN * nova::kMaxR], BT_rat[nova::kMaxN * nova::kMaxN];
   int rat_fits;                           // every exact entry fits a 64-bit numerator / denominator
   nova::Coefs coefs;                      // rounded to the coefficient precision, caller's point order
   // The kernels index frequencies in an internal point order: perm[i] is the

@@ -254,8 +254,9 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
   if (out) *out = nullptr;
   if (!points || !out) return NOVA_ERR_INVALID_ARG;
   if (m != 2 && m != 4 && m != 6 && m != 8) return NOVA_ERR_INVALID_ARG;
-  if (r != 3) return NOVA_ERR_UNSUPPORTED;
+  if (r != 3 && r != 5) return NOVA_ERR_UNSUPPORTED;
   if (n != m + r - 1) return NOVA_ERR_INVALID_ARG;
+  if (n > nova::kMaxN) return NOVA_ERR_UNSUPPORTED;   // F(8,5) would need 12 points
   if (mode != NOVA_FP32 && mode != NOVA_FP16_F32ACC) return NOVA_ERR_INVALID_ARG;
   if (coef != NOVA_COEF_ROUND_TO_MODE && coef != NOVA_COEF_FP32) return NOVA_ERR_INVALID_ARG;
 
@@ -347,6 +348,20 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
     pl->kappa2_mat[2] = cond2(Bd, n, n, &pl->norm2_mat[2]);
   }
 
+  // r = 5 plans are host-only: exact and fp64 matrices, conditioning, verification.  The device
+  // kernels are written for 3 x 3 filters; every device entry point refuses such a plan.
+  if (r != nova::kR) {
+    std::vector<double> V(nf * nf);
+    for (int i = 0; i < nf; ++i) {
+      double a = rat_to_double(al[i]), pw = 1.0;
+      for (int j = 0; j < nf; ++j) { V[i * nf + j] = pw; pw *= a; }
+    }
+    pl->kappa2_V = cond2(V, nf);
+    for (int i = 0; i < n; ++i) pl->perm[i] = i;
+    pl->device = -1;
+    *out = pl;
+    return NOVA_OK;
+  }
   const bool through_half = (mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE);
   auto rnd = [&](double v) { return through_half ? round_through_half(v) : (float)v; };
   for (int i = 0; i < m; ++i)
@@ -565,6 +580,7 @@ extern "C" int nova_plan_get_matrices(const nova_plan* p, double* AT, double* G,
 
 extern "C" int nova_plan_get_device_tables(const nova_plan* p, float* AT, float* G, float* BT) {
   if (!p) return NOVA_ERR_INVALID_ARG;
+  if (p->r != nova::kR) return NOVA_ERR_UNSUPPORTED;
   for (int i = 0; i < p->m; ++i)
     for (int q = 0; q < p->n; ++q)
       if (AT) AT[i * p->n + q] = p->coefs.AT[i][q];

@@ -80,7 +80,7 @@ def test_plan_reports_rational_overflow_and_unsupported_r():
         nv.Plan(8, pts)
     assert e.value.status == -5
     with pytest.raises(nv.NovaError) as e:
-        nv.Plan(4, point_set("std", 6), r=5)
+        nv.Plan(4, point_set("std", 6), r=4)
     assert e.value.status == -7
 
 
@@ -171,3 +171,39 @@ def test_scaled_plan_matches_the_oracle_and_keeps_symmetry_only_for_paired_scale
     assert plan.frequency_order()[1] is False
     with pytest.raises(nv.NovaError):
         nv.Plan(6, pts, scale_G=[0] * 8)
+
+
+# ---------------------------------------------------------------- host-only plans for 5 x 5 filters
+@pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("std", 6)), (4, ("nova", 6)), (6, ("std", 8)), (6, ("nova", 8))])
+def test_r5_plans_are_exact_and_host_only(m, key):
+    pts = point_set(*key)
+    plan = nv.Plan(m, pts, r=5)
+    assert plan.matrices_rational() == tc.build_matrices(m, 5, pts)
+    AT, G, BT = plan.matrices()
+    assert AT.shape == (m, m + 4) and G.shape == (m + 4, 5) and BT.shape == (m + 4, m + 4)
+    oAT, oG, oBT = (tc.to_float(M) for M in tc.build_matrices(m, 5, pts))
+    assert np.array_equal(AT, oAT) and np.array_equal(G, oG) and np.array_equal(BT, oBT)
+    assert abs(plan.kappa() / tc.kappa2_V(pts) - 1) < 1e-9
+    kap, _ = plan.kappa_matrices()
+    for got, M in zip(kap, tc.build_matrices(m, 5, pts)):
+        assert abs(got / tc.kappa2(tc.to_float(M)) - 1) < 1e-8
+    # the device path is for 3 x 3 filters: every device entry point refuses the plan
+    assert plan.filter_transform_bytes(64, 64) == 0 and plan.workspace_bytes(1, 16, 16, 64, 64) == 0
+    L = nv.lib()
+    buf = ctypes.create_string_buffer(64)
+    p16 = ctypes.c_void_p((ctypes.addressof(buf) + 15) & ~15)
+    assert L.nova_filter_transform(plan._h, p16, 8, 8, p16, None) == -7
+    assert L.nova_conv2d_fwd(plan._h, p16, p16, p16, 1, 8, 8, 8, 8, p16, 0, 0, None) == -7
+    assert plan.launch_count(1, 16, 16, 64, 64, 1 << 20) == -7
+    with pytest.raises(nv.NovaError) as e:
+        plan.device_tables()
+    assert e.value.status == -7
+
+
+def test_r5_rejects_what_it_cannot_build():
+    with pytest.raises(nv.NovaError) as e:
+        nv.Plan(8, point_set("std", 8) + [(5, 1), (-5, 1)], r=5)          # F(8,5) needs 12 points
+    assert e.value.status in (-7, -3)
+    with pytest.raises(nv.NovaError) as e:
+        nv.Plan(4, point_set("std", 6), r=4)
+    assert e.value.status == -7

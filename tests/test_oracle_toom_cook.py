@@ -199,3 +199,31 @@ def test_dyadic_points_are_exact_in_half_precision():
     # ordering of that table: well below the integer points, slightly above the 5/6, 7/6 set
     k = tc.kappa2_V(pts)
     assert tc.kappa2_V(point_set("nova", 4)) < k < 17.0 < tc.kappa2_V(point_set("std", 4))
+
+
+# ---------------------------------------------------------------- 5 x 5 filters (r = 5)
+# Table "5x5 kernel (r=5) discovery results": F(4,5) and F(6,5) on integer points have the
+# conditioning of the 3 x 3 tiles with the same number of points (2 075 and 196.9 k).  The
+# discovered r = 5 point sets are not printed, so only the integer sets can be pinned.
+R5_SETS = [(2, ("std", 4)), (4, ("std", 6)), (6, ("std", 8))]      # m, the point set with n = m + 4 points
+
+
+@pytest.mark.parametrize("m,key", R5_SETS)
+def test_r5_construction_is_exact_and_computes_the_correlation(m, key):
+    pts = point_set(*key)
+    n = m + 4
+    assert len(pts) == n
+    AT, G, BT = tc.build_matrices(m, 5, pts)
+    assert tc.decomposition_residual(m, 5, AT, G, BT) == []
+    rng = np.random.default_rng(50 + m)
+    x = [int(v) for v in rng.integers(-9, 10, n)]
+    g = [int(v) for v in rng.integers(-9, 10, 5)]
+    gt = [sum(G[p][k] * g[k] for k in range(5)) for p in range(n)]
+    xt = [sum(BT[p][j] * x[j] for j in range(n)) for p in range(n)]
+    y = [sum(AT[i][p] * gt[p] * xt[p] for p in range(n)) for i in range(m)]
+    assert y == [sum(g[k] * x[i + k] for k in range(5)) for i in range(m)]
+
+
+def test_r5_conditioning_matches_the_printed_table():
+    assert abs(tc.kappa2_V(point_set("std", 6)) / 2075 - 1) < 2e-3          # F(4,5), 7 finite points
+    assert abs(tc.kappa2_V(point_set("std", 8)) / 196.9e3 - 1) < 2e-3       # F(6,5), 9 finite points
