@@ -579,3 +579,23 @@ def test_int8_path_with_tensor_core_input_transform(kind, m, shape):
     np.testing.assert_allclose(sV2, sV, rtol=2e-6)
     if np.isfinite(e_emu) and e_emu < 1.0:
         assert conv.rel_l2(y2, y.astype(np.float64)) <= 0.25 * e_emu + 1e-3
+
+
+def test_int8_degenerate_inputs():
+    # an all-zero input: max|V| = 0, the scale is treated as 1, every code and every output is zero
+    _, g = make_conv_inputs(1, 9, 7, 16, 32, "fp16", seed=95)
+    x = np.zeros((1, 9, 7, 16), dtype=np.float16)
+    for coef in (nv.COEF_FP32, nv.COEF_ROUND_TO_MODE):
+        y, _, _, sV = gpu_conv_int8(x, g, 6, point_set("nova", 6), coef=coef)
+        assert sV == 0.0 and not y.any()
+    # an all-zero filter bank likewise (per-channel scales of zero)
+    xz, _ = make_conv_inputs(1, 9, 7, 16, 32, "fp16", seed=96)
+    y, Uq, sU, _ = gpu_conv_int8(xz, np.zeros_like(g), 6, point_set("nova", 6), quant=nv.QUANT_PER_CHANNEL)
+    assert not sU.any() and not Uq.any() and not y.any()
+    # a single pixel, fewer rows and columns than one tile
+    x1, g1 = make_conv_inputs(3, 1, 1, 16, 16, "fp16", seed=97)
+    for m in (2, 8):
+        y, _, _, _ = gpu_conv_int8(x1, g1, m, point_set("nova", m))
+        ref = conv.direct_conv_fp64(x1, g1)
+        ye = conv.winograd_conv_int8_emulated(x1, g1, m, point_set("nova", m))
+        assert conv.rel_l2(y, ref) <= 2.0 * conv.rel_l2(ye, ref) + 1e-6
