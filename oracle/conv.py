@@ -1,13 +1,13 @@
-"""Direct and Winograd 3x3 convolution on the CPU (oracle side).
+"""Direct and Winograd r x r convolution (r = 3, or 5 for the appendix's 5 x 5 extension) on the CPU (oracle side).
 
 TEST INFRASTRUCTURE ONLY - see oracle/__init__.py.
 
 Conventions (Section 2.1): cross-correlation y_i = sum_k g_k x_{i+k} (no kernel
-flip), stride 1, zero padding 1, tensors NHWC: x [N,H,W,C], g [K,3,3,C],
-y [N,H,W,K].  The paper does not say how an image is cut into tiles; the
+flip), stride 1, zero padding (r-1)/2, tensors NHWC: x [N,H,W,C], g [K,r,r,C],
+y [N,H,W,K]; the filter size r is read from g.  The paper does not say how an image is cut into tiles; the
 reading used everywhere here is: tile (th, tw) covers output rows
 m*th .. m*th+m-1, reads the n x n input patch whose top-left corner is
-(m*th - 1, m*tw - 1) from the zero-extended image, and outputs that fall
+(m*th - pad, m*tw - pad), pad = (r-1)/2, from the zero-extended image, and outputs that fall
 outside H x W are dropped.
 """
 from fractions import Fraction
@@ -28,12 +28,13 @@ def direct_conv_fp64(x, g):
     x = np.asarray(x, dtype=np.float64)
     g = np.asarray(g, dtype=np.float64)
     N, H, W, C = x.shape
-    K = g.shape[0]
-    xp = np.zeros((N, H + 2, W + 2, C), dtype=np.float64)
-    xp[:, 1:H + 1, 1:W + 1, :] = x
+    K, r = g.shape[0], g.shape[1]
+    pad = (r - 1) // 2
+    xp = np.zeros((N, H + 2 * pad, W + 2 * pad, C), dtype=np.float64)
+    xp[:, pad:H + pad, pad:W + pad, :] = x
     y = np.zeros((N, H, W, K), dtype=np.float64)
-    for a in range(3):
-        for b in range(3):
+    for a in range(r):
+        for b in range(r):
             y += xp[:, a:a + H, b:b + W, :] @ g[:, a, b, :].T
     return y
 
@@ -59,13 +60,14 @@ def rel_l2(y, y_ref):
 # --------------------------------------------------------------------------
 # tiling helpers shared by O3 / O4 (pure indexing, no arithmetic)
 # --------------------------------------------------------------------------
-def _gather_tiles(x, m):
-    """d[N,Th,Tw,a,b,C] = xz[n, m*th-1+a, m*tw-1+b, c] with zero extension."""
+def _gather_tiles(x, m, r=3):
+    """d[N,Th,Tw,a,b,C] = xz[n, m*th-pad+a, m*tw-pad+b, c] with zero extension, pad = (r-1)/2."""
     N, H, W, C = x.shape
-    n = m + 2
+    n = m + r - 1
+    pad = (r - 1) // 2
     Th, Tw = -(-H // m), -(-W // m)
-    xp = np.zeros((N, m * Th + 2, m * Tw + 2, C), dtype=x.dtype)
-    xp[:, 1:H + 1, 1:W + 1, :] = x
+    xp = np.zeros((N, m * Th + r - 1, m * Tw + r - 1, C), dtype=x.dtype)
+    xp[:, pad:H + pad, pad:W + pad, :] = x
     d = np.empty((N, Th, Tw, n, n, C), dtype=x.dtype)
     for a in range(n):
         for b in range(n):
@@ -101,12 +103,13 @@ def winograd_conv_fp64(x, g, m, points, scales=(None, None)):
     """Y = A^T [ (G g G^T) (.) (B^T d B) ] A per tile, summed over channels
     (Section B.5 for the 2-D nesting, Section 2.1 for the four steps).
     scales = (scale_G, scale_B): optional diagonal rescaling, see toom_cook.build_matrices."""
-    AT, G, BT = (tc.to_float(M_) for M_ in tc.build_matrices(m, 3, points, *scales))
+    r = np.asarray(g).shape[1]
+    AT, G, BT = (tc.to_float(M_) for M_ in tc.build_matrices(m, r, points, *scales))
     x = np.asarray(x, dtype=np.float64)
     g = np.asarray(g, dtype=np.float64)
     N, H, W, C = x.shape
     U = _two_sided(G, g, (1, 2), np.float64)            # [K,n,n,C]
-    d = _gather_tiles(x, m)                              # [N,Th,Tw,n,n,C]
+    d = _gather_tiles(x, m, r)                           # [N,Th,Tw,n,n,C]
     V = _two_sided(BT, d, (3, 4), np.float64)            # [N,Th,Tw,n,n,C]
     M = np.einsum("ntuxyc,kxyc->ntuxyk", V, U, optimize=True)
     Y = _two_sided(AT, M, (3, 4), np.float64)            # [N,Th,Tw,m,m,K]
@@ -156,14 +159,14 @@ def winograd_conv_exact(x, g, m, points):
 # --------------------------------------------------------------------------
 # O4: rounding emulation of the low-precision pipeline
 # --------------------------------------------------------------------------
-def coefficient_tables(m, points, mode, coef="mode", scales=(None, None)):
+def coefficient_tables(m, points, mode, coef="mode", scales=(None, None), r=3):
     """Transform matrices as the device evaluates them, returned as float32.
 
     mode "fp16", coef "mode": exact rational -> float64 -> float16 (round to
     nearest even) -> widened (Section 5.1 "cast to FP16"; Section C.3 "matrices
     stored in float16").  coef "fp32" or mode "fp32": rounded to float32 only.
     """
-    mats = tc.build_matrices(m, 3, points, *scales)
+    mats = tc.build_matrices(m, r, points, *scales)
     out = []
     for M_ in mats:
         a = tc.to_float(M_)
@@ -176,7 +179,7 @@ def coefficient_tables(m, points, mode, coef="mode", scales=(None, None)):
 
 def filter_transform_emulated(g, m, points, mode, coef="mode", scales=(None, None)):
     """U[K,n,n,C]: fp32-evaluated G g G^T, rounded once to the operand dtype."""
-    _, G, _ = coefficient_tables(m, points, mode, coef, scales)
+    _, G, _ = coefficient_tables(m, points, mode, coef, scales, r=np.asarray(g).shape[1])
     with np.errstate(all="ignore"):
         U = _two_sided(G, np.asarray(g), (1, 2), np.float32)
         if mode == "fp16":
@@ -194,15 +197,16 @@ def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False,
     the storage dtype.  Mode "fp32" keeps every stage in float32.  Non-finite
     values propagate (Section C.4 "Saturation").
     """
-    AT, G, BT = coefficient_tables(m, points, mode, coef, scales)
+    r = np.asarray(g).shape[1]
+    AT, G, BT = coefficient_tables(m, points, mode, coef, scales, r=r)
     x = np.asarray(x)
     N, H, W, C = x.shape
     st = np.float16 if mode == "fp16" else np.float32
     with np.errstate(all="ignore"):
         U = _two_sided(G, np.asarray(g), (1, 2), np.float32).astype(st).astype(np.float32)
-        d = _gather_tiles(x.astype(np.float32), m)
+        d = _gather_tiles(x.astype(np.float32), m, r)
         V = _two_sided(BT, d, (3, 4), np.float32).astype(st).astype(np.float32)
-        n = m + 2
+        n = m + r - 1
         Th, Tw = d.shape[1], d.shape[2]
         K = U.shape[0]
         M = np.empty((N, Th, Tw, n, n, K), dtype=np.float32)

@@ -40,8 +40,8 @@ def _rng(seed, stream):
 
 
 def make_conv_inputs(N, H, W, C, K, dtype="fp16", relu_inputs=True, he_weights=True,
-                     seed=0, c_valid=None):
-    """x [N,H,W,C] and g [K,3,3,C] in the storage dtype (numpy arrays).
+                     seed=0, c_valid=None, r=3):
+    """x [N,H,W,C] and g [K,r,r,C] in the storage dtype (numpy arrays).
 
     c_valid < C zero-fills channels c_valid..C-1 of both tensors (used when a
     3-channel image is padded to 8 channels); the He fan-in is then 9*c_valid.
@@ -50,9 +50,9 @@ def make_conv_inputs(N, H, W, C, K, dtype="fp16", relu_inputs=True, he_weights=T
     x = _rng(seed, 1).standard_normal((N, H, W, C))
     if relu_inputs:
         x = np.maximum(x, 0.0)
-    g = _rng(seed, 2).standard_normal((K, 3, 3, C))
+    g = _rng(seed, 2).standard_normal((K, r, r, C))
     if he_weights:
-        g *= np.sqrt(2.0 / (9.0 * cv))
+        g *= np.sqrt(2.0 / (float(r * r) * cv))
     if cv < C:
         x[..., cv:] = 0.0
         g[..., cv:] = 0.0

@@ -274,3 +274,56 @@ def test_int8_error_ordering_follows_the_conditioning():
     assert err[("nova", 4)] < err[("std", 4)] / 2
     assert err[("std", 6)] > 1.0 and err[("nova", 6)] < err[("std", 6)] / 20
     assert err[("std", 2)] < err[("std", 4)] < err[("std", 6)]
+
+
+# ---------------------------------------------------------------- 5 x 5 filters
+def brute_force_r(x, g):
+    N, H, W, C = x.shape
+    K, r = g.shape[0], g.shape[1]
+    pad = (r - 1) // 2
+    y = np.zeros((N, H, W, K))
+    for n in range(N):
+        for h in range(H):
+            for w in range(W):
+                for a in range(r):
+                    for b in range(r):
+                        hh, ww = h + a - pad, w + b - pad
+                        if 0 <= hh < H and 0 <= ww < W:
+                            y[n, h, w, :] += g[:, a, b, :] @ x[n, hh, ww, :]
+    return y
+
+
+def test_direct_5x5_matches_nested_loops_and_closed_forms():
+    x, g = make_conv_inputs(2, 6, 7, 3, 4, dtype="fp32", seed=41, r=5)
+    assert np.allclose(conv.direct_conv_fp64(x, g), brute_force_r(x.astype(np.float64), g.astype(np.float64)), atol=1e-12)
+    delta = np.zeros((3, 5, 5, 3))
+    for k in range(3):
+        delta[k, 2, 2, k] = 1.0                      # centre tap = identity
+    assert np.array_equal(conv.direct_conv_fp64(x, delta), x.astype(np.float64))
+    shift = np.zeros((3, 5, 5, 3))
+    for k in range(3):
+        shift[k, 0, 4, k] = 1.0                      # y[h, w] = x[h - 2, w + 2]
+    y = conv.direct_conv_fp64(x, shift)
+    assert np.array_equal(y[:, 2:, :-2, :], x[:, :-2, 2:, :].astype(np.float64)) and not y[:, :2].any() and not y[:, :, -2:].any()
+
+
+@pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("nova", 6)), (4, ("std", 6)), (6, ("nova", 8))])
+def test_winograd_5x5_fp64_equals_direct(m, key):
+    x, g = make_conv_inputs(1, 13, 10, 3, 4, dtype="fp32", seed=42, r=5)
+    y1 = conv.direct_conv_fp64(x, g)
+    y3 = conv.winograd_conv_fp64(x, g, m, point_set(*key))
+    assert conv.rel_l2(y3, y1) < 1e-9
+
+
+def test_emulation_5x5_error_levels():
+    # no exact special case exists for r = 5 (the Lagrange factors contain 1/6), so the emulation is
+    # pinned by its error against the exact result: float32 near round-off, float16 near 2^-11 per
+    # stage, and the better-conditioned 7-point set no worse than the integer one
+    x, g = make_conv_inputs(1, 12, 12, 16, 8, dtype="fp16", seed=44, r=5)
+    y1 = conv.direct_conv_fp64(x, g)
+    e32 = conv.rel_l2(conv.winograd_conv_emulated(x.astype(np.float32), g.astype(np.float32), 2, point_set("std", 4), "fp32"), y1)
+    e16 = conv.rel_l2(conv.winograd_conv_emulated(x, g, 2, point_set("std", 4), "fp16"), y1)
+    assert e32 < 5e-6 and 1e-4 < e16 < 1e-2
+    e_std = conv.rel_l2(conv.winograd_conv_emulated(x, g, 4, point_set("std", 6), "fp16"), y1)
+    e_nova = conv.rel_l2(conv.winograd_conv_emulated(x, g, 4, point_set("nova", 6), "fp16"), y1)
+    assert e_nova < e_std
