@@ -95,9 +95,10 @@ typedef void* nova_stream;            /* a cudaStream_t */
  * rationals, the decomposition identity of Section 2.4 is checked to be
  * exactly zero, and the tables are then rounded (rational -> double -> float
  * or half, round to nearest even).  Host only: works without a CUDA device.
- * r = 3 plans drive the device path.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
- * extension) builds a host-only plan - exact and fp64 matrices, verification, conditioning -
- * which every device entry point refuses with NOVA_ERR_UNSUPPORTED.
+ * r = 3 plans have every kernel.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
+ * extension; g is then [K,5,5,C] and the padding 2) runs nova_filter_transform and
+ * nova_conv2d_fwd with CUDA-core transforms around the tensor-core product; the INT8 entry
+ * points and the NOVA_FUSED* flags are for r = 3 (NOVA_ERR_UNSUPPORTED / ignored).
  * On success *out must be released with nova_plan_destroy.
  */
 int nova_plan_create(int m, int r, const nova_rat* points_host, int n,

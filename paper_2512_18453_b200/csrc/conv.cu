@@ -46,8 +46,10 @@ bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* 
   return c->v_bytes + c->m_bytes <= bytes;
 }
 
-// The device path is written for 3 x 3 filters; plans for other filter sizes are host-only.
-bool device_plan(const nova_plan* p) { return p && p->r == kR; }
+// 3 x 3 filters have every kernel; 5 x 5 filters (F(2,5), F(4,5), F(6,5)) run the CUDA-core
+// transforms around the tensor-core product.  The INT8 and the fused paths are 3 x 3 only.
+bool device_plan(const nova_plan* p) { return p && (p->r == kR || p->r == 5); }
+bool device_plan_r3(const nova_plan* p) { return p && p->r == kR; }
 bool shape_ok(int N, int H, int W, int C, int K) {
   return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
 }
@@ -56,7 +58,7 @@ bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15
 // The single-kernel path applies in half mode with the tensor-core transforms, when the
 // scratch holds a ring of at least two 128-tile blocks (or all of them).  *R = ring length.
 bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R) {
-  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev) return false;
+  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev || p->r != kR) return false;
   if (!(flags & NOVA_FUSED) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT))) return false;
   if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
   const long long NB = (g.P + 127) / 128;
@@ -74,7 +76,7 @@ bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, i
 // transform with M in an L2-resident ring of *R blocks.  The scratch holds V for all tiles
 // (padded to whole blocks) and the ring.
 bool two_kernel_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R, size_t* v_bytes) {
-  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev) return false;
+  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev || p->r != kR) return false;
   if (!(flags & NOVA_FUSED_PRODUCT_OUTPUT) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT | NOVA_FUSED))) return false;
   if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
   const long long NB = (g.P + 127) / 128;
@@ -202,7 +204,7 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
     const int relu = (flags & NOVA_RELU) ? 1 : 0;
-    if ((p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
+    if ((p->status_dev && p->r == kR && !(flags & NOVA_TRANSFORM_SIMT))
             ? launch_output_transform_tma(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
             : launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream))
       return NOVA_ERR_CUDA;
@@ -304,7 +306,7 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
 // INT8 Winograd-domain pipeline.
 namespace {
 bool int8_shape_ok(const nova_plan* p, int N, int H, int W, int C, int K) {
-  return device_plan(p) && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
+  return device_plan_r3(p) && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
 }
 struct Int8Layout {
   int pad;                  // tiles rounded up to whole 128-row blocks
@@ -324,7 +326,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
                      nova_stream stream, cudaEvent_t* ev) {
   if (!int8_shape_ok(p, N, H, W, C, K) || !aligned16(x) || !aligned16(Uq) || !aligned16(y) || !scale_U ||
       !(scale_V >= 0.f))
-    return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
+    return p && (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if (!p->status_dev) return NOVA_ERR_CUDA;
   const Geom g = make_geom(p, N, H, W, C, K);
@@ -368,17 +370,18 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
 }  // namespace
 
 extern "C" size_t nova_filter_transform_int8_bytes(const nova_plan* p, int K, int C) {
-  if (!device_plan(p) || K <= 0 || C <= 0) return 0;
+  if (!device_plan_r3(p) || K <= 0 || C <= 0) return 0;
   return (size_t)p->n * p->n * K * C;
 }
 
 extern "C" int nova_filter_transform_int8(const nova_plan* p, const void* g, int K, int C, int quant, void* Uq,
                                           float* scale_U, nova_stream stream) {
+  if (p && (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p))) return NOVA_ERR_UNSUPPORTED;
   if (!p || !aligned16(g) || !aligned16(Uq) || !scale_U || K <= 0 || C <= 0 || (K % 16) || (C % 16))
     return NOVA_ERR_INVALID_ARG;
   if (quant != NOVA_QUANT_PER_TENSOR && quant != NOVA_QUANT_PER_CHANNEL && quant != NOVA_QUANT_GIVEN)
     return NOVA_ERR_INVALID_ARG;
-  if (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) return NOVA_ERR_UNSUPPORTED;
+  if (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p)) return NOVA_ERR_UNSUPPORTED;
   const int e = launch_filter_transform_int8(p, g, K, C, Uq, scale_U, quant, stream);
   if (e) g_last_cuda_error = e;
   return e ? NOVA_ERR_CUDA : NOVA_OK;

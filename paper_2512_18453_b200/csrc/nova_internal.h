@@ -17,7 +17,7 @@ constexpr int kMaxR = 5;     // filter taps a host-only plan may have
 struct Coefs {
   float BT[kMaxN][kMaxN];
   float AT[kMaxM][kMaxN];
-  float G[kMaxN][kR];
+  float G[kMaxN][kMaxR];
 };
 
 }  // namespace nova

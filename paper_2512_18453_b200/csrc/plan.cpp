@@ -348,20 +348,6 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
     pl->kappa2_mat[2] = cond2(Bd, n, n, &pl->norm2_mat[2]);
   }
 
-  // r = 5 plans are host-only: exact and fp64 matrices, conditioning, verification.  The device
-  // kernels are written for 3 x 3 filters; every device entry point refuses such a plan.
-  if (r != nova::kR) {
-    std::vector<double> V(nf * nf);
-    for (int i = 0; i < nf; ++i) {
-      double a = rat_to_double(al[i]), pw = 1.0;
-      for (int j = 0; j < nf; ++j) { V[i * nf + j] = pw; pw *= a; }
-    }
-    pl->kappa2_V = cond2(V, nf);
-    for (int i = 0; i < n; ++i) pl->perm[i] = i;
-    pl->device = -1;
-    *out = pl;
-    return NOVA_OK;
-  }
   const bool through_half = (mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE);
   auto rnd = [&](double v) { return through_half ? round_through_half(v) : (float)v; };
   for (int i = 0; i < m; ++i)
@@ -379,7 +365,8 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
     bool used[nova::kMaxN] = {};
     for (int i = 0; i < nf; ++i)
       if (al[i].n == 0) zero_at = i;
-    bool sym = zero_at >= 0 && (nf % 2) == 1;
+    // the even/odd transforms are written for 3-tap filters; 5-tap plans use the dense ones
+    bool sym = zero_at >= 0 && (nf % 2) == 1 && r == nova::kR;
     if (sym) {
       order[cnt++] = zero_at;
       used[zero_at] = true;
@@ -458,7 +445,7 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
         }
       }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
-      if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
+      if (pl->status_dev && r == nova::kR && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
         std::vector<unsigned short> img(nova::kron_table_halves(m));
         nova::build_kron_table(pl, img.data());
         void* kd = nullptr;
@@ -580,7 +567,6 @@ extern "C" int nova_plan_get_matrices(const nova_plan* p, double* AT, double* G,
 
 extern "C" int nova_plan_get_device_tables(const nova_plan* p, float* AT, float* G, float* BT) {
   if (!p) return NOVA_ERR_INVALID_ARG;
-  if (p->r != nova::kR) return NOVA_ERR_UNSUPPORTED;
   for (int i = 0; i < p->m; ++i)
     for (int q = 0; q < p->n; ++q)
       if (AT) AT[i * p->n + q] = p->coefs.AT[i][q];

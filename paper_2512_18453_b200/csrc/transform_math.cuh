@@ -112,10 +112,11 @@ __device__ __forceinline__ void bt_all_rows(const Coefs& cf, const float2 (&in)[
   }
 }
 
-// z[i] = sum_p A^T[i][p] * in[p], i < M.
-template <int M, bool SYM, typename V>
-__device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[M + 2], V (&z)[M]) {
-  constexpr int N = M + 2;
+// z[i] = sum_p A^T[i][p] * in[p], i < M.  N = M + r - 1 points; the symmetric form is written
+// for 3-tap filters (N = M + 2).
+template <int M, bool SYM, typename V, int N = M + 2>
+__device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[N], V (&z)[M]) {
+  static_assert(!SYM || N == M + 2, "symmetric output transform: 3-tap filters only");
   if constexpr (!SYM) {
 #pragma unroll
     for (int i = 0; i < M; ++i) {

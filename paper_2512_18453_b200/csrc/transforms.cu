@@ -81,30 +81,30 @@ __global__ void set_scale_kernel(float* slot, float value) { *slot = value; }
 
 // ---------------------------------------------------------------- U = G g G^T
 // One thread per (filter k, channel pair).  g [K,3,3,C] -> U [n*n][K][C].
-template <int M, typename T, typename Sink>
+template <int M, typename T, typename Sink, int R = 3>
 __global__ void __launch_bounds__(256)
 filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ g, Sink sink,
                         int K, int C) {
-  constexpr int N = M + 2;
+  constexpr int N = M + R - 1;
   const int c2 = C >> 1;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)K * c2) return;
   const int k = (int)(idx / c2);
   const int c = (int)(idx % c2) * 2;
   sink.begin(k);
-  float2 gg[3][3];
+  float2 gg[R][R];
 #pragma unroll
-  for (int a = 0; a < 3; ++a)
+  for (int a = 0; a < R; ++a)
 #pragma unroll
-    for (int b = 0; b < 3; ++b) gg[a][b] = ld2(g + ((size_t)(k * 3 + a) * 3 + b) * C + c);
-  float2 t[N][3];
+    for (int b = 0; b < R; ++b) gg[a][b] = ld2(g + ((size_t)(k * R + a) * R + b) * C + c);
+  float2 t[N][R];
 #pragma unroll
   for (int p = 0; p < N; ++p)
 #pragma unroll
-    for (int b = 0; b < 3; ++b) {
+    for (int b = 0; b < R; ++b) {
       float2 s = mul2(cf.G[p][0], gg[0][b]);
-      s = fma2(cf.G[p][1], gg[1][b], s);
-      s = fma2(cf.G[p][2], gg[2][b], s);
+#pragma unroll
+      for (int a = 1; a < R; ++a) s = fma2(cf.G[p][a], gg[a][b], s);
       t[p][b] = s;
     }
 #pragma unroll
@@ -112,8 +112,8 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
 #pragma unroll
     for (int q = 0; q < N; ++q) {
       float2 s = mul2(cf.G[q][0], t[p][0]);
-      s = fma2(cf.G[q][1], t[p][1], s);
-      s = fma2(cf.G[q][2], t[p][2], s);
+#pragma unroll
+      for (int b = 1; b < R; ++b) s = fma2(cf.G[q][b], t[p][b], s);
       sink.put(((size_t)(p * N + q) * K + k) * C + c, s);
     }
   sink.finish();
@@ -125,12 +125,12 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
 // patch's columns (nu), keeps the n x 2 intermediate in registers, applies all n rows along
 // the patch's rows (xi) and stores the 2n frequencies (xi, nu in its group).  The n/2 groups
 // of a patch sit in one block, so the patch is read from DRAM once and from L1 afterwards.
-template <int M, typename T, bool SYM, int G, typename Sink>
+template <int M, typename T, bool SYM, int G, typename Sink, int R = 3>
 __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* __restrict__ x,
                                                       Sink& V, int H, int W, int C, int h0,
                                                       int w0, long long img, size_t out_off,
                                                       size_t f_stride) {
-  constexpr int N = M + 2;
+  constexpr int N = M + R - 1;
   constexpr int RA = (G == 0) ? 0 : 2 * G - 1;
   constexpr int RB = (G == 0) ? N - 1 : 2 * G;
   float2 ta[N], tb[N];
@@ -169,11 +169,12 @@ __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* 
   }
 }
 
-template <int M, typename T, bool SYM, typename Sink>
-__global__ void __launch_bounds__(32 * (M + 2) * 2)
+template <int M, typename T, bool SYM, typename Sink, int R = 3>
+__global__ void __launch_bounds__(32 * (M + R - 1) * 2)
 input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, Sink V,
                        int H, int W, int C, int Th, int Tw, long long p0, int pc, int pc_pad) {
-  constexpr int N = M + 2;
+  constexpr int N = M + R - 1;
+  constexpr int PAD = (R - 1) / 2;
   constexpr int WORK = 128;                       // (tile, channel pair) items per block
   // threads [g*128, g*128+128) form group g (warp-uniform)
   const int g = threadIdx.x / WORK;
@@ -186,17 +187,17 @@ input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x
   const int tw = (int)(p % Tw);
   const int th = (int)((p / Tw) % Th);
   const long long img = p / ((long long)Tw * Th);
-  const int h0 = M * th - 1, w0 = M * tw - 1;
+  const int h0 = M * th - PAD, w0 = M * tw - PAD;
   const size_t out_off = (size_t)pl * C + c;
   const size_t f_stride = (size_t)pc_pad * C;
   const T* xc = x + c;
   V.begin(0);
   switch (g) {
-    case 0: input_transform_group<M, T, SYM, 0>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
-    case 1: input_transform_group<M, T, SYM, 1>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
-    case 2: if constexpr (N >= 6) input_transform_group<M, T, SYM, 2>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
-    case 3: if constexpr (N >= 8) input_transform_group<M, T, SYM, 3>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
-    case 4: if constexpr (N >= 10) input_transform_group<M, T, SYM, 4>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 0: input_transform_group<M, T, SYM, 0, Sink, R>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 1: input_transform_group<M, T, SYM, 1, Sink, R>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 2: if constexpr (N >= 6) input_transform_group<M, T, SYM, 2, Sink, R>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 3: if constexpr (N >= 8) input_transform_group<M, T, SYM, 3, Sink, R>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
+    case 4: if constexpr (N >= 10) input_transform_group<M, T, SYM, 4, Sink, R>(cf, xc, V, H, W, C, h0, w0, img, out_off, f_stride); break;
   }
   V.finish();
 }
@@ -206,12 +207,12 @@ input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x
 // writes it and this kernel reads it in 32-byte pieces.  A thread owns one tile and VEC
 // consecutive filters; a warp covers 2 tiles x 16 such units, so that its M reads are whole
 // 32-byte sectors and its y stores are 32*VEC contiguous bytes per pixel.
-template <int M, typename T, bool SYM, int VEC>
+template <int M, typename T, bool SYM, int VEC, int R = 3>
 __global__ void __launch_bounds__(256, (M == 8 || VEC == 1) ? 2 : 2)
 output_transform_kernel(const __grid_constant__ Coefs cf, const float* __restrict__ Mb,
                         T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
                         int pc_pad, int relu) {
-  constexpr int N = M + 2;
+  constexpr int N = M + R - 1;
   using Vv = typename VecOf<VEC>::type;
   const int t = threadIdx.x;
   const int unit = blockIdx.x * 128 + (t & 15) + 16 * (t >> 5);
@@ -230,7 +231,7 @@ output_transform_kernel(const __grid_constant__ Coefs cf, const float* __restric
     Vv in[N];
 #pragma unroll
     for (int nu = 0; nu < N; ++nu) in[nu] = *reinterpret_cast<const Vv*>(src + (size_t)(xi * N + nu) * f_stride);
-    at_apply<M, SYM, Vv>(cf, in, z);
+    at_apply<M, SYM, Vv, N>(cf, in, z);
   };
   if constexpr (!SYM) {
 #pragma unroll
@@ -340,6 +341,14 @@ inline unsigned blocks_for(long long work, int threads) {
 template <int M, typename T>
 int filter_launch(const nova_plan* plan, const void* g, int K, int C, void* U, cudaStream_t s) {
   const long long work = (long long)K * (C / 2);
+  if (plan->r == 5) {
+    if constexpr (M <= 6)
+      filter_transform_kernel<M, T, StoreSink<T>, 5><<<blocks_for(work, 256), 256, 0, s>>>(
+          plan->kcoefs, (const T*)g, StoreSink<T>{(T*)U}, K, C);
+    else
+      return (int)cudaErrorInvalidValue;
+    return (int)cudaGetLastError();
+  }
   filter_transform_kernel<M, T, StoreSink<T>><<<blocks_for(work, 256), 256, 0, s>>>(
       plan->kcoefs, (const T*)g, StoreSink<T>{(T*)U}, K, C);
   return (int)cudaGetLastError();
@@ -388,6 +397,14 @@ int input_launch(const nova_plan* plan, const Geom& g, const void* x, void* V, l
   constexpr int THREADS = 32 * (M + 2) * 2;       // n/2 groups of 128 work items
   const long long work = (long long)pc * (g.C / 2);
   const unsigned grid = blocks_for(work, 128);
+  if (plan->r == 5) {                               // 5-tap filters: dense transforms only
+    if constexpr (M <= 6)
+      input_transform_kernel<M, T, false, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
+          plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
+    else
+      return (int)cudaErrorInvalidValue;
+    return (int)cudaGetLastError();
+  }
   if (plan->symmetric)
     input_transform_kernel<M, T, true, StoreSink<T>><<<grid, THREADS, 0, s>>>(
         plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
@@ -401,6 +418,17 @@ int output_launch(const nova_plan* plan, const Geom& g, const void* Mb, void* y,
                   int pc_pad, int relu, cudaStream_t s) {
   constexpr int VEC = (M == 8) ? 1 : 2;
   dim3 grid(blocks_for(g.K / VEC, 128), (unsigned)((pc + 1) / 2));
+  if (plan->r == 5) {
+    if constexpr (M <= 6) {
+      constexpr int V5 = (M == 6) ? 1 : 2;            // n = 10 at m = 6: registers as for F(8,3)
+      dim3 grid5(blocks_for(g.K / V5, 128), (unsigned)((pc + 1) / 2));
+      output_transform_kernel<M, T, false, V5, 5><<<grid5, 256, 0, s>>>(
+          plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
+    } else {
+      return (int)cudaErrorInvalidValue;
+    }
+    return (int)cudaGetLastError();
+  }
   if (plan->symmetric)
     output_transform_kernel<M, T, true, VEC><<<grid, 256, 0, s>>>(
         plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);

@@ -599,3 +599,73 @@ def test_int8_degenerate_inputs():
         ref = conv.direct_conv_fp64(x1, g1)
         ye = conv.winograd_conv_int8_emulated(x1, g1, m, point_set("nova", m))
         assert conv.rel_l2(y, ref) <= 2.0 * conv.rel_l2(ye, ref) + 1e-6
+
+
+# ---------------------------------------------------------------- 5 x 5 filters (F(2,5), F(4,5), F(6,5))
+R5_CASES = [(2, ("std", 4)), (4, ("std", 6)), (4, ("nova", 6)), (4, ("half", 6)), (6, ("nova", 8))]
+
+
+def gpu_conv_r5(x, g, m, pts, mode, flags=0, ws="default"):
+    plan = nv.Plan(m, pts, mode, r=5)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    U = plan.filter_transform(gd)
+    N, H, W, C = x.shape
+    K = g.shape[0]
+    nbytes = plan.min_workspace_bytes(N, H, W, C, K) if ws == "min" else plan.workspace_bytes(N, H, W, C, K)
+    wsp = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    y = torch.full((N, H, W, K), float("nan"), dtype=xd.dtype, device="cuda")
+    plan.conv2d(xd, U, y=y, workspace=wsp, flags=flags)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    return y.cpu().numpy(), U.cpu().numpy()
+
+
+@pytest.mark.parametrize("m,key", R5_CASES)
+@pytest.mark.parametrize("shape", [(1, 3, 5, 8, 8), (2, 13, 11, 16, 24), (2, 37, 29, 40, 72)])
+def test_r5_fp32_mode_matches_direct(m, key, shape):
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp32", False, False, seed=700 + m, r=5)
+    pts = point_set(*key)
+    y, _ = gpu_conv_r5(x, g, m, pts, nv.FP32)
+    y1 = conv.direct_conv_fp64(x, g)
+    e_gpu = conv.rel_l2(y, y1)
+    e_emu = conv.rel_l2(conv.winograd_conv_emulated(x, g, m, pts, "fp32"), y1)
+    assert np.isfinite(y).all()
+    assert e_gpu <= 3.0 * e_emu + 1e-7, (e_gpu, e_emu)
+    assert e_gpu <= {("std", 4): 1e-5, ("std", 6): 5e-3, ("nova", 6): 1e-4, ("half", 6): 1e-3, ("nova", 8): 5e-3}[key], e_gpu
+
+
+@pytest.mark.parametrize("m,key", R5_CASES)
+@pytest.mark.parametrize("shape", [(2, 13, 11, 16, 8), (2, 30, 30, 64, 64), (1, 17, 23, 136, 264)])
+@pytest.mark.parametrize("flags", [0, nv.GEMM_SIMT])
+def test_r5_fp16_mode_within_twice_the_emulation(m, key, shape, flags):
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", seed=710 + m, r=5)
+    pts = point_set(*key)
+    y, U = gpu_conv_r5(x, g, m, pts, nv.FP16_F32ACC, flags)
+    check_fp16(y, x, g, m, pts)
+    n = m + 4
+    Ue = conv.filter_transform_emulated(g, m, pts, "fp16").transpose(1, 2, 0, 3).reshape(n * n, K, C)
+    d = np.abs(U.astype(np.float32) - Ue.astype(np.float32))
+    ulp = np.maximum(np.abs(Ue.astype(np.float32)), 2.0 ** -14) * 2.0 ** -10
+    assert (d <= ulp).all() and (d > 0).mean() < 0.05
+
+
+def test_r5_chunked_relu_static_and_refusals():
+    x, g = make_conv_inputs(3, 26, 22, 64, 64, "fp16", seed=720, r=5)
+    pts = point_set("nova", 6)
+    a, _ = gpu_conv_r5(x, g, 4, pts, nv.FP16_F32ACC)
+    b, _ = gpu_conv_r5(x, g, 4, pts, nv.FP16_F32ACC, ws="min")                 # several chunks
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    c, _ = gpu_conv_r5(x, g, 4, pts, nv.FP16_F32ACC, flags=nv.RELU | nv.FUSED)  # fused flag ignored for r = 5
+    assert np.array_equal(c.view(np.uint16), np.maximum(a, 0).astype(np.float16).view(np.uint16))
+    plan = nv.Plan(4, pts, nv.FP16_F32ACC, r=5)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    U = plan.filter_transform(gd)
+    ys = torch.empty((3, 26, 22, 64), dtype=torch.float16, device="cuda")
+    plan.conv2d_static(xd, U, ys)
+    torch.cuda.synchronize()
+    assert np.array_equal(ys.cpu().numpy().view(np.uint16), a.view(np.uint16))
+    with pytest.raises(nv.NovaError) as e:
+        plan.filter_transform_int8(torch.zeros((16, 3, 3, 16), dtype=torch.float16, device="cuda"))
+    assert e.value.status == -7

@@ -173,9 +173,9 @@ def test_scaled_plan_matches_the_oracle_and_keeps_symmetry_only_for_paired_scale
         nv.Plan(6, pts, scale_G=[0] * 8)
 
 
-# ---------------------------------------------------------------- host-only plans for 5 x 5 filters
+# ---------------------------------------------------------------- plans for 5 x 5 filters
 @pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("std", 6)), (4, ("nova", 6)), (6, ("std", 8)), (6, ("nova", 8))])
-def test_r5_plans_are_exact_and_host_only(m, key):
+def test_r5_plans_are_exact(m, key):
     pts = point_set(*key)
     plan = nv.Plan(m, pts, r=5)
     assert plan.matrices_rational() == tc.build_matrices(m, 5, pts)
@@ -187,17 +187,14 @@ def test_r5_plans_are_exact_and_host_only(m, key):
     kap, _ = plan.kappa_matrices()
     for got, M in zip(kap, tc.build_matrices(m, 5, pts)):
         assert abs(got / tc.kappa2(tc.to_float(M)) - 1) < 1e-8
-    # the device path is for 3 x 3 filters: every device entry point refuses the plan
-    assert plan.filter_transform_bytes(64, 64) == 0 and plan.workspace_bytes(1, 16, 16, 64, 64) == 0
-    L = nv.lib()
-    buf = ctypes.create_string_buffer(64)
-    p16 = ctypes.c_void_p((ctypes.addressof(buf) + 15) & ~15)
-    assert L.nova_filter_transform(plan._h, p16, 8, 8, p16, None) == -7
-    assert L.nova_conv2d_fwd(plan._h, p16, p16, p16, 1, 8, 8, 8, 8, p16, 0, 0, None) == -7
-    assert plan.launch_count(1, 16, 16, 64, 64, 1 << 20) == -7
-    with pytest.raises(nv.NovaError) as e:
-        plan.device_tables()
-    assert e.value.status == -7
+    # sizes follow n = m + 4; the INT8 entry points are for 3 x 3 filters only
+    assert plan.filter_transform_bytes(64, 64) == (m + 4) ** 2 * 64 * 64 * 2
+    assert plan.workspace_bytes(1, 16, 16, 64, 64) > 0
+    assert plan.int8_workspace_bytes(1, 16, 16, 64, 64) == 0
+    assert plan.frequency_order() == (list(range(m + 4)), False)      # dense transforms, caller's order
+    a16, g16, b16 = plan.device_tables()
+    with np.errstate(over="ignore"):
+        assert np.array_equal(g16, oG.astype(np.float16).astype(np.float32)) and g16.shape == (m + 4, 5)
 
 
 def test_r5_rejects_what_it_cannot_build():
