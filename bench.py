@@ -98,11 +98,14 @@ def workload(name):
     return CONFIGS[name]
 
 
+FILTER_R = 3          # filter size of the run (--filter): 3, or 5 for the 5 x 5 extension
+
+
 def flops(c):
-    n = c.m + 2
+    n = c.m + FILTER_R - 1
     th, tw = -(-c.H // c.m), -(-c.W // c.m)
     P = c.N * th * tw
-    direct = 2.0 * c.N * c.H * c.W * c.K * c.C * 9
+    direct = 2.0 * c.N * c.H * c.W * c.K * c.C * FILTER_R * FILTER_R
     actual = 2.0 * n * n * c.K * c.C * P
     min_bytes = 2.0 * c.N * c.H * c.W * (c.C + c.K) + 2.0 * n * n * c.K * c.C
     return direct, actual, min_bytes, P
@@ -120,13 +123,13 @@ def _oracle_sample(c, budget_s):
     """Inputs for a bounded sample: as many images of the batch as fit `budget_s` seconds."""
     from oracle import conv
     from synth import make_conv_inputs
-    x, g = make_conv_inputs(1, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    x, g = make_conv_inputs(1, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed, r=FILTER_R)
     conv.direct_conv_fp64(x, g)                      # page in BLAS
     t0 = time.perf_counter()
     conv.direct_conv_fp64(x, g)
     t1 = time.perf_counter() - t0
     n_img = int(max(1, min(c.N, budget_s / max(t1, 1e-4))))
-    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed, r=FILTER_R)
     return x, g, n_img
 
 
@@ -139,7 +142,7 @@ def time_oracle(c, budget_s=20.0):
         t0 = time.perf_counter()
         conv.direct_conv_fp64(x, g)
         best = min(best, time.perf_counter() - t0)
-    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * 9
+    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * FILTER_R * FILTER_R
     return {"value": fl / best / 1e12, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
             "sample": "oracle.conv.direct_conv_fp64 (fp64, numpy) on %d of %d images of %s, best of 3"
                       % (n_img, c.N, c.name)}
@@ -152,21 +155,21 @@ def accuracy_report(c, nv, torch, n_img=2):
     import numpy as np
     from oracle import conv
     from synth import make_conv_inputs, point_set
-    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed, r=FILTER_R)
     y1 = conv.direct_conv_fp64(x, g)
     xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
     from synth import pow2_range_scales
     rep = {}
     for kind in c.point_kinds:
-        pts = point_set(kind, c.m)
+        pts = point_set(kind, c.m + FILTER_R - 3)
         # each set as constructed, and with power-of-two row scales that normalise the range of
         # U and V (diagonal rescaling D_A D_G D_B = I; conditioning unchanged)
         for label, scaled in ((kind, False), (kind + "+pow2_rows", True)):
             sc = (None, None)
             if scaled:
-                _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC).matrices()
+                _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC, r=FILTER_R).matrices()
                 sc = pow2_range_scales(G, BT)
-            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, scale_G=sc[0], scale_B=sc[1])
+            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, r=FILTER_R, scale_G=sc[0], scale_B=sc[1])
             y = plan.conv2d(xd, plan.filter_transform(gd))
             torch.cuda.synchronize()
             yh = y.cpu().numpy().astype(np.float32)
@@ -188,7 +191,7 @@ def run_reference(args):
     from oracle import conv
     c = workload(args.workload)
     x, g, n_img = _oracle_sample(c, min(6.0, 120.0 / (args.steps + args.warmup)))
-    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * 9
+    fl = 2.0 * n_img * c.H * c.W * c.K * c.C * FILTER_R * FILTER_R
     for _ in range(args.warmup):
         conv.direct_conv_fp64(x, g)
     t0 = time.perf_counter()
@@ -251,11 +254,16 @@ def run_ours(args):
     if args.images:                                  # profiling aid: a smaller batch of the same layer
         import dataclasses
         c = dataclasses.replace(c, N=args.images, name="%s[N=%d]" % (c.name, args.images))
+    n_points = c.m + 2
+    if FILTER_R == 5:                                # same number of points, tile smaller by two
+        import dataclasses
+        c = dataclasses.replace(c, m=c.m - 2, name="%s[5x5,F(%d,5)]" % (c.name, c.m - 2))
     direct, actual, min_bytes, P = flops(c)
-    pts = point_set(args.points, c.m)
-    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC)
+    pts = point_set(args.points, n_points - 2)
+    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, r=FILTER_R)
     # each rank gets its own batch (weak scaling): seed offset by rank
-    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, rank_seed(c.seed, rank))
+    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, rank_seed(c.seed, rank),
+                                  r=FILTER_R)
     g = torch.from_numpy(g_np).cuda()
     n_sets = 3
     xs = [torch.from_numpy(x_np).cuda() if i == 0 else torch.from_numpy(np.roll(x_np, i, axis=0)).cuda()
@@ -362,7 +370,7 @@ def run_ours(args):
     two = launches == 2
     chunks = 1 if (fused or two) else launches // 3
     names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
-    n2 = (c.m + 2) ** 2
+    n2 = (c.m + FILTER_R - 1) ** 2
     elt = 2
     # algorithmic bytes / flops per step of each kernel class ("Kernels")
     alg = [
@@ -386,7 +394,7 @@ def run_ours(args):
     traffic = None                 # DRAM bytes per launch of that kernel from the committed ncu capture
     if two:
         names = ["input_transform", "product+output (one kernel, M ring in L2)", "-"]
-    if not fused and not two and not args.images and chunks == 1:
+    if not fused and not two and not args.images and chunks == 1 and FILTER_R == 3:
         traffic = NCU_DRAM_BYTES.get(args.workload, {}).get(names[dom])
     roof_s = max(actual / (peaks["tflops_burst"] * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
     value = whole_job_value(world, direct, ms_per_step)
@@ -395,8 +403,8 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 (f32 accumulate)", "data": "synthetic",
         "config": {
-            "workload": "%s: F(%dx%d,3x3) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
-                        % (c.name, c.m, c.m, args.points, c.N, c.C, c.K, c.H),
+            "workload": "%s: F(%dx%d,%dx%d) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
+                        % (c.name, c.m, c.m, FILTER_R, FILTER_R, args.points, c.N, c.C, c.K, c.H),
             "step": "nova_conv2d_fwd (input transform, tcgen05 product, output transform); filter transform once per layer",
             "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 126 MB L2)" % (n_sets, n_sets * (x_np.nbytes + ys[0].numel() * 2) / 1e6),
             "workspace_mb": ws_bytes / (1 << 20), "chunks": chunks, "gemm": args.gemm,
@@ -758,6 +766,8 @@ def main():
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--accuracy", action="store_true",
                     help="report rel-L2 per point set (and per rescaled variant) even with --no-cpu-baseline")
+    ap.add_argument("--filter", type=int, default=3, choices=[3, 5],
+                    help="filter size: 5 runs the 5 x 5 extension on the same layer with the tile two smaller (same points)")
     ap.add_argument("--int8", action="store_true", help="time the INT8 Winograd-domain pipeline instead")
     ap.add_argument("--int8-quant", default="per_tensor", choices=["per_tensor", "per_channel"])
     ap.add_argument("--int8-coef", default="half", choices=["half", "fp32"],
@@ -766,6 +776,8 @@ def main():
                     help="calibrate the scale of V once instead of deriving it from every batch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    global FILTER_R
+    FILTER_R = args.filter
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg5":
