@@ -204,7 +204,7 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
     const int relu = (flags & NOVA_RELU) ? 1 : 0;
-    if ((p->status_dev && p->r == kR && !(flags & NOVA_TRANSFORM_SIMT))
+    if ((p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
             ? launch_output_transform_tma(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
             : launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream))
       return NOVA_ERR_CUDA;

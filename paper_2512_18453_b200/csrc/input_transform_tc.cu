@@ -43,9 +43,10 @@ constexpr int kMmaWarps = 4;
 constexpr int kEpiGroups = 4;
 constexpr int kTcThreads = 32 * (kProdWarps + kMmaWarps + 4 * kEpiGroups);
 
-template <int M>
+template <int M, int R = 3>
 struct TcCfg {
-  static constexpr int N = M + 2;
+  static constexpr int N = M + R - 1;
+  static constexpr int PAD = (R - 1) / 2;
   static constexpr int NF = N * N;                       // frequencies = patch elements
   static constexpr int KP = (NF + 15) / 16 * 16;         // contraction length, padded to the MMA K
   static constexpr int NFP = KP;                         // MMA N, padded to a multiple of 16
@@ -65,10 +66,10 @@ struct TcCfg {
 // ahead of a barrier it waited on for its own previous use of the same slot; therefore every
 // slot (stage or accumulator) must always be handled by the same warp (group) of a role:
 // the ring lengths are multiples of the number of warps (groups) that share the ring.
-template <int M>
+template <int M, int R = 3>
 struct TcCfgCheck {
-  static_assert(TcCfg<M>::kStages % kProdWarps == 0 && TcCfg<M>::kStages % kMmaWarps == 0, "stage ring");
-  static_assert(TcCfg<M>::kNumAcc % kMmaWarps == 0 && TcCfg<M>::kNumAcc % kEpiGroups == 0, "accumulator ring");
+  static_assert(TcCfg<M, R>::kStages % kProdWarps == 0 && TcCfg<M, R>::kStages % kMmaWarps == 0, "stage ring");
+  static_assert(TcCfg<M, R>::kNumAcc % kMmaWarps == 0 && TcCfg<M, R>::kNumAcc % kEpiGroups == 0, "accumulator ring");
   static constexpr bool ok = true;
 };
 
@@ -87,13 +88,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
 // (as float bits; first pass of the int8 pipeline's data-derived scale).  QMODE 2: V / *qslot
 // rounded to nearest even and saturated to signed 8 bit (the quantiser of the INT8 set-up,
 // Section 5.1), as one float multiplication by the reciprocal scale per value.
-template <int M, int QMODE>
+template <int M, int QMODE, int R = 3>
 __global__ void __launch_bounds__(kTcThreads, 1)
 input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmKron,
                           void* __restrict__ Vout, int C, int Th, int Tw, long long p0, int pc, int pc_pad,
                           int* __restrict__ status, float* __restrict__ qslot) {
-  using Cfg = TcCfg<M>;
-  static_assert(TcCfgCheck<M>::ok, "");
+  using Cfg = TcCfg<M, R>;
+  static_assert(TcCfgCheck<M, R>::ok, "");
   constexpr int kStages = Cfg::kStages;
   constexpr int kNumAcc = Cfg::kNumAcc;
   constexpr int kAccCols = Cfg::kAccCols;
@@ -161,8 +162,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
       if (lane == 0) {
         uint8_t* dst = ring + (size_t)stage * Cfg::kStageBytes;
         mbar_expect_tx(&full_bar[stage], 2 * Cfg::NF * 128);
-        tma_load_4d(dst, &tmX, &full_bar[stage], cblk * 128, M * tw - 1, M * th - 1, img);
-        tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - 1, M * th - 1, img);
+        tma_load_4d(dst, &tmX, &full_bar[stage], cblk * 128, M * tw - Cfg::PAD, M * th - Cfg::PAD, img);
+        tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - Cfg::PAD, M * th - Cfg::PAD, img);
       }
       __syncwarp();
     }
@@ -306,13 +307,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int M, int QMODE>
+template <int M, int QMODE, int R = 3>
 int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc, int pc_pad,
              float* qslot, cudaStream_t stream) {
-  using Cfg = TcCfg<M>;
+  using Cfg = TcCfg<M, R>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M, QMODE>,
+    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M, QMODE, R>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
@@ -343,22 +344,22 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long 
   const int sms = plan->sm_count;
   const long long units = (long long)pc * ((g.C + 127) / 128);
   const int grid = (int)(units < sms ? units : sms);
-  input_transform_tc_kernel<M, QMODE><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
+  input_transform_tc_kernel<M, QMODE, R><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
       tmX, tmK, V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev, qslot);
   return (int)cudaGetLastError();
 }
 
 }  // namespace
 
-size_t kron_table_halves(int m) {
-  const int n = m + 2, nf = n * n, kp = (nf + 15) / 16 * 16, ka = (kp + 63) / 64;
+size_t kron_table_halves(int n) {
+  const int nf = n * n, kp = (nf + 15) / 16 * 16, ka = (kp + 63) / 64;
   return (size_t)2 * ka * kp * 64;
 }
 
 // Host image of the device table: [hi|lo][K atom][frequency row, padded][64 halves].
 void build_kron_table(const nova_plan* plan, unsigned short* out) {
   const int n = plan->n, nf = n * n, kp = (nf + 15) / 16 * 16, ka = (kp + 63) / 64;
-  for (size_t i = 0; i < kron_table_halves(plan->m); ++i) out[i] = 0;
+  for (size_t i = 0; i < kron_table_halves(plan->n); ++i) out[i] = 0;
   for (int xi = 0; xi < n; ++xi)
     for (int nu = 0; nu < n; ++nu)
       for (int a = 0; a < n; ++a)
@@ -378,6 +379,14 @@ void build_kron_table(const nova_plan* plan, unsigned short* out) {
 int launch_input_transform_tc(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0,
                               int pc, int pc_pad, void* stream) {
   cudaStream_t s = (cudaStream_t)stream;
+  if (plan->r == 5) {                                 // 5 x 5 filters: n = m + 4 points, halo of 2
+    switch (plan->m) {
+      case 2: return launch_m<2, 0, 5>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+      case 4: return launch_m<4, 0, 5>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+      case 6: return launch_m<6, 0, 5>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
+    }
+    return (int)cudaErrorInvalidValue;
+  }
   switch (plan->m) {
     case 2: return launch_m<2, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);
     case 4: return launch_m<4, 0>(plan, g, x, V, p0, pc, pc_pad, nullptr, s);

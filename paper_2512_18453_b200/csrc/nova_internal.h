@@ -76,7 +76,7 @@ int launch_input_transform(const nova_plan* plan, const Geom& g, const void* x, 
                            long long p0, int pc, int pc_pad, void* stream);
 int launch_input_transform_tc(const nova_plan* plan, const Geom& g, const void* x, void* V,
                               long long p0, int pc, int pc_pad, void* stream);
-size_t kron_table_halves(int m);
+size_t kron_table_halves(int n);   // n points
 void build_kron_table(const nova_plan* plan, unsigned short* out);
 int launch_output_transform(const nova_plan* plan, const Geom& g, const void* M, void* y,
                             long long p0, int pc, int pc_pad, int relu, void* stream);

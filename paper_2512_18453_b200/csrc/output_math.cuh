@@ -27,9 +27,9 @@ __device__ __forceinline__ float2 dequant(float2 bits, float2 s) {
 
 // QUANT: the stage holds the int32 sums of the int8 pipeline; every value is converted to float
 // and multiplied by qscale (this thread's filters' s_U[k] * s_V) as it is loaded.
-template <int M, bool SYM, int VEC = 1, bool QUANT = false>
+template <int M, bool SYM, int VEC = 1, bool QUANT = false, int R = 3>
 struct OutputTile {
-  static constexpr int N = M + 2;
+  static constexpr int N = M + R - 1;
   using V = typename VecOf<VEC>::type;
   const Coefs& cf;
   uint32_t sb_even, sb_odd;      // VEC = 2 uses sb_even only
@@ -52,7 +52,7 @@ struct OutputTile {
   __device__ __forceinline__ void row(V (&z)[M]) const {
     V in[N];
     fill<XI, 0>(in);
-    at_apply<M, SYM, V>(cf, in, z);
+    at_apply<M, SYM, V, N>(cf, in, z);
   }
   // dense: Y[i][j] += A^T[i][xi] * z_xi[j] for every xi
   template <int XI>

@@ -29,9 +29,9 @@ using namespace xf;
 constexpr int kConsGroups = 3;
 constexpr int kOtThreads = 32 * (1 + 4 * kConsGroups);
 
-template <int M, int VEC>
+template <int M, int VEC, int R = 3>
 struct OtCfg {
-  static constexpr int N = M + 2;
+  static constexpr int N = M + R - 1;
   static constexpr int NF = N * N;
   static constexpr int kQuads = 4 * VEC;              // filter quads per unit: 16 * VEC filters
   static constexpr int kStageBytes = NF * kQuads * 128;   // NF * kQuads rows of 128 bytes; a multiple of 1024
@@ -44,13 +44,13 @@ struct OtCfg {
 };
 
 // QUANT: M holds the int32 sums of the int8 pipeline; scale_U[k] * *scale_V dequantises filter k.
-template <int M, typename T, bool SYM, int VEC, bool QUANT>
+template <int M, typename T, bool SYM, int VEC, bool QUANT, int R = 3>
 __global__ void __launch_bounds__(kOtThreads, 1)
 output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
                             T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
                             int pc_pad, int relu, int* __restrict__ status, const float* __restrict__ scale_U,
                             const float* __restrict__ scale_V) {
-  using Cfg = OtCfg<M, VEC>;
+  using Cfg = OtCfg<M, VEC, R>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kUnitK = 16 * VEC;                    // filters per unit
   extern __shared__ uint8_t smem_raw[];
@@ -116,7 +116,7 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
         if constexpr (VEC == 1) qs = __fmul_rn(k < K ? scale_U[k] : 0.f, sv);
         else qs = make_float2(__fmul_rn(k < K ? scale_U[k] : 0.f, sv), __fmul_rn(k + 1 < K ? scale_U[k + 1] : 0.f, sv));
       }
-      OutputTile<M, SYM, VEC, QUANT>{cf, sb_even, sb_odd, qs}.run(Y);
+      OutputTile<M, SYM, VEC, QUANT, R>{cf, sb_even, sb_odd, qs}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
 
@@ -157,25 +157,25 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int M, typename T, bool SYM, int VEC, bool QUANT>
+template <int M, typename T, bool SYM, int VEC, bool QUANT, int R = 3>
 int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
                int pc_pad, int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
-  using Cfg = OtCfg<M, VEC>;
+  using Cfg = OtCfg<M, VEC, R>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC, QUANT>,
+    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
     if (e != cudaSuccess) return (int)e;
     attr_set = true;
   }
   const long long units = (long long)(pc_pad / 8) * ((g.K + 16 * VEC - 1) / (16 * VEC));
   const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
-  output_transform_tma_kernel<M, T, SYM, VEC, QUANT><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
+  output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
       tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev, scale_U, scale_V);
   return (int)cudaGetLastError();
 }
 
-template <int M>
+template <int M, int R = 3>
 int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0, int pc, int pc_pad,
              int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
   EncodeTiledFn enc = encode_fn();
@@ -184,7 +184,7 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
   const int k4 = g.K / 4;
   cuuint64_t dims[3] = {(cuuint64_t)pc_pad * 4, (cuuint64_t)k4, (cuuint64_t)(g.n * g.n)};
   cuuint64_t strides[2] = {(cuuint64_t)pc_pad * 16, (cuuint64_t)k4 * pc_pad * 16};
-  constexpr int VEC = (M <= 6) ? 2 : 1;               // packed fp32 pairs where the registers allow
+  constexpr int VEC = (M + R - 1 <= 8) ? 2 : 1;       // packed fp32 pairs where the registers allow
   cuuint32_t box[3] = {32, 4 * VEC, (cuuint32_t)(g.n * g.n)};
   cuuint32_t estr[3] = {1, 1, 1};
   if (enc(&tmM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(Mb), dims, strides, box, estr,
@@ -192,13 +192,18 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return (int)cudaErrorUnknown;
   const bool f32 = plan->mode == NOVA_FP32;
-#define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
-  if (scale_U) {                                      // int8 pipeline (half storage only)
-    if (f32) return (int)cudaErrorInvalidValue;
-    return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
+#define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q, R>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
+  if constexpr (R != 3) {                             // 5-tap filters: dense transform, no int8 pipeline
+    if (scale_U) return (int)cudaErrorInvalidValue;
+    return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
+  } else {
+    if (scale_U) {                                    // int8 pipeline (half storage only)
+      if (f32) return (int)cudaErrorInvalidValue;
+      return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
+    }
+    if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
+    return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
   }
-  if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
-  return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
 #undef NOVA_OT
 }
 
@@ -208,6 +213,14 @@ int launch_output_transform_tma(const nova_plan* plan, const Geom& g, const void
                                 int pc, int pc_pad, int relu, void* stream, const float* scale_U,
                                 const float* scale_V) {
   cudaStream_t s = (cudaStream_t)stream;
+  if (plan->r == 5) {
+    switch (plan->m) {
+      case 2: return launch_m<2, 5>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+      case 4: return launch_m<4, 5>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+      case 6: return launch_m<6, 5>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
+    }
+    return (int)cudaErrorInvalidValue;
+  }
   switch (plan->m) {
     case 2: return launch_m<2>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);
     case 4: return launch_m<4>(plan, g, Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, s);

@@ -445,8 +445,8 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
         }
       }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
-      if (pl->status_dev && r == nova::kR && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
-        std::vector<unsigned short> img(nova::kron_table_halves(m));
+      if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
+        std::vector<unsigned short> img(nova::kron_table_halves(n));
         nova::build_kron_table(pl, img.data());
         void* kd = nullptr;
         if (cudaMalloc(&kd, img.size() * 2) == cudaSuccess) {

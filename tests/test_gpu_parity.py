@@ -669,3 +669,17 @@ def test_r5_chunked_relu_static_and_refusals():
     with pytest.raises(nv.NovaError) as e:
         plan.filter_transform_int8(torch.zeros((16, 3, 3, 16), dtype=torch.float16, device="cuda"))
     assert e.value.status == -7
+
+
+@pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("nova", 6)), (6, ("nova", 8))])
+def test_r5_tensor_core_and_cuda_core_transforms_agree(m, key):
+    # C >= 64 in half mode: tensor-core input transform and TMA-staged output transform; the flag
+    # selects the CUDA-core transforms of the same plan
+    x, g = make_conv_inputs(2, 33, 27, 192, 80, "fp16", seed=730 + m, r=5)
+    pts = point_set(*key)
+    a, _ = gpu_conv_r5(x, g, m, pts, nv.FP16_F32ACC)
+    b, _ = gpu_conv_r5(x, g, m, pts, nv.FP16_F32ACC, flags=nv.TRANSFORM_SIMT)
+    y1 = conv.direct_conv_fp64(x, g)
+    ea, eb = conv.rel_l2(a, y1), conv.rel_l2(b, y1)
+    assert abs(ea / eb - 1) < 0.05, (ea, eb)
+    assert conv.rel_l2(a, b.astype(np.float64)) < 0.5 * ea + 1e-4
