@@ -683,3 +683,33 @@ def test_r5_tensor_core_and_cuda_core_transforms_agree(m, key):
     ea, eb = conv.rel_l2(a, y1), conv.rel_l2(b, y1)
     assert abs(ea / eb - 1) < 0.05, (ea, eb)
     assert conv.rel_l2(a, b.astype(np.float64)) < 0.5 * ea + 1e-4
+
+
+# ---------------------------------------------------------------- the next-row paths at the bench's full size
+def test_cfg3_full_size_5x5_filters_sampled_against_the_oracle():
+    # the launch configuration `bench.py --filter 5` times: cfg3's layer, F(4,5) on the 8-point set;
+    # images are independent, so the first two are compared with the oracle run on those two
+    c = CONFIGS["cfg3"]
+    x, g = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed, r=5)
+    pts = point_set("nova", 6)
+    y, _ = gpu_conv_r5(x, g, 4, pts, nv.FP16_F32ACC)
+    assert np.isfinite(y.astype(np.float32)).all()
+    check_fp16(y[:2], x[:2], g, 4, pts)
+    check_fp16(y[-1:], x[-1:], g, 4, pts)
+
+
+def test_cfg3_full_size_int8_sampled_against_the_oracle():
+    # the configuration `bench.py --int8` times.  The scale of V is the maximum over the whole batch:
+    # the oracle runs on three images with that scale given, and must agree that it covers them
+    c = CONFIGS["cfg3"]
+    x, g = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    pts = point_set("nova", 6)
+    y, Uq, sU, sV = gpu_conv_int8(x, g, 6, pts, coef=nv.COEF_ROUND_TO_MODE)
+    pick = [0, 17, 31]
+    ye, parts = conv.winograd_conv_int8_emulated(x[pick], g, 6, pts, coef="mode", scale_V=sV, return_parts=True)
+    assert np.abs(parts["Vq"]).max() <= 127 and sV > 0
+    np.testing.assert_allclose(sU, parts["scale_U"], rtol=2e-6)
+    y1 = conv.direct_conv_fp64(x[pick], g)
+    e_gpu, e_emu = conv.rel_l2(y[pick], y1), conv.rel_l2(ye, y1)
+    assert (e_gpu <= 2.0 * e_emu) if e_emu < 1.0 else (e_gpu >= 0.5), (e_gpu, e_emu)
+    assert conv.rel_l2(y[pick], ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3
