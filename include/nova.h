@@ -97,8 +97,7 @@ typedef void* nova_stream;            /* a cudaStream_t */
  * or half, round to nearest even).  Host only: works without a CUDA device.
  * r = 3 plans have every kernel.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
  * extension; g is then [K,5,5,C] and the padding 2) runs nova_filter_transform and
- * nova_conv2d_fwd with the same kernels instantiated for n = m + 4 and dense transform
- * arithmetic; the INT8 entry points and the NOVA_FUSED* flags are for r = 3
+ * nova_conv2d_fwd with the same kernels instantiated for n = m + 4; the INT8 entry points and the NOVA_FUSED* flags are for r = 3
  * (NOVA_ERR_UNSUPPORTED / ignored).
  * On success *out must be released with nova_plan_destroy.
  */

@@ -365,8 +365,7 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
     bool used[nova::kMaxN] = {};
     for (int i = 0; i < nf; ++i)
       if (al[i].n == 0) zero_at = i;
-    // the even/odd transforms are written for 3-tap filters; 5-tap plans use the dense ones
-    bool sym = zero_at >= 0 && (nf % 2) == 1 && r == nova::kR;
+    bool sym = zero_at >= 0 && (nf % 2) == 1;
     if (sym) {
       order[cnt++] = zero_at;
       used[zero_at] = true;

@@ -112,11 +112,10 @@ __device__ __forceinline__ void bt_all_rows(const Coefs& cf, const float2 (&in)[
   }
 }
 
-// z[i] = sum_p A^T[i][p] * in[p], i < M.  N = M + r - 1 points; the symmetric form is written
-// for 3-tap filters (N = M + 2).
+// z[i] = sum_p A^T[i][p] * in[p], i < M.  N = M + r - 1 points: 0, (N - 2) / 2 pairs +-a, infinity.
 template <int M, bool SYM, typename V, int N = M + 2>
 __device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[N], V (&z)[M]) {
-  static_assert(!SYM || N == M + 2, "symmetric output transform: 3-tap filters only");
+  constexpr int NP = (N - 2) / 2;
   if constexpr (!SYM) {
 #pragma unroll
     for (int i = 0; i < M; ++i) {
@@ -126,9 +125,9 @@ __device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[N], V (&
       z[i] = s;
     }
   } else {
-    V sm[M / 2], df[M / 2];
+    V sm[NP], df[NP];
 #pragma unroll
-    for (int q = 0; q < M / 2; ++q) {
+    for (int q = 0; q < NP; ++q) {
       sm[q] = vadd(in[1 + 2 * q], in[2 + 2 * q]);
       df[q] = vsub(in[1 + 2 * q], in[2 + 2 * q]);
     }
@@ -136,7 +135,7 @@ __device__ __forceinline__ void at_apply(const Coefs& cf, const V (&in)[N], V (&
     for (int i = 0; i < M; ++i) {
       V s = (i & 1) ? vmul(cf.AT[i][1], df[0]) : vmul(cf.AT[i][1], sm[0]);
 #pragma unroll
-      for (int q = 1; q < M / 2; ++q)
+      for (int q = 1; q < NP; ++q)
         s = (i & 1) ? vfma(cf.AT[i][1 + 2 * q], df[q], s) : vfma(cf.AT[i][1 + 2 * q], sm[q], s);
       if (i == 0) s = vadd(s, in[0]);
       if (i == M - 1) s = vadd(s, in[N - 1]);

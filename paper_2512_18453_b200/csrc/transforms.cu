@@ -397,12 +397,17 @@ int input_launch(const nova_plan* plan, const Geom& g, const void* x, void* V, l
   constexpr int THREADS = 32 * (M + 2) * 2;       // n/2 groups of 128 work items
   const long long work = (long long)pc * (g.C / 2);
   const unsigned grid = blocks_for(work, 128);
-  if (plan->r == 5) {                               // 5-tap filters: dense transforms only
-    if constexpr (M <= 6)
-      input_transform_kernel<M, T, false, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
-          plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
-    else
+  if (plan->r == 5) {                               // 5-tap filters: n = m + 4 points
+    if constexpr (M <= 6) {
+      if (plan->symmetric)
+        input_transform_kernel<M, T, true, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
+            plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
+      else
+        input_transform_kernel<M, T, false, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
+            plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
+    } else {
       return (int)cudaErrorInvalidValue;
+    }
     return (int)cudaGetLastError();
   }
   if (plan->symmetric)
@@ -422,8 +427,12 @@ int output_launch(const nova_plan* plan, const Geom& g, const void* Mb, void* y,
     if constexpr (M <= 6) {
       constexpr int V5 = (M == 6) ? 1 : 2;            // n = 10 at m = 6: registers as for F(8,3)
       dim3 grid5(blocks_for(g.K / V5, 128), (unsigned)((pc + 1) / 2));
-      output_transform_kernel<M, T, false, V5, 5><<<grid5, 256, 0, s>>>(
-          plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
+      if (plan->symmetric)
+        output_transform_kernel<M, T, true, V5, 5><<<grid5, 256, 0, s>>>(
+            plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
+      else
+        output_transform_kernel<M, T, false, V5, 5><<<grid5, 256, 0, s>>>(
+            plan->kcoefs, (const float*)Mb, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu);
     } else {
       return (int)cudaErrorInvalidValue;
     }

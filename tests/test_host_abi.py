@@ -191,7 +191,7 @@ def test_r5_plans_are_exact(m, key):
     assert plan.filter_transform_bytes(64, 64) == (m + 4) ** 2 * 64 * 64 * 2
     assert plan.workspace_bytes(1, 16, 16, 64, 64) > 0
     assert plan.int8_workspace_bytes(1, 16, 16, 64, 64) == 0
-    assert plan.frequency_order() == (list(range(m + 4)), False)      # dense transforms, caller's order
+    assert plan.frequency_order() == (list(range(m + 4)), True)       # symmetric set already in internal order
     a16, g16, b16 = plan.device_tables()
     with np.errstate(over="ignore"):
         assert np.array_equal(g16, oG.astype(np.float16).astype(np.float32)) and g16.shape == (m + 4, 5)
