@@ -221,10 +221,15 @@ int nova_conv2d_fwd_timed(const nova_plan* plan, const void* x_dev, const void* 
                           float* kernel_ms_host);
 
 /*
- * The same call for host tensors: copies x_host to x_stage_dev, runs
- * nova_conv2d_fwd, copies the result to y_host, all on `stream`.  The staging
- * buffers are device memory of the sizes of x and y.  Host buffers should be
- * page-locked for the copies to be asynchronous.
+ * The same call for host tensors: x_host is copied to x_stage_dev, convolved into
+ * y_stage_dev and copied to y_host.  The batch is cut into up to eight groups of
+ * images so that the copy in, the kernels and the copy out of different groups
+ * overlap: the copies run on two streams the library creates once per device, the
+ * kernels on `stream`; all of it is ordered after the work already in `stream`, and
+ * `stream` waits for the last copy.  The staging buffers are device memory of the
+ * sizes of x and y, the workspace as for nova_conv2d_fwd.  Host buffers must be
+ * page-locked for the copies to overlap.  The first call on a device creates the
+ * streams and events; calls from several host threads are serialised.
  */
 int nova_conv2d_fwd_host(const nova_plan* plan, const void* x_host, const void* U_dev, void* y_host,
                          int N, int H, int W, int C, int K,

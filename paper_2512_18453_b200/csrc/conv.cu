@@ -250,17 +250,75 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   return st;
 }
 
+// Streams and events of the host-buffer entry point, one set per device, made on first use.
+namespace {
+constexpr int kHostGroups = 8;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr, copied[kHostGroups] = {}, computed[kHostGroups] = {};
+};
+std::mutex g_pipe_mu;
+HostPipe g_pipe[64];
+
+HostPipe* host_pipe() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe& hp = g_pipe[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < kHostGroups && ok; ++i)
+      ok = cudaEventCreateWithFlags(&hp.copied[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
+}
+}  // namespace
+
+// The batch is cut into up to eight groups of images (images are independent): group i is copied in
+// on one internal stream, convolved on the caller's stream and copied out on another internal
+// stream, so that the two copy directions and the kernels overlap.  Everything is ordered after the
+// work already in `stream`, and `stream` waits for the last copy out.
 extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, const void* U, void* y_host,
                                     int N, int H, int W, int C, int K, void* x_stage, void* y_stage,
                                     void* ws, size_t ws_bytes, int flags, nova_stream stream) {
-  if (!p || !x_host || !y_host || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (!p || !x_host || !y_host || !x_stage || !y_stage || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t xb = (size_t)N * H * W * C * elt_bytes(p->mode);
-  const size_t yb = (size_t)N * H * W * K * elt_bytes(p->mode);
-  if (cudaMemcpyAsync(x_stage, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return NOVA_ERR_CUDA;
-  const int st = nova_conv2d_fwd(p, x_stage, U, y_stage, N, H, W, C, K, ws, ws_bytes, flags, stream);
-  if (st != NOVA_OK) return st;
-  if (cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return NOVA_ERR_CUDA;
+  const size_t x_img = (size_t)H * W * C * elt_bytes(p->mode);
+  const size_t y_img = (size_t)H * W * K * elt_bytes(p->mode);
+  std::lock_guard<std::mutex> lock(g_pipe_mu);
+  HostPipe* hp = host_pipe();
+  if (!hp) return NOVA_ERR_CUDA;
+  const int groups = N < kHostGroups ? N : kHostGroups;
+  const int per = (N + groups - 1) / groups;
+  if (cudaEventRecord(hp->start, s) != cudaSuccess || cudaStreamWaitEvent(hp->in, hp->start, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(hp->out, hp->start, 0) != cudaSuccess)
+    return NOVA_ERR_CUDA;
+  for (int gi = 0, n0 = 0; n0 < N; ++gi, n0 += per) {
+    const int n = (N - n0) < per ? (N - n0) : per;
+    const char* xh = static_cast<const char*>(x_host) + (size_t)n0 * x_img;
+    char* xs = static_cast<char*>(x_stage) + (size_t)n0 * x_img;
+    char* ys = static_cast<char*>(y_stage) + (size_t)n0 * y_img;
+    char* yh = static_cast<char*>(y_host) + (size_t)n0 * y_img;
+    if (cudaMemcpyAsync(xs, xh, (size_t)n * x_img, cudaMemcpyHostToDevice, hp->in) != cudaSuccess ||
+        cudaEventRecord(hp->copied[gi], hp->in) != cudaSuccess ||
+        cudaStreamWaitEvent(s, hp->copied[gi], 0) != cudaSuccess)
+      return NOVA_ERR_CUDA;
+    const int st = nova_conv2d_fwd(p, xs, U, ys, n, H, W, C, K, ws, ws_bytes, flags, stream);
+    if (st != NOVA_OK) return st;
+    if (cudaEventRecord(hp->computed[gi], s) != cudaSuccess ||
+        cudaStreamWaitEvent(hp->out, hp->computed[gi], 0) != cudaSuccess ||
+        cudaMemcpyAsync(yh, ys, (size_t)n * y_img, cudaMemcpyDeviceToHost, hp->out) != cudaSuccess)
+      return NOVA_ERR_CUDA;
+  }
+  if (cudaEventRecord(hp->done, hp->out) != cudaSuccess || cudaStreamWaitEvent(s, hp->done, 0) != cudaSuccess)
+    return NOVA_ERR_CUDA;
   return NOVA_OK;
 }
 

@@ -319,6 +319,27 @@ def test_host_buffer_entry_point():
     assert np.array_equal(yh.numpy(), y_dev)
 
 
+def test_host_buffer_entry_point_pipelines_ragged_groups():
+    # 11 images: groups of 2, 2, 2, 2, 2, 1 overlap their copies and kernels; two calls in a row reuse
+    # the internal streams and events; the result must be that of the device-resident call, bit for bit
+    N, H, W, C, K = 11, 26, 22, 64, 72
+    pts = point_set("nova", 4)
+    plan = nv.Plan(4, pts)
+    xs = torch.empty(N, H, W, C, dtype=torch.float16, device="cuda")
+    ys = torch.empty(N, H, W, K, dtype=torch.float16, device="cuda")
+    ws = torch.empty(plan.workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device="cuda")
+    for seed in (461, 462):
+        x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=seed)
+        U = plan.filter_transform(torch.from_numpy(g).cuda())
+        xh = torch.from_numpy(x).pin_memory()
+        yh = torch.full((N, H, W, K), float("nan"), dtype=torch.float16).pin_memory()
+        plan.conv2d_host(xh, U, yh, xs, ys, ws, flags=nv.RELU)
+        torch.cuda.synchronize()
+        y_dev, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC, flags=nv.RELU)
+        assert np.array_equal(yh.numpy(), y_dev)
+        assert plan.device_status() == 0
+
+
 # ---------------------------------------------------------------- the workload configurations at full size
 def _run_config(name, kind):
     c = CONFIGS[name]
