@@ -372,7 +372,7 @@ def run_ours(args):
     names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
     n2 = (c.m + FILTER_R - 1) ** 2
     elt = 2
-    # algorithmic bytes / flops per step of each kernel class ("Kernels")
+    # algorithmic bytes / flops per step of each kernel class
     alg = [
         ("hbm", 2.0 * c.N * c.H * c.W * c.C + elt * n2 * P * c.C),        # read x, write V
         ("tensor", actual),                                                # 2 n^2 K C P flop

@@ -1,7 +1,7 @@
 """GPU parity: the CUDA path through the C ABI against the CPU oracle, element
 by element on the same seeded inputs.
 
-Tolerances (written here, derived in the design doc):
+Tolerances (fp32: the stated absolute bounds; fp16 and int8: relative to the CPU emulation of the same roundings):
   fp32 mode : rel-L2 vs the fp64 direct convolution <= 1e-5 (m <= 4), <= 1e-4
               (m = 6); m = 8 is bounded by 1.5x the fp32 emulation of the same
               pipeline (the arithmetic's own limit, about 1e-4 .. 3e-4).
