@@ -126,6 +126,17 @@ int nova_plan_create_scaled(int m, int r, const nova_rat* points_host, int n,
  */
 int nova_snap_to_rational(double x, int max_den, nova_rat* out);
 
+/*
+ * Symmetric search (Section "Symmetric Search"): among the point sets made of pairs (p, -p), plus 0
+ * when n_finite is odd, with p a positive fraction of denominator <= max_den and p <= max_abs, the
+ * one whose Vandermonde matrix has the lowest kappa_2; every combination is evaluated.
+ * points_out receives n_finite + 1 points in the order 0, +p1, -p1, .. (p1 < p2 < ..), infinity;
+ * *kappa2_out (may be null) the winning condition number.  With max_den = 6 and max_abs = 2 the
+ * search returns the paper's discovered sets for F(4,3), F(6,3) and F(8,3) (n_finite = 5, 7, 9).
+ * NOVA_ERR_UNSUPPORTED if more than four million combinations would have to be tried.
+ */
+int nova_symmetric_search(int n_finite, int max_den, int max_abs, nova_rat* points_out, double* kappa2_out);
+
 /* Snap n_finite continuous points (the paper uses max_den = 10), append infinity and build the
  * plan; NOVA_ERR_DUPLICATE_POINT if two points snap to the same rational. */
 int nova_plan_create_f64(int m, int r, const double* finite_points_host, int n_finite, int max_den,

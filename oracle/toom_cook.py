@@ -164,3 +164,21 @@ def kappa2(M):
 
 def kappa2_V(points):
     return kappa2(vandermonde(points))
+
+
+def symmetric_search(n_finite, d_max=6, p_max=2):
+    """Symmetric search (Section "Symmetric Search"): configurations made of pairs (p, -p), plus 0
+    when the number of finite points is odd.  Candidates p are the positive rationals of the
+    snap-to-rational grid (denominator <= d_max) up to p_max; every combination is evaluated and
+    the one with the lowest kappa_2 of the Vandermonde matrix wins.  Returns (finite points in the
+    order 0, +p1, -p1, +p2, -p2, .. with p1 < p2 < .., kappa_2).  Plain enumeration."""
+    import itertools
+    cands = sorted({Fraction(a, b) for b in range(1, d_max + 1) for a in range(1, p_max * b + 1)})
+    pairs = n_finite // 2
+    best, best_k = None, None
+    for combo in itertools.combinations(cands, pairs):
+        pts = ([Fraction(0)] if n_finite % 2 else []) + [s * p for p in combo for s in (1, -1)]
+        k = kappa2(np.array([[float(a) ** j for j in range(n_finite)] for a in pts]))
+        if best is None or k < best_k:
+            best, best_k = pts, k
+    return best, best_k

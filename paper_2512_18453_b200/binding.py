@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
     "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
     "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
-    "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices",
+    "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices", "nova_symmetric_search",
     "nova_filter_transform_int8_bytes", "nova_filter_transform_int8", "nova_conv2d_int8_workspace_bytes",
     "nova_conv2d_fwd_int8", "nova_conv2d_fwd_int8_timed",
 )
@@ -62,6 +62,8 @@ def lib():
     L.nova_plan_create_f64.restype = i
     L.nova_snap_to_rational.argtypes = [ctypes.c_double, i, rp]
     L.nova_snap_to_rational.restype = i
+    L.nova_symmetric_search.argtypes = [i, i, i, rp, dp]
+    L.nova_symmetric_search.restype = i
     L.nova_verify_decomposition.argtypes = [i, i, i, rp, rp, rp]
     L.nova_verify_decomposition.restype = i
     L.nova_plan_get_matrices_rational.argtypes = [vp, rp, rp, rp]
@@ -155,6 +157,14 @@ def snap_to_rational(x, max_den=10):
     r = _Rat()
     _check(lib().nova_snap_to_rational(float(x), int(max_den), ctypes.byref(r)), "nova_snap_to_rational")
     return int(r.num), int(r.den)
+
+
+def symmetric_search(n_finite, max_den=6, max_abs=2):
+    """Best-conditioned symmetric point set on the snap grid: ([(num, den), .., (1, 0)], kappa_2)."""
+    pts = (_Rat * (n_finite + 1))()
+    k = ctypes.c_double()
+    _check(lib().nova_symmetric_search(n_finite, max_den, max_abs, pts, ctypes.byref(k)), "nova_symmetric_search")
+    return [(int(p.num), int(p.den)) for p in pts], k.value
 
 
 def verify_decomposition(m, r, AT, G, BT):

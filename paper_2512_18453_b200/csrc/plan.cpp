@@ -500,6 +500,61 @@ extern "C" int nova_snap_to_rational(double x, int max_den, nova_rat* out) {
   return NOVA_OK;
 }
 
+extern "C" int nova_symmetric_search(int n_finite, int max_den, int max_abs, nova_rat* points_out,
+                                     double* kappa2_out) {
+  if (!points_out || n_finite < 2 || n_finite >= nova::kMaxN || max_den < 1 || max_den > 64 || max_abs < 1 ||
+      max_abs > 5)
+    return NOVA_ERR_INVALID_ARG;
+  // candidates: the positive fractions a/b in lowest terms, b <= max_den, a/b <= max_abs, ascending
+  std::vector<std::pair<int, int>> cand;
+  for (int b = 1; b <= max_den; ++b)
+    for (int a = 1; a <= max_abs * b; ++a)
+      if (gcd128(a, b) == 1) cand.push_back({a, b});
+  std::sort(cand.begin(), cand.end(), [](const std::pair<int, int>& x, const std::pair<int, int>& y) {
+    return (long long)x.first * y.second < (long long)y.first * x.second;
+  });
+  const int pairs = n_finite / 2, nc = (int)cand.size();
+  if (pairs > nc) return NOVA_ERR_INVALID_ARG;
+  double combos = 1;
+  for (int i = 0; i < pairs; ++i) combos = combos * (nc - i) / (i + 1);
+  if (combos > 4e6) return NOVA_ERR_UNSUPPORTED;       // keep the enumeration to seconds
+  std::vector<int> idx(pairs), best_idx;
+  for (int i = 0; i < pairs; ++i) idx[i] = i;
+  double best = INFINITY;
+  std::vector<double> V(n_finite * n_finite), pts(n_finite);
+  for (;;) {
+    int k = 0;
+    if (n_finite & 1) pts[k++] = 0.0;
+    for (int i = 0; i < pairs; ++i) {
+      const double p = (double)cand[idx[i]].first / (double)cand[idx[i]].second;
+      pts[k++] = p;
+      pts[k++] = -p;
+    }
+    for (int i = 0; i < n_finite; ++i) {
+      double pw = 1.0;
+      for (int j = 0; j < n_finite; ++j) { V[i * n_finite + j] = pw; pw *= pts[i]; }
+    }
+    const double kap = cond2(V, n_finite);
+    if (kap < best) { best = kap; best_idx = idx; }
+    int i = pairs - 1;                                  // next combination in lexicographic order
+    while (i >= 0 && idx[i] == nc - pairs + i) --i;
+    if (i < 0) break;
+    ++idx[i];
+    for (int j = i + 1; j < pairs; ++j) idx[j] = idx[j - 1] + 1;
+  }
+  int k = 0;
+  if (n_finite & 1) { points_out[k].num = 0; points_out[k].den = 1; ++k; }
+  for (int i = 0; i < pairs; ++i) {
+    const std::pair<int, int>& c = cand[best_idx[i]];
+    points_out[k].num = c.first; points_out[k].den = c.second; ++k;
+    points_out[k].num = -c.first; points_out[k].den = c.second; ++k;
+  }
+  points_out[k].num = 1;
+  points_out[k].den = 0;                                // the point at infinity, last
+  if (kappa2_out) *kappa2_out = best;
+  return NOVA_OK;
+}
+
 extern "C" int nova_plan_create_f64(int m, int r, const double* finite_points, int n_finite, int max_den,
                                     int mode, int coef, nova_plan** out) {
   if (out) *out = nullptr;

@@ -204,3 +204,19 @@ def test_r5_rejects_what_it_cannot_build():
     with pytest.raises(nv.NovaError) as e:
         nv.Plan(4, point_set("std", 6), r=4)
     assert e.value.status == -7
+
+
+def test_symmetric_search_through_the_abi_finds_the_discovered_sets():
+    for m in (4, 6, 8):
+        pts, k = nv.symmetric_search(m + 1, 6, 2)
+        assert pts == point_set("nova", m)                       # Table 3, infinity last
+        assert abs(k / tc.kappa2_V(point_set("nova", m)) - 1) < 1e-9
+        plan = nv.Plan(m, pts)                                   # and the set builds a verified plan
+        assert abs(plan.kappa() / k - 1) < 1e-9
+    for n_finite, d in ((3, 6), (4, 5), (5, 8)):                 # same answer as the oracle's enumeration
+        pts, k = nv.symmetric_search(n_finite, d, 2)
+        opts, ok = tc.symmetric_search(n_finite, d)
+        assert [(p.numerator, p.denominator) for p in opts] == pts[:-1] and abs(k / ok - 1) < 1e-9
+    with pytest.raises(nv.NovaError) as e:                       # too many combinations to enumerate
+        nv.symmetric_search(9, 30, 5)
+    assert e.value.status == -7
