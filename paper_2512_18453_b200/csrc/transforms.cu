@@ -124,7 +124,7 @@ filter_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ 
 // (tile, channel pair) and one group of two B^T rows: it applies those two rows along the
 // patch's columns (nu), keeps the n x 2 intermediate in registers, applies all n rows along
 // the patch's rows (xi) and stores the 2n frequencies (xi, nu in its group).  The n/2 groups
-// of a patch sit in one block, so the patch is read from DRAM once and from L1 afterwards.
+// of a patch are rows of the grid: the patch comes from DRAM once and from L2 for the other groups.
 template <int M, typename T, bool SYM, int G, typename Sink, int R = 3>
 __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* __restrict__ x,
                                                       Sink& V, int H, int W, int C, int h0,
@@ -170,16 +170,20 @@ __device__ __forceinline__ void input_transform_group(const Coefs& cf, const T* 
 }
 
 template <int M, typename T, bool SYM, typename Sink, int R = 3>
-__global__ void __launch_bounds__(32 * (M + R - 1) * 2)
+__global__ void __launch_bounds__(128)
 input_transform_kernel(const __grid_constant__ Coefs cf, const T* __restrict__ x, Sink V,
                        int H, int W, int C, int Th, int Tw, long long p0, int pc, int pc_pad) {
   constexpr int N = M + R - 1;
   constexpr int PAD = (R - 1) / 2;
   constexpr int WORK = 128;                       // (tile, channel pair) items per block
   // threads [g*128, g*128+128) form group g (warp-uniform)
-  const int g = threadIdx.x / WORK;
+  // blockIdx.y is the group of B^T rows: every warp of a block - and, since blocks are handed out
+  // with x fastest, nearly every block resident at a time - runs the same unrolled code, which
+  // keeps it in the instruction cache (with all groups in one block the kernel spent most of its
+  // issue slots waiting for instructions).
+  const int g = blockIdx.y;
   const int c2 = C >> 1;
-  const long long idx = (long long)blockIdx.x * WORK + (threadIdx.x % WORK);
+  const long long idx = (long long)blockIdx.x * WORK + threadIdx.x;
   if (idx >= (long long)pc * c2) return;
   const int pl = (int)(idx / c2);
   const int c = (int)(idx % c2) * 2;
@@ -375,9 +379,9 @@ int filter_launch_int8(const nova_plan* plan, const void* g, int K, int C, void*
 template <int M, typename T>
 int input_launch_int8(const nova_plan* plan, const Geom& g, const void* x, void* Vq, float* slot, int pass,
                       long long p0, int pc, int pc_pad, cudaStream_t s) {
-  constexpr int THREADS = 32 * (M + 2) * 2;
+  constexpr int THREADS = 128;
   const long long work = (long long)pc * (g.C / 2);
-  const unsigned grid = blocks_for(work, 128);
+  const dim3 grid(blocks_for(work, 128), (M + 2) / 2);      // y: one block row per group of two B^T rows
 #define NOVA_IT8(SYMV, SINK, ...)                                                                         \
   input_transform_kernel<M, T, SYMV, SINK><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, __VA_ARGS__, g.H, \
                                                                    g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad)
@@ -394,16 +398,17 @@ int input_launch_int8(const nova_plan* plan, const Geom& g, const void* x, void*
 template <int M, typename T>
 int input_launch(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc,
                  int pc_pad, cudaStream_t s) {
-  constexpr int THREADS = 32 * (M + 2) * 2;       // n/2 groups of 128 work items
+  constexpr int THREADS = 128;
   const long long work = (long long)pc * (g.C / 2);
-  const unsigned grid = blocks_for(work, 128);
+  const dim3 grid(blocks_for(work, 128), (M + 2) / 2);      // y: one block row per group of two B^T rows
+  const dim3 grid5(blocks_for(work, 128), (M + 4) / 2);
   if (plan->r == 5) {                               // 5-tap filters: n = m + 4 points
     if constexpr (M <= 6) {
       if (plan->symmetric)
-        input_transform_kernel<M, T, true, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
+        input_transform_kernel<M, T, true, StoreSink<T>, 5><<<grid5, THREADS, 0, s>>>(
             plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
       else
-        input_transform_kernel<M, T, false, StoreSink<T>, 5><<<grid, 32 * (M + 4) * 2, 0, s>>>(
+        input_transform_kernel<M, T, false, StoreSink<T>, 5><<<grid5, THREADS, 0, s>>>(
             plan->kcoefs, (const T*)x, StoreSink<T>{(T*)V}, g.H, g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad);
     } else {
       return (int)cudaErrorInvalidValue;
