@@ -67,7 +67,7 @@ bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, i
   if (r > NB) r = NB;
   if (r < 2 && r < NB) return false;
   if (r < 1) return false;
-  if (r > 64) r = 64;
+  if (r > 8) r = 8;                                   // the rings stay inside the L2; longer ones were never validated
   *R = (int)r;
   return true;
 }

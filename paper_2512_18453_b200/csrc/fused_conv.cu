@@ -63,11 +63,14 @@ struct ConvShape {
 // ---------------------------------------------------------------- counters
 __device__ __forceinline__ bool ctr_wait(const uint32_t* ctr, uint32_t target, volatile int* abort_flag,
                                          const int* abort_all) {
+  const uint64_t t0 = global_ns();
   for (uint32_t i = 0; i < kCtrSpinLimit; ++i) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
     if (v >= target) return true;
-    if ((i & 31u) == 31u && (*abort_flag || *reinterpret_cast<const volatile int*>(abort_all))) return false;
+    if ((i & 31u) == 31u && (*abort_flag || *reinterpret_cast<const volatile int*>(abort_all) ||
+                             global_ns() - t0 > kWaitLimitNs))
+      return false;
     __nanosleep(64);
   }
   return false;

@@ -9,6 +9,7 @@ namespace nova {
 namespace sm100 {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // two seconds: far beyond any healthy wait of these kernels
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -47,12 +48,20 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the limit is hit or another role gave up.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kWaitLimitNs of wall time (a probe may suspend the thread for a
+// hardware-defined time, so a count of probes alone bounds nothing useful) or when another
+// role has given up.  Returns false in both cases.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_test(bar, parity)) return true;      // the common case in a full pipeline: no suspend
+  const uint64_t t0 = global_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
     if (mbar_try(bar, parity)) return true;
-    if ((spin & 15u) == 15u && *abort_flag) return false;
+    if ((spin & 15u) == 15u && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) return false;
   }
   return false;
 }
