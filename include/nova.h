@@ -326,6 +326,17 @@ int nova_conv2d_fwd_int8_timed(const nova_plan* plan, const void* x_dev, const v
                                void* workspace_dev, size_t workspace_bytes, int flags, nova_stream stream,
                                float* ms_host);
 
+/*
+ * Self-test of the failure reporting (no counterpart in the paper).  Every wait inside the
+ * kernels is bounded by the clock; when one expires the kernel records NOVA_ERR_DEVICE_TIMEOUT in
+ * the plan's status word and returns normally.  This call launches one warp that waits, with a
+ * limit of limit_ms (1..1000) milliseconds, on a barrier that nothing completes, so that the path
+ * from an expired wait to nova_last_device_status can be exercised on a healthy GPU.
+ * *waited_ns_host receives the time the warp waited.  Synchronises `stream`; allocates one word.
+ */
+int nova_selftest_wait_timeout(const nova_plan* plan, unsigned limit_ms, unsigned long long* waited_ns_host,
+                               nova_stream stream);
+
 /* 2x2 max pooling, stride 2, NHWC, H and W even, C % 8 == 0 (used between the
  * blocks of a VGG-style stack; not part of the paper's method).  `mode`
  * selects half or float elements. */

@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = (
     "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
     "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
     "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices", "nova_symmetric_search",
+    "nova_selftest_wait_timeout",
     "nova_filter_transform_int8_bytes", "nova_filter_transform_int8", "nova_conv2d_int8_workspace_bytes",
     "nova_conv2d_fwd_int8", "nova_conv2d_fwd_int8_timed",
 )
@@ -62,6 +63,8 @@ def lib():
     L.nova_plan_create_f64.restype = i
     L.nova_snap_to_rational.argtypes = [ctypes.c_double, i, rp]
     L.nova_snap_to_rational.restype = i
+    L.nova_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint, ctypes.POINTER(ctypes.c_ulonglong), vp]
+    L.nova_selftest_wait_timeout.restype = i
     L.nova_symmetric_search.argtypes = [i, i, i, rp, dp]
     L.nova_symmetric_search.restype = i
     L.nova_verify_decomposition.argtypes = [i, i, i, rp, rp, rp]
@@ -380,6 +383,14 @@ class Plan:
             return y, list(ms)
         _check(lib().nova_conv2d_fwd_int8(*args), "nova_conv2d_fwd_int8")
         return y
+
+    def selftest_wait_timeout(self, limit_ms=50):
+        """Let one warp's bounded wait expire after limit_ms; returns the nanoseconds it waited.
+        device_status() then reports (and clears) the time-out."""
+        w = ctypes.c_ulonglong()
+        _check(lib().nova_selftest_wait_timeout(self._h, int(limit_ms), ctypes.byref(w), _stream()),
+               "nova_selftest_wait_timeout")
+        return int(w.value)
 
     def device_status(self):
         return lib().nova_last_device_status(self._h, _stream())

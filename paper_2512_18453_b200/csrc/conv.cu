@@ -9,6 +9,7 @@
 #include <mutex>
 
 #include "nova_internal.h"
+#include "sm100.cuh"
 
 namespace nova {
 namespace {
@@ -470,6 +471,45 @@ extern "C" int nova_conv2d_fwd_int8_timed(const nova_plan* p, const void* x, con
     cudaEventElapsedTime(&ms[3], ev[0], ev[3]);
   }
   for (auto& e : ev) cudaEventDestroy(e);
+  return st;
+}
+
+// ---------------------------------------------------------------------------
+// Self-test of the failure reporting: one warp waits on an mbarrier phase that nothing completes,
+// with the same bounded wait the kernels use but a caller-chosen limit, and reports the expiry
+// through the plan's status word.  The wait ends by the clock; nothing faults or hangs.
+namespace nova {
+static __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns, unsigned long long* waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    sm100::mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const uint64_t t0 = sm100::global_ns();
+  const bool ok = sm100::mbar_wait_limited(&bar, 0, &abort_flag, limit_ns, 1u << 16);
+  if (threadIdx.x == 0) {
+    *waited_ns = sm100::global_ns() - t0;
+    if (!ok) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+  }
+}
+}  // namespace nova
+
+extern "C" int nova_selftest_wait_timeout(const nova_plan* p, unsigned limit_ms, unsigned long long* waited_ns_host,
+                                          nova_stream stream) {
+  if (!p || !waited_ns_host || limit_ms < 1 || limit_ms > 1000) return NOVA_ERR_INVALID_ARG;
+  if (!p->status_dev) return NOVA_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned long long* w = nullptr;
+  if (cudaMalloc((void**)&w, sizeof(*w)) != cudaSuccess) return NOVA_ERR_CUDA;
+  wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(p->status_dev, (unsigned long long)limit_ms * 1000000ull, w);
+  int st = cudaGetLastError() == cudaSuccess ? NOVA_OK : NOVA_ERR_CUDA;
+  if (st == NOVA_OK && (cudaMemcpyAsync(waited_ns_host, w, sizeof(*w), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                        cudaStreamSynchronize(s) != cudaSuccess))
+    st = NOVA_ERR_CUDA;
+  cudaFree(w);
   return st;
 }
 

@@ -56,14 +56,18 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait: gives up after kWaitLimitNs of wall time (a probe may suspend the thread for a
 // hardware-defined time, so a count of probes alone bounds nothing useful) or when another
 // role has given up.  Returns false in both cases.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  uint64_t limit_ns, uint32_t max_probes) {
   if (mbar_test(bar, parity)) return true;      // the common case in a full pipeline: no suspend
   const uint64_t t0 = global_ns();
-  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+  for (uint32_t spin = 0; spin < max_probes; ++spin) {
     if (mbar_try(bar, parity)) return true;
-    if ((spin & 15u) == 15u && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) return false;
+    if ((spin & 15u) == 15u && (*abort_flag || global_ns() - t0 > limit_ns)) return false;
   }
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limited(bar, parity, abort_flag, kWaitLimitNs, kSpinLimit);
 }
 // The same wait for a whole (converged) warp.  Every lane probes the barrier itself: a
 // satisfied wait is one test_wait, a few cycles; there is no broadcast from an elected lane.

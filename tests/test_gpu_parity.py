@@ -734,3 +734,18 @@ def test_cfg3_full_size_int8_sampled_against_the_oracle():
     e_gpu, e_emu = conv.rel_l2(y[pick], y1), conv.rel_l2(ye, y1)
     assert (e_gpu <= 2.0 * e_emu) if e_emu < 1.0 else (e_gpu >= 0.5), (e_gpu, e_emu)
     assert conv.rel_l2(y[pick], ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable():
+    # a bounded wait that nothing satisfies runs out by the clock; the status word carries the
+    # time-out to the host, reading it clears it, and the next convolution works as usual
+    x, g = make_conv_inputs(1, 12, 12, 64, 64, "fp16", seed=99)
+    pts = point_set("nova", 4)
+    plan = nv.Plan(4, pts)
+    assert plan.device_status() == 0
+    waited = plan.selftest_wait_timeout(50)
+    assert 50e6 <= waited <= 1.5e9
+    assert plan.device_status() == -9
+    assert plan.device_status() == 0
+    y, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC)
+    check_fp16(y, x, g, 4, pts)
