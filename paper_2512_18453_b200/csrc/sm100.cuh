@@ -59,10 +59,15 @@ __device__ __forceinline__ uint64_t global_ns() {
 __device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                   uint64_t limit_ns, uint32_t max_probes) {
   if (mbar_test(bar, parity)) return true;      // the common case in a full pipeline: no suspend
-  const uint64_t t0 = global_ns();
+  uint64_t t0 = 0;                              // the clock is read only once a wait turns out long
   for (uint32_t spin = 0; spin < max_probes; ++spin) {
     if (mbar_try(bar, parity)) return true;
-    if ((spin & 15u) == 15u && (*abort_flag || global_ns() - t0 > limit_ns)) return false;
+    if ((spin & 15u) == 15u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) return false;
+    }
   }
   return false;
 }
