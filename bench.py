@@ -337,6 +337,18 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     status = plan.device_status()
 
+    # ---- spread of single steps: 100 steps timed one by one (an event pair each), median and minimum
+    n_single = min(100, args.steps)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_single)]
+    for i, (a0, a1) in enumerate(evs):
+        a0.record()
+        step(i)
+        a1.record()
+    torch.cuda.synchronize()
+    singles = sorted(a0.elapsed_time(a1) for a0, a1 in evs)
+    step_stats = {"n": n_single, "median_us": 1e3 * singles[len(singles) // 2], "min_us": 1e3 * singles[0],
+                  "note": "single steps between their own event pairs; the headline ms_per_step is the mean of the back-to-back run"}
+
     # ---- per-kernel durations (events around each kernel, same steps, separate pass)
     kms = [0.0, 0.0, 0.0]
     prof_steps = min(args.steps, 20)
@@ -416,6 +428,7 @@ def run_ours(args):
                           "tensor_us": actual / (peaks["tflops_burst"] * 1e12) * 1e6,
                           "hbm_us": min_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
         "kernels_ms_per_step": {n_: v for n_, v in zip(names, kms) if n_ != "-"},
+        "single_step": step_stats,
         "filter_transform_ms": filter_ms,
         "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"],
