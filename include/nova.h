@@ -96,9 +96,9 @@ typedef void* nova_stream;            /* a cudaStream_t */
  * exactly zero, and the tables are then rounded (rational -> double -> float
  * or half, round to nearest even).  Host only: works without a CUDA device.
  * r = 3 plans have every kernel.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
- * extension; g is then [K,5,5,C] and the padding 2) runs nova_filter_transform and
- * nova_conv2d_fwd with the same kernels instantiated for n = m + 4; the INT8 entry points and the NOVA_FUSED* flags are for r = 3
- * (NOVA_ERR_UNSUPPORTED / ignored).
+ * extension; g is then [K,5,5,C] and the padding 2) runs the filter transforms and the
+ * convolutions, INT8 pipeline included, with the same kernels instantiated for n = m + 4;
+ * the NOVA_FUSED* flags are ignored for such plans.
  * On success *out must be released with nova_plan_destroy.
  */
 int nova_plan_create(int m, int r, const nova_rat* points_host, int n,
@@ -295,7 +295,8 @@ int nova_conv2d_launch_count(const nova_plan* plan, int N, int H, int W, int C, 
  * the product over the input
  * channels is exact int32 arithmetic on the tensor cores (tcgen05 kind::i8), and the output
  * transform runs in float on float(M) * (s_U[k] * s_V), rounded once to half.  x, g and y are
- * half tensors as in nova_conv2d_fwd.  C and K must be multiples of 16.
+ * half tensors as in nova_conv2d_fwd (g is [K,5,5,C] for a plan with r = 5).  C and K must be
+ * multiples of 16.
  *
  * nova_filter_transform_int8: g [K,3,3,C] half -> Uq (nova_filter_transform_int8_bytes() bytes,
  * opaque layout) and scale_U_dev[K] floats (device).  quant: one of NOVA_QUANT_*.

@@ -258,7 +258,8 @@ def winograd_conv_int8_emulated(x, g, m, points, per_channel=False, scale_U=None
     converted to float32, multiplied by the float32 product s_U[k] * s_V, and the output
     transform is evaluated in float32 and rounded once to float16.
     """
-    AT, G, BT = coefficient_tables(m, points, "fp16", coef, scales)
+    r = np.asarray(g).shape[1]
+    AT, G, BT = coefficient_tables(m, points, "fp16", coef, scales, r=r)
     x = np.asarray(x)
     N, H, W, C = x.shape
     with np.errstate(all="ignore"):
@@ -271,13 +272,13 @@ def winograd_conv_int8_emulated(x, g, m, points, per_channel=False, scale_U=None
             sU = np.broadcast_to(np.asarray(scale_U, dtype=np.float32), (K,)).copy()
         sU = np.where(sU == 0, np.float32(1), sU).astype(np.float32)
         Uq = quantize_int8(U, sU[:, None, None, None])
-        d = _gather_tiles(x.astype(np.float32), m)
+        d = _gather_tiles(x.astype(np.float32), m, r)
         V = _two_sided(BT, d, (3, 4), np.float32)                              # [N,Th,Tw,n,n,C]
         sV = int8_scale(np.abs(V).max()) if scale_V is None else np.float32(scale_V)
         if sV == 0:
             sV = np.float32(1)
         Vq = quantize_int8(V, sV)
-        n = m + 2
+        n = m + r - 1
         Th, Tw = d.shape[1], d.shape[2]
         Mi = np.empty((N, Th, Tw, n, n, K), dtype=np.int64)
         for p in range(n):

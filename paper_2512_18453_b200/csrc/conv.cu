@@ -48,9 +48,8 @@ bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* 
 }
 
 // 3 x 3 filters have every kernel; 5 x 5 filters (F(2,5), F(4,5), F(6,5)) run the CUDA-core
-// transforms around the tensor-core product.  The INT8 and the fused paths are 3 x 3 only.
+// same kernels instantiated for n = m + 4.  The fused paths are 3 x 3 only.
 bool device_plan(const nova_plan* p) { return p && (p->r == kR || p->r == 5); }
-bool device_plan_r3(const nova_plan* p) { return p && p->r == kR; }
 bool shape_ok(int N, int H, int W, int C, int K) {
   return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
 }
@@ -365,7 +364,7 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
 // INT8 Winograd-domain pipeline.
 namespace {
 bool int8_shape_ok(const nova_plan* p, int N, int H, int W, int C, int K) {
-  return device_plan_r3(p) && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
+  return device_plan(p) && p->mode == NOVA_FP16_F32ACC && shape_ok(N, H, W, C, K) && (C % 16) == 0 && (K % 16) == 0;
 }
 struct Int8Layout {
   int pad;                  // tiles rounded up to whole 128-row blocks
@@ -385,7 +384,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
                      nova_stream stream, cudaEvent_t* ev) {
   if (!int8_shape_ok(p, N, H, W, C, K) || !aligned16(x) || !aligned16(Uq) || !aligned16(y) || !scale_U ||
       !(scale_V >= 0.f))
-    return p && (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
+    return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if (!p->status_dev) return NOVA_ERR_CUDA;
   const Geom g = make_geom(p, N, H, W, C, K);
@@ -429,18 +428,18 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
 }  // namespace
 
 extern "C" size_t nova_filter_transform_int8_bytes(const nova_plan* p, int K, int C) {
-  if (!device_plan_r3(p) || K <= 0 || C <= 0) return 0;
+  if (!device_plan(p) || K <= 0 || C <= 0) return 0;
   return (size_t)p->n * p->n * K * C;
 }
 
 extern "C" int nova_filter_transform_int8(const nova_plan* p, const void* g, int K, int C, int quant, void* Uq,
                                           float* scale_U, nova_stream stream) {
-  if (p && (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p))) return NOVA_ERR_UNSUPPORTED;
+  if (p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p))) return NOVA_ERR_UNSUPPORTED;
   if (!p || !aligned16(g) || !aligned16(Uq) || !scale_U || K <= 0 || C <= 0 || (K % 16) || (C % 16))
     return NOVA_ERR_INVALID_ARG;
   if (quant != NOVA_QUANT_PER_TENSOR && quant != NOVA_QUANT_PER_CHANNEL && quant != NOVA_QUANT_GIVEN)
     return NOVA_ERR_INVALID_ARG;
-  if (p->mode != NOVA_FP16_F32ACC || !device_plan_r3(p)) return NOVA_ERR_UNSUPPORTED;
+  if (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   const int e = launch_filter_transform_int8(p, g, K, C, Uq, scale_U, quant, stream);
   if (e) g_last_cuda_error = e;
   return e ? NOVA_ERR_CUDA : NOVA_OK;

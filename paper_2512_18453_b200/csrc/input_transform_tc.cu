@@ -404,6 +404,18 @@ int launch_input_transform_tc_int8(const nova_plan* plan, const Geom& g, const v
 #define NOVA_TC8(MM) \
   return pass == 0 ? launch_m<MM, 1>(plan, g, x, Vq, p0, pc, pc_pad, slot, s) \
                    : launch_m<MM, 2>(plan, g, x, Vq, p0, pc, pc_pad, slot, s)
+  if (plan->r == 5) {
+#define NOVA_TC8R5(MM) \
+  return pass == 0 ? launch_m<MM, 1, 5>(plan, g, x, Vq, p0, pc, pc_pad, slot, s) \
+                   : launch_m<MM, 2, 5>(plan, g, x, Vq, p0, pc, pc_pad, slot, s)
+    switch (plan->m) {
+      case 2: NOVA_TC8R5(2);
+      case 4: NOVA_TC8R5(4);
+      case 6: NOVA_TC8R5(6);
+    }
+#undef NOVA_TC8R5
+    return (int)cudaErrorInvalidValue;
+  }
   switch (plan->m) {
     case 2: NOVA_TC8(2);
     case 4: NOVA_TC8(4);

@@ -193,8 +193,11 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
     return (int)cudaErrorUnknown;
   const bool f32 = plan->mode == NOVA_FP32;
 #define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q, R>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
-  if constexpr (R != 3) {                             // 5-tap filters: no int8 pipeline
-    if (scale_U) return (int)cudaErrorInvalidValue;
+  if constexpr (R != 3) {                             // 5-tap filters
+    if (scale_U) {
+      if (f32) return (int)cudaErrorInvalidValue;
+      return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
+    }
     if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
     return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
   } else {

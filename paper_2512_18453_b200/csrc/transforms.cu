@@ -363,15 +363,27 @@ int filter_launch_int8(const nova_plan* plan, const void* g, int K, int C, void*
                        cudaStream_t s) {
   const long long work = (long long)K * (C / 2);
   const int per_channel = (quant & NOVA_QUANT_PER_CHANNEL) ? 1 : 0;
+  const bool r5 = plan->r == 5;
+  if (r5 && M > 6) return (int)cudaErrorInvalidValue;
   if (!(quant & NOVA_QUANT_GIVEN)) {
     cudaError_t e = cudaMemsetAsync(scales, 0, sizeof(float) * K, s);
     if (e != cudaSuccess) return (int)e;
-    filter_transform_kernel<M, T, AbsmaxSink><<<blocks_for(work, 256), 256, 0, s>>>(
-        plan->kcoefs, (const T*)g, AbsmaxSink{(unsigned*)scales, per_channel, 0.f, nullptr}, K, C);
+    const AbsmaxSink sink{(unsigned*)scales, per_channel, 0.f, nullptr};
+    if (r5) {
+      if constexpr (M <= 6)
+        filter_transform_kernel<M, T, AbsmaxSink, 5><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, sink, K, C);
+    } else {
+      filter_transform_kernel<M, T, AbsmaxSink><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, sink, K, C);
+    }
     scales_from_absmax_kernel<<<1, 256, 0, s>>>(scales, K, per_channel);
   }
-  filter_transform_kernel<M, T, QuantSink><<<blocks_for(work, 256), 256, 0, s>>>(
-      plan->kcoefs, (const T*)g, QuantSink{(int8_t*)Uq, scales, 1, 0.f}, K, C);
+  const QuantSink qsink{(int8_t*)Uq, scales, 1, 0.f};
+  if (r5) {
+    if constexpr (M <= 6)
+      filter_transform_kernel<M, T, QuantSink, 5><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, qsink, K, C);
+  } else {
+    filter_transform_kernel<M, T, QuantSink><<<blocks_for(work, 256), 256, 0, s>>>(plan->kcoefs, (const T*)g, qsink, K, C);
+  }
   return (int)cudaGetLastError();
 }
 // int8 input transform over tiles p0 .. p0+pc-1.  pass 0: absmax into *slot (zeroed by the caller);
@@ -385,6 +397,24 @@ int input_launch_int8(const nova_plan* plan, const Geom& g, const void* x, void*
 #define NOVA_IT8(SYMV, SINK, ...)                                                                         \
   input_transform_kernel<M, T, SYMV, SINK><<<grid, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, __VA_ARGS__, g.H, \
                                                                    g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad)
+#define NOVA_IT8R5(SYMV, SINK, ...)                                                                       \
+  input_transform_kernel<M, T, SYMV, SINK, 5><<<grid5, THREADS, 0, s>>>(plan->kcoefs, (const T*)x, __VA_ARGS__, g.H, \
+                                                                       g.W, g.C, g.Th, g.Tw, p0, pc, pc_pad)
+  if (plan->r == 5) {
+    if constexpr (M <= 6) {
+      const dim3 grid5(blocks_for(work, 128), (M + 4) / 2);
+      if (pass == 0) {
+        if (plan->symmetric) NOVA_IT8R5(true, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
+        else NOVA_IT8R5(false, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
+      } else {
+        if (plan->symmetric) NOVA_IT8R5(true, QuantSink, QuantSink{(int8_t*)Vq, slot, 0, 0.f});
+        else NOVA_IT8R5(false, QuantSink, QuantSink{(int8_t*)Vq, slot, 0, 0.f});
+      }
+      return (int)cudaGetLastError();
+    } else {
+      return (int)cudaErrorInvalidValue;
+    }
+  }
   if (pass == 0) {
     if (plan->symmetric) NOVA_IT8(true, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
     else NOVA_IT8(false, AbsmaxSink, AbsmaxSink{(unsigned*)slot, 0, 0.f, nullptr});
@@ -393,6 +423,7 @@ int input_launch_int8(const nova_plan* plan, const Geom& g, const void* x, void*
     else NOVA_IT8(false, QuantSink, QuantSink{(int8_t*)Vq, slot, 0, 0.f});
   }
 #undef NOVA_IT8
+#undef NOVA_IT8R5
   return (int)cudaGetLastError();
 }
 template <int M, typename T>

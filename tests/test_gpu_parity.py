@@ -672,7 +672,7 @@ def test_r5_fp16_mode_within_twice_the_emulation(m, key, shape, flags):
     assert (d <= ulp).all() and (d > 0).mean() < 0.05
 
 
-def test_r5_chunked_relu_static_and_refusals():
+def test_r5_chunked_relu_and_static():
     x, g = make_conv_inputs(3, 26, 22, 64, 64, "fp16", seed=720, r=5)
     pts = point_set("nova", 6)
     a, _ = gpu_conv_r5(x, g, 4, pts, nv.FP16_F32ACC)
@@ -687,9 +687,6 @@ def test_r5_chunked_relu_static_and_refusals():
     plan.conv2d_static(xd, U, ys)
     torch.cuda.synchronize()
     assert np.array_equal(ys.cpu().numpy().view(np.uint16), a.view(np.uint16))
-    with pytest.raises(nv.NovaError) as e:
-        plan.filter_transform_int8(torch.zeros((16, 3, 3, 16), dtype=torch.float16, device="cuda"))
-    assert e.value.status == -7
 
 
 @pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("nova", 6)), (6, ("nova", 8))])
@@ -749,3 +746,32 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
     assert plan.device_status() == 0
     y, _, _ = gpu_conv(x, g, 4, pts, nv.FP16_F32ACC)
     check_fp16(y, x, g, 4, pts)
+
+
+@pytest.mark.parametrize("m,key", [(2, ("std", 4)), (4, ("nova", 6)), (4, ("half", 6)), (6, ("nova", 8))])
+@pytest.mark.parametrize("shape,coef", [((2, 13, 11, 16, 16), nv.COEF_FP32), ((2, 30, 30, 64, 80), nv.COEF_ROUND_TO_MODE),
+                                        ((1, 17, 23, 144, 272), nv.COEF_ROUND_TO_MODE)])
+def test_r5_int8_path_matches_the_emulation(m, key, shape, coef):
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", seed=800 + m, r=5)
+    pts = point_set(*key)
+    plan = nv.Plan(m, pts, nv.FP16_F32ACC, coef, r=5)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    Uq, sU = plan.filter_transform_int8(gd, nv.QUANT_PER_CHANNEL)
+    y = plan.conv2d_int8(xd, Uq, sU)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    y = y.cpu().numpy()
+    ye, parts = conv.winograd_conv_int8_emulated(x, g, m, pts, per_channel=True,
+                                                 coef="fp32" if coef == nv.COEF_FP32 else "mode", return_parts=True)
+    np.testing.assert_allclose(sU.cpu().numpy(), parts["scale_U"], rtol=2e-6)
+    n = m + 4
+    dU = np.abs(Uq.cpu().numpy().astype(np.int32) - parts["Uq"].transpose(1, 2, 0, 3).reshape(n * n, K, C).astype(np.int32))
+    assert dU.max() <= 1 and (dU > 0).mean() < 2e-3
+    y1 = conv.direct_conv_fp64(x, g)
+    e_gpu, e_emu = conv.rel_l2(y, y1), conv.rel_l2(ye, y1)
+    if not np.isfinite(e_emu) or e_emu >= 1.0:
+        assert (not np.isfinite(e_gpu)) or e_gpu >= 0.5, (e_gpu, e_emu)
+    else:
+        assert e_gpu <= 2.0 * e_emu, (e_gpu, e_emu)
+        assert conv.rel_l2(y, ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3

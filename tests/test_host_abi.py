@@ -187,10 +187,10 @@ def test_r5_plans_are_exact(m, key):
     kap, _ = plan.kappa_matrices()
     for got, M in zip(kap, tc.build_matrices(m, 5, pts)):
         assert abs(got / tc.kappa2(tc.to_float(M)) - 1) < 1e-8
-    # sizes follow n = m + 4; the INT8 entry points are for 3 x 3 filters only
+    # sizes follow n = m + 4
     assert plan.filter_transform_bytes(64, 64) == (m + 4) ** 2 * 64 * 64 * 2
     assert plan.workspace_bytes(1, 16, 16, 64, 64) > 0
-    assert plan.int8_workspace_bytes(1, 16, 16, 64, 64) == 0
+    assert plan.int8_workspace_bytes(1, 16, 16, 64, 64) > 0
     assert plan.frequency_order() == (list(range(m + 4)), True)       # symmetric set already in internal order
     a16, g16, b16 = plan.device_tables()
     with np.errstate(over="ignore"):
