@@ -472,14 +472,19 @@ def run_int8(args):
     if args.images:
         import dataclasses
         c = dataclasses.replace(c, N=args.images, name="%s[N=%d]" % (c.name, args.images))
+    n_points = c.m + 2
+    if FILTER_R == 5:                                # same number of points, tile smaller by two
+        import dataclasses
+        c = dataclasses.replace(c, m=c.m - 2, name="%s[5x5,F(%d,5)]" % (c.name, c.m - 2))
     direct, actual, _, P = flops(c)
-    n2 = (c.m + 2) ** 2
+    n2 = n_points ** 2
     min_bytes = 2.0 * c.N * c.H * c.W * (c.C + c.K) + 1.0 * n2 * c.K * c.C
-    pts = point_set(args.points, c.m)
+    pts = point_set(args.points, n_points - 2)
     coef = nv.COEF_FP32 if args.int8_coef == "fp32" else nv.COEF_ROUND_TO_MODE
-    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef)
+    plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef, r=FILTER_R)
     quant = nv.QUANT_PER_CHANNEL if args.int8_quant == "per_channel" else nv.QUANT_PER_TENSOR
-    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, rank_seed(c.seed, rank))
+    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, rank_seed(c.seed, rank),
+                                  r=FILTER_R)
     g = torch.from_numpy(g_np).cuda()
     n_sets = 3
     xs = [torch.from_numpy(np.roll(x_np, i, axis=0)).cuda() for i in range(n_sets)]
@@ -595,8 +600,8 @@ def run_int8(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8 (s32 accumulate)",
         "data": "synthetic",
         "config": {
-            "workload": "%s: F(%dx%d,3x3) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
-                        % (c.name, c.m, c.m, args.points, c.N, c.C, c.K, c.H),
+            "workload": "%s: F(%dx%d,%dx%d) %s points, N=%d C=%d K=%d H=W=%d per GPU, NHWC, ReLU'd N(0,1) x He-normal"
+                        % (c.name, c.m, c.m, FILTER_R, FILTER_R, args.points, c.N, c.C, c.K, c.H),
             "step": "nova_conv2d_fwd_int8 (%s scale of U, %s scale of V, %s coefficient tables)"
                     % (args.int8_quant, "static" if scale_V > 0 else "data-derived", args.int8_coef),
             "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 126 MB L2)"
@@ -630,15 +635,15 @@ def accuracy_report_int8(c, nv, torch, coef, coef_name, n_img=2):
     import numpy as np
     from oracle import conv
     from synth import make_conv_inputs, point_set, pow2_range_scales
-    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    x, g = make_conv_inputs(n_img, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed, r=FILTER_R)
     y1 = conv.direct_conv_fp64(x, g)
     xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
     rep = {}
     for kind in c.point_kinds:
-        pts = point_set(kind, c.m)
-        _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC).matrices()
+        pts = point_set(kind, c.m + FILTER_R - 3)
+        _, G, BT = nv.Plan(c.m, pts, nv.FP16_F32ACC, r=FILTER_R).matrices()
         for label, sc in ((kind, (None, None)), (kind + "+pow2_rows", pow2_range_scales(G, BT))):
-            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef, scale_G=sc[0], scale_B=sc[1])
+            plan = nv.Plan(c.m, pts, nv.FP16_F32ACC, coef, r=FILTER_R, scale_G=sc[0], scale_B=sc[1])
             for qname, quant in (("per_tensor", nv.QUANT_PER_TENSOR), ("per_channel", nv.QUANT_PER_CHANNEL)):
                 Uq, sU = plan.filter_transform_int8(gd, quant)
                 y = plan.conv2d_int8(xd, Uq, sU, 0.0)
