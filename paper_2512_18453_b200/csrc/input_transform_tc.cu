@@ -240,13 +240,12 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
 #pragma unroll
           for (int cc = 0; cc < kMaxCols; cc += 4)
             if (col0 + cc < Cfg::NF) {
-              uint32_t w = 0;
+              uint32_t q[4];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                int q;
-                asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(q) : "f"(__fmul_rn(__uint_as_float(r[cc + j]), qs)));
-                w |= (uint32_t)(q & 0xff) << (8 * j);
-              }
+              for (int j = 0; j < 4; ++j)
+                asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(q[j]) : "f"(__fmul_rn(__uint_as_float(r[cc + j]), qs)));
+              // the low bytes of the four codes, packed with three byte permutations
+              const uint32_t w = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
               const uint32_t p1 = __shfl_xor_sync(0xffffffffu, w, 1);
               const uint32_t t = __byte_perm(w, p1, (li & 1) ? 0x3715 : 0x6240);
               const uint32_t p2 = __shfl_xor_sync(0xffffffffu, t, 2);
