@@ -177,46 +177,60 @@ def coefficient_tables(m, points, mode, coef="mode", scales=(None, None), r=3):
     return out  # AT, G, BT
 
 
+def _stage_dtypes(mode):
+    """(storage dtype of U, V and y; dtype the sums are evaluated in) for an arithmetic mode.
+
+    "fp16": binary16 storage, sums in float32 (Section 5.1 "FP16 Setup": transforms computed
+    in FP32 and cast to FP16; Section C.3: intermediates float32).  "fp32": float32 storage;
+    every stored element is ONE rounding of a sum carried in float64, so that what the mode
+    loses is the float32 storage of U, V, M and y and nothing else.  The paper only names the
+    mode ("FP32 baseline", Section 5.1); this reading is the one under which the F(8,3) tile with
+    well-conditioned points stays below a relative error of 1e-4 (sums carried in float32 sit at
+    1.2e-4 .. 1.7e-4 for that tile)."""
+    if mode == "fp16":
+        return np.float16, np.float32
+    return np.float32, np.float64
+
+
 def filter_transform_emulated(g, m, points, mode, coef="mode", scales=(None, None)):
-    """U[K,n,n,C]: fp32-evaluated G g G^T, rounded once to the operand dtype."""
+    """U[K,n,n,C]: G g G^T evaluated in the mode's sum precision, rounded once to the operand dtype."""
     _, G, _ = coefficient_tables(m, points, mode, coef, scales, r=np.asarray(g).shape[1])
+    st, ev = _stage_dtypes(mode)
     with np.errstate(all="ignore"):
-        U = _two_sided(G, np.asarray(g), (1, 2), np.float32)
-        if mode == "fp16":
-            U = U.astype(np.float16)
+        U = _two_sided(G, np.asarray(g), (1, 2), ev).astype(st)
     return U
 
 
 def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False, scales=(None, None)):
     """The four steps with the pipeline's rounding points:
 
-    tables rounded as in coefficient_tables; U and V evaluated in float32 and
-    rounded once to the operand dtype (float16 in mode "fp16"); the product
-    summed over channels in float32 (products of two float16 values are exact
-    in float32); the output transform evaluated in float32 and rounded once to
-    the storage dtype.  Mode "fp32" keeps every stage in float32.  Non-finite
-    values propagate (Section C.4 "Saturation").
+    tables rounded as in coefficient_tables; U and V evaluated in the mode's sum precision
+    (float32 in mode "fp16") and rounded once to the operand dtype (float16); the product summed
+    over channels in float32 (products of two float16 values are exact in float32) and stored as
+    float32; the output transform evaluated in the sum precision and rounded once to the
+    storage dtype.  Mode "fp32" stores U, V, M and y in float32 and carries every sum in float64
+    (see _stage_dtypes).  Non-finite values propagate (Section C.4 "Saturation").
     """
     r = np.asarray(g).shape[1]
     AT, G, BT = coefficient_tables(m, points, mode, coef, scales, r=r)
     x = np.asarray(x)
     N, H, W, C = x.shape
-    st = np.float16 if mode == "fp16" else np.float32
+    st, ev = _stage_dtypes(mode)
     with np.errstate(all="ignore"):
-        U = _two_sided(G, np.asarray(g), (1, 2), np.float32).astype(st).astype(np.float32)
-        d = _gather_tiles(x.astype(np.float32), m, r)
-        V = _two_sided(BT, d, (3, 4), np.float32).astype(st).astype(np.float32)
+        U = _two_sided(G, np.asarray(g), (1, 2), ev).astype(st).astype(ev)
+        d = _gather_tiles(x.astype(ev), m, r)
+        V = _two_sided(BT, d, (3, 4), ev).astype(st).astype(ev)
         n = m + r - 1
         Th, Tw = d.shape[1], d.shape[2]
         K = U.shape[0]
         M = np.empty((N, Th, Tw, n, n, K), dtype=np.float32)
         for p in range(n):
             for q in range(n):
-                M[:, :, :, p, q, :] = V[:, :, :, p, q, :] @ U[:, p, q, :].T
-        Y = _two_sided(AT, M, (3, 4), np.float32)
+                M[:, :, :, p, q, :] = V[:, :, :, p, q, :] @ U[:, p, q, :].T     # summed in ev, stored float32
+        Y = _two_sided(AT, M, (3, 4), ev)
         y = _scatter_tiles(Y, H, W)
         if apply_relu:
-            y = np.where(y < 0, np.float32(0), y)   # negative -> 0; NaN and +inf pass through
+            y = np.where(y < 0, ev(0), y)   # negative -> 0; NaN and +inf pass through
         y = y.astype(st)
     return y
 
@@ -226,16 +240,14 @@ def winograd_conv_emulated(x, g, m, points, mode, coef="mode", apply_relu=False,
 # Validation"; Section "Rational Coefficients in Practice")
 # --------------------------------------------------------------------------
 def quantize_int8(v, scale):
-    """Symmetric quantiser: round(v / scale) to nearest, ties to even, saturated to [-128, 127].
-    As is customary in quantised inference the division is carried out as one float32
-    multiplication by the reciprocal scale r = 1 / scale, itself one float32 division per scale
-    (the decision is taken in float32).  scale may be an array broadcastable against v; a zero
-    scale (an all-zero tensor) is treated as 1."""
+    """Symmetric quantiser: round(v / scale) to nearest, ties to even, saturated to [-128, 127]
+    (Section 5.1 "INT8 Setup": s = max|.|/127; the plain definition).  The quotient is one float32
+    division and the rounding decision is taken on that float32 value.  scale may be an array
+    broadcastable against v; a zero scale (an all-zero tensor) is treated as 1."""
     v = np.asarray(v, dtype=np.float32)
     s = np.asarray(scale, dtype=np.float32)
     s = np.where(s == 0, np.float32(1), s)
-    r = (np.float32(1) / s).astype(np.float32)
-    q = np.rint(v * r)                                  # float32 product; rint = ties to even
+    q = np.rint((v / s).astype(np.float32))             # float32 quotient; rint = ties to even
     return np.clip(q, -128, 127).astype(np.int8)
 
 

@@ -39,10 +39,18 @@ def build(force=False, verbose=False):
         common += ["-Xptxas", "-v"]
     procs = []
     objs = []
+    # an object is rebuilt when its source, any header of csrc/ or the public header is newer
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
+    headers.append(os.path.join(ROOT, "include", "nova.h"))
+    newest_header = max(os.path.getmtime(h) for h in headers)
     for src in SOURCES:
         obj = os.path.join(objdir, src.rsplit(".", 1)[0] + ".o")
         objs.append(obj)
-        cmd = [_nvcc()] + common + ["-x", "cu", "-c", os.path.join(CSRC, src), "-o", obj]
+        path = os.path.join(CSRC, src)
+        if (not force and not verbose and os.path.exists(obj)
+                and os.path.getmtime(obj) > max(os.path.getmtime(path), newest_header)):
+            continue
+        cmd = [_nvcc()] + common + ["-x", "cu", "-c", path, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for src, p in procs:

@@ -35,6 +35,18 @@ POINT_SETS = {
     ("nova", 8): _sym((2, 5), (5, 6), (1, 1), (7, 6)),
     # Table "Dtype-aware vs unconstrained discovery": dyadic points, exact in binary16
     ("dyadic", 4): _sym((3, 4), (5, 4)),
+    # Not from the paper: rational sets that are NOT symmetric about 0, in no particular order.
+    # Section 2.1 needs distinct points and nothing else; these exercise the general (dense) form
+    # of the transforms, which no printed set reaches.
+    ("asym", 2): [(1, 2), (-1, 1), (0, 1), INF],
+    ("asym", 4): [(3, 7), (-2, 1), (0, 1), (5, 4), (-1, 3), INF],
+    ("asym", 6): [(1, 1), (-1, 2), (2, 3), (0, 1), (-3, 2), (5, 4), (-3, 4), INF],
+    ("asym", 8): [(2, 5), (-6, 5), (1, 1), (-1, 2), (0, 1), (7, 6), (-3, 4), (5, 6), (-1, 1), INF],
+    # The discovered sets of Table 3 listed in another order (infinity stays last): the result is
+    # the same convolution; only the order of the transformed-domain coordinates changes.
+    ("shuf", 4): [(-7, 6), (5, 6), (0, 1), (7, 6), (-5, 6), INF],
+    ("shuf", 6): [(1, 1), (-3, 5), (7, 6), (0, 1), (-1, 1), (3, 5), (-7, 6), INF],
+    ("shuf", 8): [(-5, 6), (1, 1), (2, 5), (-7, 6), (0, 1), (7, 6), (-2, 5), (5, 6), (-1, 1), INF],
 }
 
 

@@ -119,10 +119,118 @@ def test_emulation_rounds_operands_to_fp16():
     assert 0.3 < e16c / e16 < 3
 
 
+# ---------------------------------------------------------------- the rounding points, one at a time
+# Each case below is built so that exactly ONE rounding of the half pipeline does anything, and the
+# expected output is computed here in exact rational arithmetic with that single rounding applied
+# by numpy's correctly rounded double -> half conversion.  F(2,3) on {0, 1, -1, inf}: the tables
+# hold only 0, +-1, +-1/2 (exact in half, products with them exact).
+def _exact_f23_with_roundings(x, g, round_U, round_V):
+    """The four steps on one F(2,3) problem in fractions; fl16 applied to U and/or V only.
+    Returns (y as fractions, every value that the float32 stages must hold exactly)."""
+    from fractions import Fraction as Fr
+    from oracle import toom_cook as tc
+    AT, G, BT = tc.build_matrices(2, 3, point_set("std", 2))
+    fl16 = lambda v: Fr(float(np.float16(float(v))))
+    N, H, W, C = x.shape
+    K = g.shape[0]
+    xf = [[[[Fr(float(x[i, h, w, c])) for c in range(C)] for w in range(W)] for h in range(H)] for i in range(N)]
+    U = [[[[sum(G[p][a] * Fr(float(g[k, a, b, c])) * G[q][b] for a in range(3) for b in range(3))
+            for c in range(C)] for k in range(K)] for q in range(4)] for p in range(4)]
+    held32 = [U[p][q][k][c] for p in range(4) for q in range(4) for k in range(K) for c in range(C)]
+    if round_U:
+        U = [[[[fl16(v) for v in kc] for kc in qk] for qk in pq] for pq in U]
+    y = {}
+    for i in range(N):
+        for th in range(-(-H // 2)):
+            for tw in range(-(-W // 2)):
+                def d(a, b, c):
+                    h, w = 2 * th - 1 + a, 2 * tw - 1 + b
+                    return xf[i][h][w][c] if 0 <= h < H and 0 <= w < W else Fr(0)
+                V = [[[sum(BT[p][a] * d(a, b, c) * BT[q][b] for a in range(4) for b in range(4))
+                       for c in range(C)] for q in range(4)] for p in range(4)]
+                held32 += [v for pq in V for qc in pq for v in qc]
+                if round_V:
+                    V = [[[fl16(v) for v in qc] for qc in pq] for pq in V]
+                for k in range(K):
+                    Mm = [[sum(U[p][q][k][c] * V[p][q][c] for c in range(C)) for q in range(4)] for p in range(4)]
+                    held32 += [v for row in Mm for v in row]
+                    for oi in range(2):
+                        for oj in range(2):
+                            h, w = 2 * th + oi, 2 * tw + oj
+                            if h < H and w < W:
+                                y[(i, h, w, k)] = sum(AT[oi][p] * Mm[p][q] * AT[oj][q] for p in range(4) for q in range(4))
+                                held32.append(y[(i, h, w, k)])
+    return y, held32
+
+
+def _check_single_rounding_case(x, g, round_U, round_V):
+    from fractions import Fraction as Fr
+    y_want, held32 = _exact_f23_with_roundings(x, g, round_U, round_V)
+    # the case is only valid if no float32 stage rounds: every such value fits 24 bits
+    assert all(Fr(float(np.float32(float(v)))) == v for v in held32)
+    y_other, _ = _exact_f23_with_roundings(x, g, False, False)
+    want = np.zeros(x.shape[:3] + (g.shape[0],), dtype=np.float16)
+    differs = 0
+    for key, v in y_want.items():
+        want[key] = np.float16(float(v))                  # the one rounding to the storage type
+        differs += np.float16(float(v)) != np.float16(float(y_other[key]))
+    assert differs >= len(y_want) // 4                    # the rounding under test is visible in the output
+    got = conv.winograd_conv_emulated(x, g, 2, point_set("std", 2), "fp16")
+    assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    return want
+
+
+def test_emulation_rounds_U_to_half_exactly_once():
+    # filters k * 2^-11: G g G^T are multiples of 2^-13 with up to 15 significant bits, so U must
+    # round; inputs are -1, 0, 1, so V is a small integer and every later sum is exact in float32
+    rng = np.random.default_rng(51)
+    g = (rng.integers(-2047, 2048, (3, 3, 3, 2)) * 2.0 ** -11).astype(np.float16)
+    x = rng.integers(-1, 2, (1, 5, 4, 2)).astype(np.float16)
+    _check_single_rounding_case(x, g, round_U=True, round_V=False)
+
+
+def test_emulation_rounds_V_to_half_exactly_once():
+    # inputs k * 2^-10 below 2: B^T d B are multiples of 2^-10 with up to 13 significant bits, so V
+    # must round; filters are multiples of 4, so U is a small integer
+    rng = np.random.default_rng(52)
+    x = (rng.integers(-2047, 2048, (1, 5, 4, 2)) * 2.0 ** -10).astype(np.float16)
+    g = (4 * rng.integers(-1, 2, (3, 3, 3, 2))).astype(np.float16)
+    _check_single_rounding_case(x, g, round_U=False, round_V=True)
+
+
+def test_emulation_sums_the_channels_in_float32_not_half():
+    # 4096 channels of ones: every output of the 2 x 2 image sees 4 pixels x 4096 channels = 16384,
+    # a power of two that half holds; the frequency (inf, inf) alone sums 4096 products 1 * 1, and
+    # the others sum up to 4096 * 3.  A sum carried in half stalls at 2048 (its ulp becomes 2).
+    C = 4096
+    x = np.ones((1, 2, 2, C), dtype=np.float16)
+    g = np.ones((1, 3, 3, C), dtype=np.float16)
+    y = conv.winograd_conv_emulated(x, g, 2, point_set("std", 2), "fp16")
+    assert np.array_equal(y, np.full((1, 2, 2, 1), 16384.0, dtype=np.float16))
+
+
+def test_fp32_emulation_stores_float32_and_sums_in_float64():
+    # mode "fp32": one rounding per stored element.  With inputs whose exact U, V, M and y all fit
+    # 24 bits the result is exact; and a channel sum that float32 accumulation would get wrong
+    # (2^24 + 1 + 1 + ... in float32 stays at 2^24) is right because the sum is carried in float64
+    rng = np.random.default_rng(53)
+    x = rng.integers(-3, 4, (1, 4, 6, 3)).astype(np.float32)
+    g = (4 * rng.integers(-3, 4, (2, 3, 3, 3))).astype(np.float32)
+    y = conv.winograd_conv_emulated(x, g, 2, point_set("std", 2), "fp32")
+    assert y.dtype == np.float32 and np.array_equal(y.astype(np.float64), conv.direct_conv_fp64(x, g))
+    C = 64
+    x = np.ones((1, 2, 2, C), dtype=np.float32)
+    g = np.zeros((1, 3, 3, C), dtype=np.float32)
+    g[0, 1, 1, :] = 1.0
+    g[0, 1, 1, 0] = 2.0 ** 24                       # y[0,0] = 2^24 + 63: not a float32, rounds to 2^24 + 64
+    y = conv.winograd_conv_emulated(x, g, 2, point_set("std", 2), "fp32")
+    assert y[0, 0, 0, 0] == np.float32(2.0 ** 24 + 64)
+
+
 def test_fp32_emulation_meets_stated_tolerances():
     x, g = make_conv_inputs(2, 14, 14, 32, 16, "fp32", True, True, seed=42)
     y1 = conv.direct_conv_fp64(x, g)
-    for kind, m, tol in [("std", 2, 1e-5), ("std", 4, 1e-5), ("nova", 4, 1e-5), ("nova", 6, 1e-4), ("nova", 8, 2e-4)]:
+    for kind, m, tol in [("std", 2, 1e-5), ("std", 4, 1e-5), ("nova", 4, 1e-5), ("nova", 6, 1e-4), ("nova", 8, 1e-4)]:
         e = conv.rel_l2(conv.winograd_conv_emulated(x, g, m, point_set(kind, m), "fp32"), y1)
         assert e < tol, (kind, m, e)
 
