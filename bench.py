@@ -24,11 +24,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch (cold caches) of the kernels of the default
-# path, from the ncu capture summarised in profiles/three_kernels_cfg3.md; retake when a kernel changes.
-NCU_DRAM_BYTES = {"cfg3": {"input_transform": 102833152, "product_tcgen05": 273757952,
-                           "output_transform": 241308160}}
-
 METRIC = "fp16 Winograd conv TFLOP/s (direct-equivalent)"
 UNIT = "TFLOP/s"
 
@@ -213,6 +208,57 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def alu_ceiling(c, P, clocks):
+    """Third ceiling beside tensor flops and HBM bytes: the fp32 arithmetic of the output transform,
+    the one transform of the half pipeline that runs on the CUDA cores (the input transform is a
+    tensor-core contraction).  Counted as executed for a point set symmetric about 0 - the +-pairs
+    share their even / odd sums and the rows of 0 and infinity are copies - in fp32 lane-operations
+    (an FMA, an add or a multiply on one value), against 128 lanes per SM per clock at the SM clock
+    sampled during the run (the maximum clock if none was sampled)."""
+    m, n = c.m, c.m + FILTER_R - 1
+    q = (n - 2) // 2                                   # +-pairs
+    row = 2 * q + m * q + 2                            # A^T applied to one row of M: sums/differences, m outputs, 2 copies added
+    col = q * m * (2 + m) + 2 * m                      # per pair and column: sum, difference, m multiply-adds; rows 0 and infinity
+    ops = n * row + col
+    dense = m * n * n + m * m * n
+    mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+    lanes = 148 * 128
+    total = float(ops) * P * c.K
+    return {"alu_us": total / (lanes * mhz * 1e6) * 1e6, "lane_ops_per_tile_filter": ops, "dense_lane_ops_per_tile_filter": dense,
+            "sm_mhz": mhz, "kernel": "output transform (fp32, CUDA cores)"}
+
+
+def run_fabric(args):
+    """SM <-> L2 / HBM rates by access kind: a buffer that stays in L2 (48 MiB) and one that does
+    not (1 GiB), all SMs and a quarter of them (per-SM against chip-wide limits)."""
+    import torch
+    import paper_2512_18453_b200 as nv
+    from synth import point_set
+    torch.cuda.set_device(0)
+    plan = nv.Plan(2, point_set("std", 2))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    kinds = {0: "ld.global.v4", 1: "st.global.v4", 2: "half the warps load, half store", 3: "bulk copy global->shared",
+             4: "bulk copy global->shared + st.global.v4", 5: "bulk copy shared->global",
+             6: "bulk copy global->shared + shared->global"}
+    rows = []
+    for mib in (48, 1024):
+        n = mib << 20
+        src = torch.ones(n, dtype=torch.uint8, device="cuda")
+        dst = torch.empty(n, dtype=torch.uint8, device="cuda")
+        iters = 20 if mib == 48 else 2
+        for ctas in (sms, sms // 4):
+            for kind, label in kinds.items():
+                for depth in ((4, 12) if kind in (3, 4, 6) else (1,)):
+                    ms = plan.probe_fabric(kind, src, dst, iters=iters, ctas=ctas, depth=depth)
+                    moved = n * iters * (2 if kind in (4, 6) else 1)
+                    rows.append({"buffer_mib": mib, "ctas": ctas, "kind": label, "depth": depth if kind in (3, 4, 6) else None,
+                                 "ms": ms, "tb_per_s": moved / (ms * 1e-3) / 1e12,
+                                 "bytes_per_clk_per_sm_at_1965mhz": moved / (ms * 1e-3) / ctas / 1.965e9})
+        del src, dst
+    assert plan.device_status() == 0
+    print(json.dumps({"fabric": rows}))
+
+
 def rank_seed(base_seed, rank):
     """Each rank draws its own batch (weak scaling): the seed is offset by the rank."""
     return base_seed + 100 * rank
@@ -273,12 +319,6 @@ def run_ours(args):
         else int(args.workspace_mb * (1 << 20))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     flags = {"auto": 0, "tcgen05": nv.GEMM_TCGEN05, "simt": nv.GEMM_SIMT}[args.gemm]
-    if args.fused:
-        flags |= nv.FUSED
-    if args.two_kernel:
-        flags |= nv.FUSED_PRODUCT_OUTPUT
-    if args.split:
-        plan.set_role_split(*[int(v) for v in args.split.split(",")])
     launches = plan.launch_count(c.N, c.H, c.W, c.C, c.K, ws_bytes, flags)
 
     # S1, once per layer: timed on its own
@@ -378,9 +418,7 @@ def run_ours(args):
         return
 
     peaks = read_peaks()
-    fused = launches == 1
-    two = launches == 2
-    chunks = 1 if (fused or two) else launches // 3
+    chunks = launches // 3
     names = ["input_transform", "product_tcgen05" if flags != nv.GEMM_SIMT else "product_simt", "output_transform"]
     n2 = (c.m + FILTER_R - 1) ** 2
     elt = 2
@@ -392,22 +430,14 @@ def run_ours(args):
     ]
     dom = max(range(3), key=lambda i: kms[i])
     bound, work = alg[dom]
-    if fused:
-        # one kernel does the whole step: its work is the path's (the larger of the two ceilings)
-        names = ["-", "fused_conv (input transform | tcgen05 product | output transform roles)", "-"]
-        t_tensor = actual / (peaks["tflops_burst"] * 1e12)
-        t_hbm = min_bytes / (peaks["hbm_gbs"] * 1e9)
-        bound, work = ("tensor", actual) if t_tensor > t_hbm else ("hbm", min_bytes)
     dur_launch = kms[dom] * 1e-3 / chunks
     if bound == "tensor":
         achieved, peak, runit = work / chunks / dur_launch / 1e12, peaks["tflops_burst"], "TFLOP/s"
     else:
         achieved, peak, runit = work / chunks / dur_launch / 1e9, peaks["hbm_gbs"], "GB/s"
-    traffic = None                 # DRAM bytes per launch of that kernel from the committed ncu capture
-    if two:
-        names = ["input_transform", "product+output (one kernel, M ring in L2)", "-"]
-    if not fused and not two and not args.images and chunks == 1 and FILTER_R == 3:
-        traffic = NCU_DRAM_BYTES.get(args.workload, {}).get(names[dom])
+    # DRAM bytes per launch come from an ncu capture, which this run is not: null here
+    traffic = None
+    alu = alu_ceiling(c, P, clocks)
     roof_s = max(actual / (peaks["tflops_burst"] * 1e12), min_bytes / (peaks["hbm_gbs"] * 1e9))
     value = whole_job_value(world, direct, ms_per_step)
     out = {
@@ -426,13 +456,15 @@ def run_ours(args):
         "path_roofline": {"roofline_us": roof_s * 1e6, "achieved_us": ms_per_step * 1e3,
                           "frac": roof_s / (ms_per_step * 1e-3), "peaks": peaks["source"],
                           "tensor_us": actual / (peaks["tflops_burst"] * 1e12) * 1e6,
-                          "hbm_us": min_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
+                          "hbm_us": min_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                          "alu_us": alu["alu_us"], "alu": alu},
         "kernels_ms_per_step": {n_: v for n_, v in zip(names, kms) if n_ != "-"},
         "single_step": step_stats,
         "filter_transform_ms": filter_ms,
         "roofline": {"kernel": names[dom], "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
-                     "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["source"],
-                     "launch_us": dur_launch * 1e6},
+                     "frac": achieved / peak, "traffic": traffic,
+                     "traffic_note": "null: DRAM counters are taken under ncu, never in a timed run",
+                     "peak_source": peaks["source"], "launch_us": dur_launch * 1e6},
         "e2e": {"value": world * direct / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(x_np.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)},
         "gpu_launches": launches * args.steps,
@@ -678,7 +710,7 @@ def run_vgg(args):
     x_np, weights = make_vgg_inputs(N)
     x = torch.from_numpy(x_np).cuda()
     Us = [plan.filter_transform(torch.from_numpy(w).cuda()) for w in weights]
-    flags = nv.RELU | (nv.FUSED if args.fused else 0)
+    flags = nv.RELU
     # buffers: activations of every layer, one scratch sized for the largest layer
     shapes, hw, c_in = [], 224, 8
     for (ci, co, pool) in VGG16_LAYERS:
@@ -759,7 +791,7 @@ def run_vgg(args):
         "config": {"workload": "cfg5: VGG-16 conv stack, 13 layers, N=%d, 224x224x3 (padded to 8 channels), F(%dx%d,3x3) %s points"
                                % (N, m, m, args.points),
                    "step": "13 x nova_conv2d_fwd (ReLU fused) + 5 x nova_maxpool2x2, CUDA graph replay",
-                   "workspace_mb": ws_bytes / (1 << 20), "fused": bool(args.fused)},
+                   "workspace_mb": ws_bytes / (1 << 20)},
         "images_per_s": N / (ms * 1e-3), "layers_ms": layers_ms, "gpu_launches": launches * steps, "device_status": status,
         "accuracy": acc, "clocks": clocks,
     }
@@ -778,9 +810,8 @@ def main():
     ap.add_argument("--gemm", default="auto", choices=["auto", "tcgen05", "simt"])
     ap.add_argument("--workspace-mb", type=float, default=None)
     ap.add_argument("--launch", default="graph", choices=["graph", "direct"])
-    ap.add_argument("--fused", action="store_true", help="the single role-specialised kernel instead of one kernel per step")
-    ap.add_argument("--two-kernel", action="store_true", help="input transform, then product+output in one kernel")
-    ap.add_argument("--split", default="", help="CTAs for the input-transform and product roles, e.g. 30,60")
+    ap.add_argument("--fabric", action="store_true",
+                    help="measure the SM <-> L2 / HBM rates by access kind (nova_probe_fabric) and print them")
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--accuracy", action="store_true",
                     help="report rel-L2 per point set (and per rescaled variant) even with --no-cpu-baseline")
@@ -798,6 +829,8 @@ def main():
     FILTER_R = args.filter
     if args.impl == "reference":
         run_reference(args)
+    elif args.fabric:
+        run_fabric(args)
     elif args.workload == "cfg5":
         run_vgg(args)
     elif args.int8:

@@ -19,7 +19,10 @@
  * named *_dev are device pointers, *_host host pointers; the caller owns every
  * buffer.  Device work is enqueued on `stream` (a cudaStream_t passed as
  * void*) and is asynchronous.  There is no CPU fallback: without a CUDA device
- * the device entry points return NOVA_ERR_CUDA.
+ * the device entry points return NOVA_ERR_CUDA.  A plan belongs to the device
+ * that was current when it was created (its status word and tables live
+ * there); a device entry point called with another device current returns
+ * NOVA_ERR_INVALID_ARG.
  */
 #ifndef NOVA_H_
 #define NOVA_H_
@@ -50,11 +53,6 @@ enum {
   NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
   NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
   NOVA_GEMM_TCGEN05 = 2 << 8, /* force the tcgen05 tensor-core product kernel */
-  NOVA_FUSED = 1 << 11,     /* run the three steps as ONE persistent kernel whose CTAs are specialised
-                               by role and exchange tiles through L2-resident rings (half mode, C >= 64;
-                               otherwise ignored); the default is one kernel per step */
-  NOVA_FUSED_PRODUCT_OUTPUT = 1 << 12, /* two kernels: the input transform, then product and output transform
-                               in one kernel with the product M in an L2-resident ring (half mode, C >= 64) */
   NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
                                    where the tensor-core formulation applies, the output transform
                                    without TMA staging (testing) */
@@ -97,8 +95,7 @@ typedef void* nova_stream;            /* a cudaStream_t */
  * or half, round to nearest even).  Host only: works without a CUDA device.
  * r = 3 plans have every kernel.  r = 5 (F(2,5), F(4,5), F(6,5); the appendix's 5 x 5
  * extension; g is then [K,5,5,C] and the padding 2) runs the filter transforms and the
- * convolutions, INT8 pipeline included, with the same kernels instantiated for n = m + 4;
- * the NOVA_FUSED* flags are ignored for such plans.
+ * convolutions, INT8 pipeline included, with the same kernels instantiated for n = m + 4.
  * On success *out must be released with nova_plan_destroy.
  */
 int nova_plan_create(int m, int r, const nova_rat* points_host, int n,
@@ -169,17 +166,12 @@ int nova_plan_get_device_tables(const nova_plan* plan, float* AT_host, float* G_
 /* The library indexes the n*n transformed-domain coordinates ("frequencies") of U in an
  * internal point order: frequency (xi, nu) of U is the pair of caller points
  * (perm_host[xi], perm_host[nu]).  For a set that is symmetric about 0 ({0, +-a_1, ..,
- * +-a_q, infinity}, as every set in the paper is) the internal order is 0, +a_1, -a_1, ..,
- * infinity and *symmetric_host is 1: the transforms then share the even/odd partial sums
+ * +-a_q, infinity}, as every set in the paper is, given in any order) the internal order is 0,
+ * +a_1, -a_1, .., infinity - the pairs in the order in which their first member appears in the
+ * caller's list - and *symmetric_host is 1: the transforms then share the even/odd partial sums
  * of each +-pair and skip the structural zeros (Appendix A, "symmetric point sets").
  * Any other set keeps the caller's order and dense transforms.  Either pointer may be null. */
 int nova_plan_frequency_order(const nova_plan* plan, int* perm_host, int* symmetric_host);
-
-/* Tuning of the single-kernel path (NOVA_FUSED): how many CTAs run the input transform; the
- * others run the transformed-domain product and the output transform side by side.  n_product
- * is ignored (kept for ABI stability); n_input = 0 restores the default share.  Not thread-safe
- * against concurrent nova_conv2d_fwd on the same plan. */
-int nova_plan_set_role_split(nova_plan* plan, int n_input, int n_product);
 
 /* kappa_2 = sigma_max/sigma_min of the Vandermonde matrix V_ij = a_i^j over the
  * n-1 finite points only (Section 2.2, "Vandermonde Conditioning"). */
@@ -337,6 +329,23 @@ int nova_conv2d_fwd_int8_timed(const nova_plan* plan, const void* x_dev, const v
  */
 int nova_selftest_wait_timeout(const nova_plan* plan, unsigned limit_ms, unsigned long long* waited_ns_host,
                                nova_stream stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): the rate at which the multiprocessors move bytes
+ * to and from the L2 / device memory with one kind of access, timed with CUDA events.  The
+ * transformed input and the transformed-domain product of the pipeline above cross that path
+ * twice each, so these rates bound it.  One persistent CTA on each of `ctas` multiprocessors walks
+ * `bytes` (a multiple of 16 KiB, at least 128 KiB) `iters` times:
+ *   kind 0 vector loads; 1 vector stores; 2 half the warps load and half store;
+ *   3 bulk asynchronous copies global -> shared, `depth` (1..12) 16 KiB pieces in flight per CTA;
+ *   4 kind 3 plus vector stores from the other warps; 5 bulk copies shared -> global; 6 kinds 3 + 5.
+ * Kinds 0-2 move `bytes` per iteration in total; 4 and 6 move `bytes` in each direction.
+ * src_dev (read) and dst_dev (written, contents undefined afterwards) are 128-byte aligned device
+ * buffers of `bytes`.  *ms_host receives the time of the `iters` passes.  Must run on the plan's
+ * device; synchronises `stream`; allocates 64 bytes for the duration of the call.
+ */
+int nova_probe_fabric(const nova_plan* plan, int kind, const void* src_dev, void* dst_dev, size_t bytes,
+                      int iters, int ctas, int depth, float* ms_host, nova_stream stream);
 
 /* 2x2 max pooling, stride 2, NHWC, H and W even, C % 8 == 0 (used between the
  * blocks of a VGG-style stack; not part of the paper's method).  `mode`

@@ -11,18 +11,16 @@ RELU = 1
 GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
 TRANSFORM_SIMT = 1 << 10
-FUSED = 1 << 11
-FUSED_PRODUCT_OUTPUT = 1 << 12
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
     "nova_plan_kappa", "nova_filter_transform_bytes", "nova_filter_transform",
     "nova_conv2d_workspace_bytes", "nova_conv2d_min_workspace_bytes", "nova_conv2d_fwd",
     "nova_conv2d_fwd_host", "nova_conv2d_fwd_timed", "nova_conv2d_launch_count", "nova_maxpool2x2", "nova_last_device_status",
-    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_plan_set_role_split", "nova_last_cuda_error",
+    "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_last_cuda_error",
     "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
     "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices", "nova_symmetric_search",
-    "nova_selftest_wait_timeout",
+    "nova_selftest_wait_timeout", "nova_probe_fabric",
     "nova_filter_transform_int8_bytes", "nova_filter_transform_int8", "nova_conv2d_int8_workspace_bytes",
     "nova_conv2d_fwd_int8", "nova_conv2d_fwd_int8_timed",
 )
@@ -82,8 +80,8 @@ def lib():
     L.nova_plan_get_device_tables.restype = i
     L.nova_plan_frequency_order.argtypes = [vp, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.nova_plan_frequency_order.restype = i
-    L.nova_plan_set_role_split.argtypes = [vp, i, i]
-    L.nova_plan_set_role_split.restype = i
+    L.nova_probe_fabric.argtypes = [vp, i, vp, vp, sz, i, i, i, fp, vp]
+    L.nova_probe_fabric.restype = i
     L.nova_last_cuda_error.argtypes = []
     L.nova_last_cuda_error.restype = i
     L.nova_plan_kappa.argtypes = [vp, dp]
@@ -267,8 +265,12 @@ class Plan:
         _check(lib().nova_plan_frequency_order(self._h, perm, ctypes.byref(sym)), "nova_plan_frequency_order")
         return list(perm), bool(sym.value)
 
-    def set_role_split(self, n_input, n_product):
-        _check(lib().nova_plan_set_role_split(self._h, n_input, n_product), "nova_plan_set_role_split")
+    def probe_fabric(self, kind, src, dst, iters=10, ctas=148, depth=8):
+        """nova_probe_fabric on two uint8 CUDA tensors of equal size; returns milliseconds for `iters` passes."""
+        ms = ctypes.c_float()
+        _check(lib().nova_probe_fabric(self._h, kind, src.data_ptr(), dst.data_ptr(), src.numel(), iters, ctas, depth,
+                                       ctypes.byref(ms), _stream()), "nova_probe_fabric")
+        return ms.value
 
     def kappa(self):
         k = ctypes.c_double()

@@ -2,7 +2,7 @@
 //
 // The tiles of a problem are processed in chunks sized so that the transformed
 // input V (operand type) and the transformed-domain product M (float) of one
-// chunk stay resident in the 126 MB L2: input transform -> product -> output
+// chunk fit the caller's scratch: input transform -> product -> output
 // transform per chunk, all on the caller's stream, no host synchronisation.
 #include <cuda_runtime.h>
 
@@ -47,50 +47,19 @@ bool choose_chunking(const nova_plan* p, const Geom& g, size_t bytes, Chunking* 
   return c->v_bytes + c->m_bytes <= bytes;
 }
 
-// 3 x 3 filters have every kernel; 5 x 5 filters (F(2,5), F(4,5), F(6,5)) run the CUDA-core
-// same kernels instantiated for n = m + 4.  The fused paths are 3 x 3 only.
+// 3 x 3 filters and 5 x 5 filters (F(2,5), F(4,5), F(6,5)) run the same kernels, instantiated
+// for n = m + 2 and n = m + 4.
 bool device_plan(const nova_plan* p) { return p && (p->r == kR || p->r == 5); }
 bool shape_ok(int N, int H, int W, int C, int K) {
   return N > 0 && H > 0 && W > 0 && C > 0 && K > 0 && (C % 8) == 0 && (K % 8) == 0;
 }
 bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-// The single-kernel path applies in half mode with the tensor-core transforms, when the
-// scratch holds a ring of at least two 128-tile blocks (or all of them).  *R = ring length.
-bool fused_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R) {
-  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev || p->r != kR) return false;
-  if (!(flags & NOVA_FUSED) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT))) return false;
-  if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
-  const long long NB = (g.P + 127) / 128;
-  if (bytes < 2 * kAlign) return false;
-  long long r = (long long)((bytes - 2 * kAlign) / fused_block_bytes(p, g.C, g.K));
-  if (r > NB) r = NB;
-  if (r < 2 && r < NB) return false;
-  if (r < 1) return false;
-  if (r > 8) r = 8;                                   // the rings stay inside the L2; longer ones were never validated
-  *R = (int)r;
-  return true;
-}
-
-// Two-kernel path: the input transform over all tiles, then ONE kernel for product and output
-// transform with M in an L2-resident ring of *R blocks.  The scratch holds V for all tiles
-// (padded to whole blocks) and the ring.
-bool two_kernel_applies(const nova_plan* p, const Geom& g, size_t bytes, int flags, int* R, size_t* v_bytes) {
-  if (p->mode != NOVA_FP16_F32ACC || !p->kron_dev || !p->fused_ctr_dev || !p->status_dev || p->r != kR) return false;
-  if (!(flags & NOVA_FUSED_PRODUCT_OUTPUT) || (flags & (NOVA_GEMM_SIMT | NOVA_TRANSFORM_SIMT | NOVA_FUSED))) return false;
-  if (g.C < 64 || g.P > (long long)p->fused_ctr_blocks * 128 || g.P >= (1ll << 24)) return false;
-  const long long NB = (g.P + 127) / 128;
-  const size_t vb = round_up((size_t)g.n * g.n * NB * 128 * g.C * 2, kAlign);
-  const size_t mblock = (size_t)g.n * g.n * 128 * g.K * 4;
-  if (bytes < vb + 2 * kAlign) return false;
-  long long r = (long long)((bytes - vb - kAlign) / mblock);
-  if (r > NB) r = NB;
-  if (r > 8) r = 8;                                   // keep the ring well inside the L2
-  if (r < 2 && r < NB) return false;
-  if (r < 1) return false;
-  *R = (int)r;
-  *v_bytes = vb;
-  return true;
+// The plan's status word, its tables and the built-in scratch belong to one device: the device
+// entry points refuse to run with another one current.
+bool on_plan_device(const nova_plan* p) {
+  int dev = -1;
+  return p->device >= 0 && cudaGetDevice(&dev) == cudaSuccess && dev == p->device;
 }
 
 bool use_tcgen05(const nova_plan* p, int flags) {
@@ -113,7 +82,11 @@ extern "C" int nova_filter_transform(const nova_plan* p, const void* g, int K, i
   if (!p || !aligned16(g) || !aligned16(U) || K <= 0 || C <= 0 || (K % 8) || (C % 8))
     return NOVA_ERR_INVALID_ARG;
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
-  return launch_filter_transform(p, g, K, C, U, stream) == 0 ? NOVA_OK : NOVA_ERR_CUDA;
+  if (p->device < 0) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
+  const int e = p->mode == NOVA_FP32 ? launch_filter_transform_f32(p, g, K, C, U, stream)
+                                     : launch_filter_transform(p, g, K, C, U, stream);
+  return e == 0 ? NOVA_OK : NOVA_ERR_CUDA;
 }
 
 extern "C" size_t nova_conv2d_min_workspace_bytes(const nova_plan* p, int N, int H, int W, int C, int K) {
@@ -138,10 +111,6 @@ extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W,
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   Geom g = make_geom(p, N, H, W, C, K);
-  int R = 0;
-  size_t vb = 0;
-  if (fused_applies(p, g, workspace_bytes, flags, &R)) return 1;
-  if (two_kernel_applies(p, g, workspace_bytes, flags, &R, &vb)) return 2;
   Chunking c;
   if (!choose_chunking(p, g, workspace_bytes, &c)) return NOVA_ERR_WORKSPACE;
   return 3 * c.chunks;
@@ -158,30 +127,9 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if ((flags & NOVA_GEMM_TCGEN05) && p->mode == NOVA_FP32) return NOVA_ERR_UNSUPPORTED;
+  if (p->device < 0) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
   Geom g = make_geom(p, N, H, W, C, K);
-  int R = 0;
-  if (fused_applies(p, g, ws_bytes, flags, &R)) {
-    cudaStream_t s = (cudaStream_t)stream;
-    if (ev) cudaEventRecord(ev[1], s);
-    const int e = launch_fused_conv(p, g, x, U, y, ws, R, (flags & NOVA_RELU) ? 1 : 0, stream);
-    if (ev) cudaEventRecord(ev[2], s);
-    if (e) g_last_cuda_error = e;
-    return e ? NOVA_ERR_CUDA : NOVA_OK;
-  }
-  size_t vb = 0;
-  if (two_kernel_applies(p, g, ws_bytes, flags, &R, &vb)) {
-    cudaStream_t s = (cudaStream_t)stream;
-    const int pad = (int)((g.P + 127) / 128 * 128);
-    if (ev) cudaEventRecord(ev[0], s);
-    int e = launch_input_transform_tc(p, g, x, ws, 0, (int)g.P, pad, stream);
-    if (ev) cudaEventRecord(ev[1], s);
-    if (!e)
-      e = launch_fused_product_output(p, g, x, ws, U, y, reinterpret_cast<float*>(static_cast<char*>(ws) + vb), R,
-                                      (flags & NOVA_RELU) ? 1 : 0, stream);
-    if (ev) { cudaEventRecord(ev[2], s); cudaEventRecord(ev[3], s); }
-    if (e) g_last_cuda_error = e;
-    return e ? NOVA_ERR_CUDA : NOVA_OK;
-  }
   Chunking c;
   if (!choose_chunking(p, g, ws_bytes, &c)) return NOVA_ERR_WORKSPACE;
   const bool tc = use_tcgen05(p, flags);
@@ -194,9 +142,11 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   for (long long p0 = 0; p0 < g.P; p0 += c.pc, ++ci) {
     const int pc = (int)((g.P - p0) < c.pc ? (g.P - p0) : c.pc);
     if (ev) cudaEventRecord(ev[4 * ci + 0], s);
+    const bool f32 = p->mode == NOVA_FP32;
     const bool tc_in = tc && p->kron_dev && C >= 64 && !(flags & NOVA_TRANSFORM_SIMT);
-    if (tc_in ? launch_input_transform_tc(p, g, x, Vb, p0, pc, c.pc_pad, stream)
-              : launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream))
+    if (f32     ? launch_input_transform_f32(p, g, x, Vb, p0, pc, c.pc_pad, stream)
+        : tc_in ? launch_input_transform_tc(p, g, x, Vb, p0, pc, c.pc_pad, stream)
+                : launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream))
       return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 1], s);
     const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream)
@@ -204,7 +154,8 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
     const int relu = (flags & NOVA_RELU) ? 1 : 0;
-    if ((p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
+    if (f32 ? launch_output_transform_f32(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
+        : (p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
             ? launch_output_transform_tma(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
             : launch_output_transform(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream))
       return NOVA_ERR_CUDA;
@@ -226,19 +177,13 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   if (!kernel_ms) return NOVA_ERR_INVALID_ARG;
   const int launches = nova_conv2d_launch_count(p, N, H, W, C, K, ws_bytes, flags);
   if (launches < 0) return launches;
-  const bool fused = launches == 1, two = launches == 2;
-  const int chunks = (fused || two) ? 1 : launches / 3;
+  const int chunks = launches / 3;
   cudaEvent_t* ev = new cudaEvent_t[4 * chunks];
   for (int i = 0; i < 4 * chunks; ++i) cudaEventCreate(&ev[i]);
   int st = conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, ev);
   if (st == NOVA_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st = NOVA_ERR_CUDA;
   kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
-  if (st == NOVA_OK && fused) {
-    cudaEventElapsedTime(&kernel_ms[1], ev[1], ev[2]);      // the one kernel does all three steps
-  } else if (st == NOVA_OK && two) {
-    cudaEventElapsedTime(&kernel_ms[0], ev[0], ev[1]);      // input transform
-    cudaEventElapsedTime(&kernel_ms[1], ev[1], ev[2]);      // product + output transform in one kernel
-  } else if (st == NOVA_OK)
+  if (st == NOVA_OK)
     for (int c = 0; c < chunks; ++c)
       for (int k = 0; k < 3; ++k) {
         float ms = 0.f;
@@ -354,6 +299,8 @@ extern "C" int nova_conv2d_fwd_static(const nova_plan* p, const void* x, const v
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   if (nova_conv2d_min_workspace_bytes(p, N, H, W, C, K) > NOVA_STATIC_SCRATCH_BYTES)
     return NOVA_ERR_STATIC_LIMIT;
+  if (p->device < 0) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;   // the scratch looked up below is the current device's
   void* ws = nullptr;
   const int st = static_scratch_address(&ws);
   if (st != NOVA_OK) return st;
@@ -387,6 +334,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
     return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
   if (!p->status_dev) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
   const Geom g = make_geom(p, N, H, W, C, K);
   if (g.P >= (1ll << 24)) return NOVA_ERR_UNSUPPORTED;
   const Int8Layout l = int8_layout(g);
@@ -440,6 +388,8 @@ extern "C" int nova_filter_transform_int8(const nova_plan* p, const void* g, int
   if (quant != NOVA_QUANT_PER_TENSOR && quant != NOVA_QUANT_PER_CHANNEL && quant != NOVA_QUANT_GIVEN)
     return NOVA_ERR_INVALID_ARG;
   if (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) return NOVA_ERR_UNSUPPORTED;
+  if (p->device < 0) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
   const int e = launch_filter_transform_int8(p, g, K, C, Uq, scale_U, quant, stream);
   if (e) g_last_cuda_error = e;
   return e ? NOVA_ERR_CUDA : NOVA_OK;

@@ -1,10 +1,12 @@
 // Transformed-domain product on CUDA cores (Section 2.1 step 3, summed over
 // input channels): for every frequency f,
-//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c]   (float accumulation),
-// stored as [f][K/4][pc_pad][4] like the tensor-core kernel's output.
+//   M[f][p][k] = sum_c V[f][p][c] * U[f][k][c],
+// stored as float [f][K/4][pc_pad][4] like the tensor-core kernel's output.
 // This is the product kernel of the fp32 mode (a single-pass TF32 tensor-core
 // product cannot meet a 1e-5 tolerance) and a cross-check for the tcgen05
-// kernel in fp16 mode.
+// kernel in fp16 mode.  Half operands accumulate in float (their products are
+// exact in float); float operands accumulate in double and the sum is rounded
+// once to float, like every stored tensor of the fp32 mode.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -17,6 +19,10 @@ constexpr int BM = 64, BN = 64, BK = 16;
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__half v) { return __half2float(v); }
+template <typename T> struct AccOf { using type = float; };
+template <> struct AccOf<float> { using type = double; };
+__device__ __forceinline__ float mac(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ double mac(float a, float b, double c) { return fma((double)a, (double)b, c); }
 
 // 256 threads, each a 4 x 4 block of the 64 x 64 output tile.
 template <typename T>
@@ -33,7 +39,8 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;           // tx -> k, ty -> p
   const int lr = tid >> 2, lc = (tid & 3) * 4;      // loader: row 0..63, 4 channels at lc
-  float acc[4][4] = {};
+  using Acc = typename AccOf<T>::type;
+  Acc acc[4][4] = {};
   for (int c0 = 0; c0 < C; c0 += BK) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -53,7 +60,7 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) acc[i][j] = mac(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
@@ -64,7 +71,7 @@ gemm_simt_kernel(const T* __restrict__ V, const T* __restrict__ U, float* __rest
     const int k = kb + tx * 4;                        // K % 8 == 0: a filter quad is all in or all out
     if (k < K)
       *reinterpret_cast<float4*>(Mf + ((size_t)(k >> 2) * pc_pad + p) * 4) =
-          make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+          make_float4((float)acc[i][0], (float)acc[i][1], (float)acc[i][2], (float)acc[i][3]);
   }
 }
 

@@ -23,6 +23,7 @@
 
 #include "nova_internal.h"
 #include "sm100.cuh"
+#include "tma_host.h"
 
 namespace nova {
 namespace {
@@ -201,30 +202,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
 // [nfreq][rows][inner] elements of `esize` bytes, frequency stride in elements;
 // box = [1][box_rows][box_inner], 128-byte swizzle (box_inner * esize == 128).
 bool make_map_3d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base, int inner, int rows,
                  long long freq_stride_elems, int nfreq, int box_inner, int box_rows) {
-  EncodeTiledFn enc = get_encode_fn();
+  EncodeTiledFn enc = tensor_map_encoder();
   if (!enc) return false;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)nfreq};
   cuuint64_t strides[2] = {(cuuint64_t)inner * esize, (cuuint64_t)freq_stride_elems * esize};
@@ -239,13 +221,7 @@ template <int BLOCK_N, bool I8>
 int launch_n(int sms, const void* V, const void* U, float* M, int nfreq, int pc, int pc_pad, int C, int K,
              int* status, cudaStream_t stream) {
   using L = SmemLayout<BLOCK_N>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BLOCK_N, I8>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return (int)e;
-    attr_set = true;
-  }
+  if (cudaError_t e = allow_dynamic_smem(gemm_tcgen05_kernel<BLOCK_N, I8>, L::kTotal); e != cudaSuccess) return (int)e;
   CUtensorMap tmV, tmU;
   const CUtensorMapDataType dt = I8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
   constexpr int esize = I8 ? 1 : 2;

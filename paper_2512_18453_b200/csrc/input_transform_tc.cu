@@ -33,6 +33,7 @@
 
 #include "nova_internal.h"
 #include "sm100.cuh"
+#include "tma_host.h"
 
 namespace nova {
 namespace {
@@ -287,37 +288,12 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
 template <int M, int QMODE, int R = 3>
 int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc, int pc_pad,
              float* qslot, cudaStream_t stream) {
   using Cfg = TcCfg<M, R>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(input_transform_tc_kernel<M, QMODE, R>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
-    if (e != cudaSuccess) return (int)e;
-    attr_set = true;
-  }
-  EncodeTiledFn enc = encode_fn();
+  if (cudaError_t e = allow_dynamic_smem(input_transform_tc_kernel<M, QMODE, R>, Cfg::kTotal); e != cudaSuccess) return (int)e;
+  EncodeTiledFn enc = tensor_map_encoder();
   if (!enc) return (int)cudaErrorUnknown;
   CUtensorMap tmX, tmK;
   {

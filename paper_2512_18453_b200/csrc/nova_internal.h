@@ -47,9 +47,6 @@ struct nova_plan {
   int* status_dev;                        // device status word (null without a device)
   int device;                             // device that owns status_dev
   int sm_count;                           // multiprocessors of that device
-  uint32_t* fused_ctr_dev;                // per-block counters of the fused kernel (may be null)
-  int fused_ctr_blocks;                   // capacity of fused_ctr_dev in 128-tile blocks
-  int fused_nI, fused_nG;                 // CTAs given to the input-transform / product roles (0 = default)
 };
 
 namespace nova {
@@ -95,11 +92,12 @@ int launch_gemm_tcgen05_i8(const nova_plan* plan, const void* V, const void* U, 
                            int pc_pad, int C, int K, int* status_dev, void* stream);
 int launch_gemm_simt_i8(const void* V, const void* U, int32_t* M, int nfreq, int pc, int pc_pad, int C, int K,
                         void* stream);
-int launch_fused_conv(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, void* ws,
-                      int R, int relu, void* stream);
-int launch_fused_product_output(const nova_plan* plan, const Geom& g, const void* x, const void* V, const void* U,
-                                void* y, float* Mring, int R, int relu, void* stream);
-size_t fused_block_bytes(const nova_plan* plan, int C, int K);
+// fp32 mode: sums carried in double, one rounding per stored float
+int launch_filter_transform_f32(const nova_plan* plan, const void* g, int K, int C, void* U, void* stream);
+int launch_input_transform_f32(const nova_plan* plan, const Geom& g, const void* x, void* V, long long p0, int pc,
+                               int pc_pad, void* stream);
+int launch_output_transform_f32(const nova_plan* plan, const Geom& g, const void* M, void* y, long long p0, int pc,
+                                int pc_pad, int relu, void* stream);
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,
                      int nfreq, int pc, int pc_pad, int C, int K, void* stream);
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M,

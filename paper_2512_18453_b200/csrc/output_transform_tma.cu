@@ -18,6 +18,7 @@
 
 #include "nova_internal.h"
 #include "sm100.cuh"
+#include "tma_host.h"
 #include "output_math.cuh"
 #include "transform_math.cuh"
 
@@ -138,36 +139,11 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
 template <int M, typename T, bool SYM, int VEC, bool QUANT, int R = 3>
 int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
                int pc_pad, int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
   using Cfg = OtCfg<M, VEC, R>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kTotal);
-    if (e != cudaSuccess) return (int)e;
-    attr_set = true;
-  }
+  if (cudaError_t e = allow_dynamic_smem(output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R>, Cfg::kTotal); e != cudaSuccess) return (int)e;
   const long long units = (long long)(pc_pad / 8) * ((g.K + 16 * VEC - 1) / (16 * VEC));
   const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
   output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
@@ -178,7 +154,7 @@ int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, voi
 template <int M, int R = 3>
 int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long long p0, int pc, int pc_pad,
              int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
-  EncodeTiledFn enc = encode_fn();
+  EncodeTiledFn enc = tensor_map_encoder();
   if (!enc) return (int)cudaErrorUnknown;
   CUtensorMap tmM;
   const int k4 = g.K / 4;
@@ -191,23 +167,11 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return (int)cudaErrorUnknown;
-  const bool f32 = plan->mode == NOVA_FP32;
+  if (plan->mode == NOVA_FP32) return (int)cudaErrorInvalidValue;   // the fp32 mode has its own transforms
 #define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q, R>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
-  if constexpr (R != 3) {                             // 5-tap filters
-    if (scale_U) {
-      if (f32) return (int)cudaErrorInvalidValue;
-      return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
-    }
-    if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
-    return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
-  } else {
-    if (scale_U) {                                    // int8 pipeline (half storage only)
-      if (f32) return (int)cudaErrorInvalidValue;
-      return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
-    }
-    if (plan->symmetric) return f32 ? NOVA_OT(float, true, false) : NOVA_OT(__half, true, false);
-    return f32 ? NOVA_OT(float, false, false) : NOVA_OT(__half, false, false);
-  }
+  if (scale_U)                                        // int8 pipeline: M holds int32 sums
+    return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
+  return plan->symmetric ? NOVA_OT(__half, true, false) : NOVA_OT(__half, false, false);
 #undef NOVA_OT
 }
 

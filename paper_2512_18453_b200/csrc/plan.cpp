@@ -435,14 +435,6 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
         pl->device = dev;
         cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev);
       }
-      if (pl->status_dev) {
-        const int cap = 1 << 16;                       // blocks of 128 tiles
-        uint32_t* cd = nullptr;
-        if (cudaMalloc((void**)&cd, (size_t)(3 * cap + 4) * sizeof(uint32_t)) == cudaSuccess) {
-          pl->fused_ctr_dev = cd;
-          pl->fused_ctr_blocks = cap;
-        }
-      }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
       if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
         std::vector<unsigned short> img(nova::kron_table_halves(n));
@@ -486,14 +478,27 @@ extern "C" int nova_snap_to_rational(double x, int max_den, nova_rat* out) {
   i128 X = (i128)(long long)std::ldexp(fr, 53);
   int s = 53 - e;
   while (s < 0) { X *= 2; ++s; }
+  // For a denominator b the closest numerator is one of the two integers around x b (exactly:
+  // floor(X b / 2^s) and its successor), clamped to [-5b, 5b]; the winner over all b is found by
+  // cross-multiplication.  Ties follow the order of the definition's enumeration (Algorithm 2:
+  // b ascending, then a ascending, strict "<"): the smaller b, then the smaller a, stays.
   long long best_a = 0, best_b = 1;
   i128 best_num = -1;
-  for (long long b = 1; b <= max_den; ++b)          // Algorithm 2's scan order; strict "<" keeps the first of a tie
-    for (long long a = -5 * b; a <= 5 * b; ++a) {
-      i128 num = X * b - ((i128)a << s);
+  for (long long b = 1; b <= max_den; ++b) {
+    const i128 Xb = X * b;
+    i128 fl = Xb >> s;                                  // arithmetic shift: floor for negative values too
+    long long cand[2] = {(long long)fl, (long long)fl + 1};
+    for (int t = 0; t < 2; ++t) {
+      long long a = cand[t];
+      if (a < -5 * b) a = -5 * b;
+      if (a > 5 * b) a = 5 * b;
+      if (t == 1 && a == cand[0]) continue;             // both clamped to the same end
+      cand[t] = a;
+      i128 num = Xb - ((i128)a << s);
       if (num < 0) num = -num;
       if (best_num < 0 || num * best_b < best_num * b) { best_num = num; best_a = a; best_b = b; }
     }
+  }
   const long long g = (long long)gcd128(best_a, best_b);
   out->num = best_a / (g ? g : 1);
   out->den = best_b / (g ? g : 1);
@@ -607,7 +612,6 @@ extern "C" void nova_plan_destroy(nova_plan* plan) {
   if (!plan) return;
   if (plan->status_dev) cudaFree(plan->status_dev);
   if (plan->kron_dev) cudaFree(plan->kron_dev);
-  if (plan->fused_ctr_dev) cudaFree(plan->fused_ctr_dev);
   delete plan;
 }
 
@@ -638,13 +642,6 @@ extern "C" int nova_plan_frequency_order(const nova_plan* p, int* perm, int* sym
   if (perm)
     for (int i = 0; i < p->n; ++i) perm[i] = p->perm[i];
   if (symmetric) *symmetric = p->symmetric;
-  return NOVA_OK;
-}
-
-extern "C" int nova_plan_set_role_split(nova_plan* p, int n_input, int n_product) {
-  if (!p || n_input < 0 || n_product < 0) return NOVA_ERR_INVALID_ARG;
-  p->fused_nI = n_input;
-  p->fused_nG = n_product;
   return NOVA_OK;
 }
 

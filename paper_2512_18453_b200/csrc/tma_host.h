@@ -1,0 +1,36 @@
+// Host-side helpers of the TMA kernels: the driver's tensor-map encoder, looked up once.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+namespace nova {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry-point query (the library does not
+// link libcuda).  The function-local static is initialised exactly once, also when several host
+// threads make their first call at the same time; null if the driver lacks the entry point.
+inline EncodeTiledFn tensor_map_encoder() {
+  static const EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      return (EncodeTiledFn)p;
+    return (EncodeTiledFn) nullptr;
+  }();
+  return fn;
+}
+
+// Opt a kernel in to `bytes` of dynamic shared memory.  The attribute belongs to the (function,
+// device) pair, so it is set on every launch path rather than remembered per process: the call
+// is a few hundred nanoseconds of host time.
+template <typename Kernel>
+inline cudaError_t allow_dynamic_smem(Kernel kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+}  // namespace nova

@@ -1,7 +1,8 @@
 // Transform kernels of the Winograd pipeline (Section 2.1 steps 1, 2 and 4 in
 // their 2-D nested form, Appendix B.5): U = G g G^T, V = B^T d B, Y = A^T M A.
-// Each is evaluated in float from coefficient tables held in the constant bank
-// (a __grid_constant__ parameter) and rounded once to the destination type.
+// Half storage: each is evaluated in float from coefficient tables held in the constant bank
+// (a __grid_constant__ parameter) and rounded once to half (or quantised, for the int8
+// pipeline).  The fp32 mode's transforms are in fp32_path.cu.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -485,14 +486,15 @@ int output_launch(const nova_plan* plan, const Geom& g, const void* Mb, void* y,
 
 }  // namespace
 
+// Half storage only: the fp32 mode has its own transform kernels.
 #define NOVA_DISPATCH_M_T(FN, ...)                                                   \
   do {                                                                               \
-    const bool f32 = plan->mode == NOVA_FP32;                                        \
+    if (plan->mode == NOVA_FP32) return (int)cudaErrorInvalidValue;                  \
     switch (plan->m) {                                                               \
-      case 2: return f32 ? FN<2, float>(__VA_ARGS__) : FN<2, __half>(__VA_ARGS__);   \
-      case 4: return f32 ? FN<4, float>(__VA_ARGS__) : FN<4, __half>(__VA_ARGS__);   \
-      case 6: return f32 ? FN<6, float>(__VA_ARGS__) : FN<6, __half>(__VA_ARGS__);   \
-      case 8: return f32 ? FN<8, float>(__VA_ARGS__) : FN<8, __half>(__VA_ARGS__);   \
+      case 2: return FN<2, __half>(__VA_ARGS__);                                     \
+      case 4: return FN<4, __half>(__VA_ARGS__);                                     \
+      case 6: return FN<6, __half>(__VA_ARGS__);                                     \
+      case 8: return FN<8, __half>(__VA_ARGS__);                                     \
     }                                                                                \
     return (int)cudaErrorInvalidValue;                                               \
   } while (0)
