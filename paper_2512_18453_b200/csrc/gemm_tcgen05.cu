@@ -4,7 +4,7 @@
 // or, for the int8 pipeline (I8), signed 8-bit x signed 8-bit -> int32 (exact).
 //
 // Persistent, warp-specialised kernel.  One CTA per SM walks a list of work
-// items (f, 128-row block of tiles p, BLOCK_N-wide block of filters k):
+// items (f, 128-row block of tiles p, BLOCK_N-wide block of filters k; the filter blocks of a (f, p) pair one after the other):
 //   warp 0    TMA producer: 128B-swizzled [rows][64 channels] boxes of V and U
 //             into a 4-stage shared-memory ring, completion on mbarriers;
 //   warp 1    issues tcgen05.mma (kind::f16, M=128, N=BLOCK_N, K=16) from
@@ -48,7 +48,7 @@ template <int BLOCK_N, bool I8>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
                     float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
-                    int* __restrict__ status) {
+                    int* __restrict__ status, const uint8_t* __restrict__ Vdrop) {
   using L = SmemLayout<BLOCK_N>;
   constexpr int BLOCK_K = I8 ? kRowBytes : kRowBytes / 2;   // elements of K per stage
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
@@ -66,19 +66,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const int num_pb = (pc + BLOCK_M - 1) / BLOCK_M;
   const int num_kb = (K + BLOCK_N - 1) / BLOCK_N;
   const int num_ks = (C + BLOCK_K - 1) / BLOCK_K;
-  const long long num_items = (long long)nfreq * num_pb * num_kb;
-  // Item i of this CTA is item blockIdx.x + i * gridDim.x, with the row block outermost and
-  // DESCENDING (then frequency, then filter block): the input transform wrote V in ascending
-  // tile order, so the highest row blocks are the ones still in L2; and the row blocks this
-  // kernel finishes last - the lowest - are the ones the output transform reads first.
-  const unsigned per_pb = (unsigned)nfreq * (unsigned)num_kb;
-  const uint32_t n_local = num_items > blockIdx.x ? (uint32_t)((num_items - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0u;
+  // The work list is (row block, frequency), the row block outermost and DESCENDING: the input
+  // transform wrote V in ascending tile order, so the highest row blocks are the ones still in
+  // L2; and the row blocks this kernel finishes last - the lowest - are the ones the output
+  // transform reads first.  Pair i of this CTA is pair blockIdx.x + i * gridDim.x; the CTA runs
+  // the pair's filter blocks one after the other (items), so that it is the only reader of the
+  // pair's rows of V and knows when they have been read for the last time.
+  const long long num_pairs = (long long)nfreq * num_pb;
+  const uint32_t pairs_local = num_pairs > blockIdx.x ? (uint32_t)((num_pairs - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0u;
+  const uint32_t n_local = pairs_local * (uint32_t)num_kb;
   auto item_of = [&](uint32_t local, int& pb, int& f, int& kb) {
-    const unsigned it = blockIdx.x + local * gridDim.x;
-    pb = num_pb - 1 - (int)(it / per_pb);
-    const unsigned rem = it % per_pb;
-    f = (int)(rem / (unsigned)num_kb);
-    kb = (int)(rem % (unsigned)num_kb);
+    const unsigned pair = blockIdx.x + (local / (unsigned)num_kb) * gridDim.x;
+    pb = num_pb - 1 - (int)(pair / (unsigned)nfreq);
+    f = (int)(pair % (unsigned)nfreq);
+    kb = (int)(local % (unsigned)num_kb);
   };
 
   if (threadIdx.x == 0) {
@@ -99,6 +100,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_base_slot;
   bool timed_out = false;
+  // everything above touched no global memory: it may overlap the tail of the preceding kernel
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     // ---------------- TMA producer
@@ -128,6 +132,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tmem_d = tmem_base + acc * BLOCK_N;
+      int item_pb, item_f, item_kb;
+      item_of(local, item_pb, item_f, item_kb);
       for (int ks = 0; ks < num_ks; ++ks) {
         if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -150,6 +156,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
           if (ks == num_ks - 1) umma_commit(&tmem_full[acc]);
         }
         __syncwarp();
+        // V is scratch and this was the last read of the 128 rows x 128 bytes that have just
+        // landed in shared memory: drop those lines from the L2, so that the ones still dirty
+        // there (the input transform wrote them moments ago) are never written back.
+        if (Vdrop && item_kb == num_kb - 1) {
+          const uint8_t* line = Vdrop + (((size_t)item_f * pc_pad + (size_t)item_pb * BLOCK_M) * C) * (I8 ? 1 : 2) +
+                                (size_t)ks * kRowBytes;
+          const size_t pitch = (size_t)C * (I8 ? 1 : 2);
+#pragma unroll
+          for (int r = 0; r < BLOCK_M / 32; ++r) l2_discard_line(line + (size_t)(r * 32 + lane) * pitch);
+        }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
@@ -229,10 +245,12 @@ int launch_n(int sms, const void* V, const void* U, float* M, int nfreq, int pc,
   if (!make_map_3d(&tmV, dt, esize, V, C, pc, (long long)pc_pad * C, nfreq, BLOCK_K, BLOCK_M) ||
       !make_map_3d(&tmU, dt, esize, U, C, K, (long long)K * C, nfreq, BLOCK_K, BLOCK_N))
     return (int)cudaErrorUnknown;
-  const long long items = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M) * ((K + BLOCK_N - 1) / BLOCK_N);
-  const int grid = (int)(items < sms ? items : sms);
-  gemm_tcgen05_kernel<BLOCK_N, I8><<<grid, kThreads, L::kTotal, stream>>>(tmV, tmU, M, nfreq, pc, pc_pad, C, K, status);
-  return (int)cudaGetLastError();
+  const long long pairs = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M);
+  const int grid = (int)(pairs < sms ? pairs : sms);
+  // V may be dropped from the L2 after its last read when the pieces read are whole 128-byte lines
+  const bool drop = ((size_t)C * esize) % kRowBytes == 0 && (reinterpret_cast<uintptr_t>(V) % kRowBytes) == 0;
+  return (int)launch_overlapped(gemm_tcgen05_kernel<BLOCK_N, I8>, grid, kThreads, L::kTotal, stream, tmV, tmU, M, nfreq,
+                                pc, pc_pad, C, K, status, drop ? (const uint8_t*)V : (const uint8_t*)nullptr);
 }
 
 }  // namespace

@@ -144,14 +144,18 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
   bool timed_out = false;
+  // the constant Kronecker table belongs to the plan: it may be fetched while the preceding
+  // kernel of the stream is still draining; everything else waits for that kernel
+  if (warp == 0 && lane == 0) {
+    mbar_expect_tx(kron_bar, Cfg::kKronBytes);
+    for (int b = 0; b < 2 * Cfg::KA; ++b)
+      tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, &tmKron, kron_bar, 0, b * Cfg::NFP);
+  }
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp < kProdWarps) {
     // ---------------- TMA producers
-    if (warp == 0 && lane == 0) {
-      mbar_expect_tx(kron_bar, Cfg::kKronBytes);
-      for (int b = 0; b < 2 * Cfg::KA; ++b)
-        tma_load_2d(kron + (size_t)b * Cfg::NFP * 128, &tmKron, kron_bar, 0, b * Cfg::NFP);
-    }
     for (uint32_t local = warp; local < n_local && !timed_out; local += kProdWarps) {
       const unsigned u = blockIdx.x + local * gridDim.x;
       const int cblk = (int)(u % (unsigned)CB);
@@ -319,9 +323,8 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long 
   const int sms = plan->sm_count;
   const long long units = (long long)pc * ((g.C + 127) / 128);
   const int grid = (int)(units < sms ? units : sms);
-  input_transform_tc_kernel<M, QMODE, R><<<grid, kTcThreads, Cfg::kTotal, stream>>>(
-      tmX, tmK, V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev, qslot);
-  return (int)cudaGetLastError();
+  return (int)launch_overlapped(input_transform_tc_kernel<M, QMODE, R>, grid, kTcThreads, Cfg::kTotal, stream, tmX, tmK,
+                                V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev, qslot);
 }
 
 }  // namespace

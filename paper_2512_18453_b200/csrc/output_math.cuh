@@ -103,6 +103,18 @@ struct OutputTile {
   }
 };
 
+// Streaming stores of y (written once, not read again by this library): evict-first in the caches,
+// so that the lines of M the kernel has yet to read are not pushed out by its own output.
+__device__ __forceinline__ void vstore_cs(__half* p, float v) {
+  __stcs(reinterpret_cast<unsigned short*>(p), __half_as_ushort(__float2half_rn(v)));
+}
+__device__ __forceinline__ void vstore_cs(__half* p, float2 v) {
+  const __half2 h = __floats2half2_rn(v.x, v.y);
+  __stcs(reinterpret_cast<unsigned*>(p), *reinterpret_cast<const unsigned*>(&h));
+}
+__device__ __forceinline__ void vstore_cs(float* p, float v) { __stcs(p, v); }
+__device__ __forceinline__ void vstore_cs(float* p, float2 v) { __stcs(reinterpret_cast<float2*>(p), v); }
+
 // Round Y to the storage type and store the m x m outputs of one (tile, filter): pixel (i, j)
 // goes to dst + (i * W + j) * K.  rows / cols = how many of the tile's rows / columns lie inside
 // the image (m for an interior tile: no per-store predicate then).  ReLU keeps NaN and +inf.
@@ -116,7 +128,7 @@ __device__ __forceinline__ void store_tile(const V (&Y)[M][M], T* dst, size_t ro
       T* p = dst;
 #pragma unroll
       for (int j = 0; j < M; ++j) {
-        vstore(p, vmax_lo(Y[i][j], lo));
+        vstore_cs(p, vmax_lo(Y[i][j], lo));
         p += K;
       }
       dst += row_stride;
@@ -128,7 +140,7 @@ __device__ __forceinline__ void store_tile(const V (&Y)[M][M], T* dst, size_t ro
         T* p = dst;
 #pragma unroll
         for (int j = 0; j < M; ++j) {
-          if (j < cols) vstore(p, vmax_lo(Y[i][j], lo));
+          if (j < cols) vstore_cs(p, vmax_lo(Y[i][j], lo));
           p += K;
         }
       }

@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(kOtThreads, 1)
 output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
                             T* __restrict__ y, int H, int W, int K, int Th, int Tw, long long p0, int pc,
                             int pc_pad, int relu, int* __restrict__ status, const float* __restrict__ scale_U,
-                            const float* __restrict__ scale_V) {
+                            const float* __restrict__ scale_V, const float* __restrict__ Mbase) {
   using Cfg = OtCfg<M, VEC, R>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kUnitK = 16 * VEC;                    // filters per unit
@@ -76,6 +76,8 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
   }
   __syncthreads();
   bool timed_out = false;
+  pdl_launch_dependents();       // the set-up above may overlap the tail of the preceding kernel
+  pdl_wait();
 
   if (warp == 0) {
     // ---------------- TMA producer
@@ -120,6 +122,15 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
       OutputTile<M, SYM, VEC, QUANT, R>{cf, sb_even, sb_odd, qs}.run(Y);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[stage]);
+      // This unit was the only reader of its box of M (scratch): drop the lines from the L2 so
+      // that the ones still dirty there are never written back to device memory.
+      {
+        const int k4 = K >> 2;
+        for (int i = w * 32 + lane; i < Cfg::NF * Cfg::kQuads; i += 128) {
+          const int f = i / Cfg::kQuads, kq_abs = kg * Cfg::kQuads + i % Cfg::kQuads;
+          if (kq_abs < k4) l2_discard_line(Mbase + (((size_t)f * k4 + kq_abs) * pc_pad + (size_t)tg * 8) * 4);
+        }
+      }
 
       const int pl = tg * 8 + t;
       if (pl < pc && k < K) {
@@ -140,15 +151,15 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
 }
 
 template <int M, typename T, bool SYM, int VEC, bool QUANT, int R = 3>
-int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, void* y, long long p0, int pc,
+int launch_one(const nova_plan* plan, const Geom& g, const CUtensorMap& tmM, const float* Mb, void* y, long long p0, int pc,
                int pc_pad, int relu, const float* scale_U, const float* scale_V, cudaStream_t stream) {
   using Cfg = OtCfg<M, VEC, R>;
   if (cudaError_t e = allow_dynamic_smem(output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R>, Cfg::kTotal); e != cudaSuccess) return (int)e;
   const long long units = (long long)(pc_pad / 8) * ((g.K + 16 * VEC - 1) / (16 * VEC));
   const int grid = (int)(units < plan->sm_count ? units : plan->sm_count);
-  output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R><<<grid, kOtThreads, Cfg::kTotal, stream>>>(
-      tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu, plan->status_dev, scale_U, scale_V);
-  return (int)cudaGetLastError();
+  return (int)launch_overlapped(output_transform_tma_kernel<M, T, SYM, VEC, QUANT, R>, grid, kOtThreads, Cfg::kTotal,
+                                stream, tmM, plan->kcoefs, (T*)y, g.H, g.W, g.K, g.Th, g.Tw, p0, pc, pc_pad, relu,
+                                plan->status_dev, scale_U, scale_V, Mb);
 }
 
 template <int M, int R = 3>
@@ -168,7 +179,7 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* Mb, void* y, long
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return (int)cudaErrorUnknown;
   if (plan->mode == NOVA_FP32) return (int)cudaErrorInvalidValue;   // the fp32 mode has its own transforms
-#define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q, R>(plan, g, tmM, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
+#define NOVA_OT(TT, SYMV, Q) launch_one<M, TT, SYMV, VEC, Q, R>(plan, g, tmM, (const float*)Mb, y, p0, pc, pc_pad, relu, scale_U, scale_V, stream)
   if (scale_U)                                        // int8 pipeline: M holds int32 sums
     return plan->symmetric ? NOVA_OT(__half, true, true) : NOVA_OT(__half, false, true);
   return plan->symmetric ? NOVA_OT(__half, true, false) : NOVA_OT(__half, false, false);

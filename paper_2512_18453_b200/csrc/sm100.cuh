@@ -250,6 +250,20 @@ __host__ __device__ constexpr uint32_t umma_idesc_f16_amn(int M, int N) {
   return umma_idesc_f16(M, N) | (1u << 15);
 }
 
+// Tell the L2 that the 128-byte line at `p` (128-byte aligned, global memory) holds nothing of
+// value any more: if the line is resident and dirty it is dropped instead of written back.  Used
+// on scratch tensors right after their only reader has fetched them; the next reader of such a
+// line must be preceded by a writer.
+__device__ __forceinline__ void l2_discard_line(const void* p) {
+  asm volatile("discard.global.L2 [%0], 128;" ::"l"(p) : "memory");
+}
+
+// Programmatic dependent launch.  pdl_launch_dependents: the next kernel of the stream may be
+// scheduled as soon as every CTA of this grid has said so (or exited).  pdl_wait: block until
+// the kernels this grid depends on have completed and their memory operations are visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot_smem)),
                "r"(cols)
