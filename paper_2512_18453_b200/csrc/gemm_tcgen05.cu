@@ -48,7 +48,7 @@ template <int BLOCK_N, bool I8>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
                     float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
-                    int* __restrict__ status, const uint8_t* __restrict__ Vdrop) {
+                    int* __restrict__ status, const uint8_t* __restrict__ Vdrop, int f_major) {
   using L = SmemLayout<BLOCK_N>;
   constexpr int BLOCK_K = I8 ? kRowBytes : kRowBytes / 2;   // elements of K per stage
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
@@ -69,7 +69,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   // The work list is (row block, frequency), the row block outermost and DESCENDING: the input
   // transform wrote V in ascending tile order, so the highest row blocks are the ones still in
   // L2; and the row blocks this kernel finishes last - the lowest - are the ones the output
-  // transform reads first.  Pair i of this CTA is pair blockIdx.x + i * gridDim.x; the CTA runs
+  // transform reads first.  With f_major the frequency is outermost instead (see the launcher).
+  // Pair i of this CTA is pair blockIdx.x + i * gridDim.x; the CTA runs
   // the pair's filter blocks one after the other (items), so that it is the only reader of the
   // pair's rows of V and knows when they have been read for the last time.
   const long long num_pairs = (long long)nfreq * num_pb;
@@ -77,8 +78,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const uint32_t n_local = pairs_local * (uint32_t)num_kb;
   auto item_of = [&](uint32_t local, int& pb, int& f, int& kb) {
     const unsigned pair = blockIdx.x + (local / (unsigned)num_kb) * gridDim.x;
-    pb = num_pb - 1 - (int)(pair / (unsigned)nfreq);
-    f = (int)(pair % (unsigned)nfreq);
+    if (f_major) { f = (int)(pair / (unsigned)num_pb); pb = num_pb - 1 - (int)(pair % (unsigned)num_pb); }
+    else { pb = num_pb - 1 - (int)(pair / (unsigned)nfreq); f = (int)(pair % (unsigned)nfreq); }
     kb = (int)(local % (unsigned)num_kb);
   };
 
@@ -247,10 +248,17 @@ int launch_n(int sms, const void* V, const void* U, float* M, int nfreq, int pc,
     return (int)cudaErrorUnknown;
   const long long pairs = (long long)nfreq * ((pc + BLOCK_M - 1) / BLOCK_M);
   const int grid = (int)(pairs < sms ? pairs : sms);
+  // Work order.  Row-block-major re-streams all of U once per row block; that is free while U
+  // stays in the L2 (8 MB at C = K = 256) and costs device-memory reads once it does not (52 MB at
+  // C = K = 512 with 100 frequencies: 164 MB read per launch).  Frequency-major lets the CTAs that
+  // run at the same time share each U tile in the L2, at the price of the row-block hand-over with
+  // the neighbouring kernels.  Measured: 93 -> 84 us per step at C = K = 512, no difference at 256,
+  // 7 % slower for a layer with K = 64 and 196 row blocks; hence the threshold on the size of U.
+  const bool f_major = (size_t)nfreq * K * C * esize > ((size_t)32 << 20);
   // V may be dropped from the L2 after its last read when the pieces read are whole 128-byte lines
   const bool drop = ((size_t)C * esize) % kRowBytes == 0 && (reinterpret_cast<uintptr_t>(V) % kRowBytes) == 0;
   return (int)launch_overlapped(gemm_tcgen05_kernel<BLOCK_N, I8>, grid, kThreads, L::kTotal, stream, tmV, tmU, M, nfreq,
-                                pc, pc_pad, C, K, status, drop ? (const uint8_t*)V : (const uint8_t*)nullptr);
+                                pc, pc_pad, C, K, status, drop ? (const uint8_t*)V : (const uint8_t*)nullptr, f_major ? 1 : 0);
 }
 
 }  // namespace

@@ -881,3 +881,24 @@ def test_r5_int8_path_matches_the_emulation(m, key, shape, coef):
     else:
         assert e_gpu <= 2.0 * e_emu, (e_gpu, e_emu)
         assert conv.rel_l2(y, ye.astype(np.float64)) <= 0.25 * e_emu + 1e-3
+
+
+def test_fabric_probe_runs_every_kind_and_reports_plausible_rates():
+    # the measurement aid behind the documented SM <-> L2 rates: every access kind completes on a small
+    # L2-resident buffer without a time-out and at a rate between 0.2 and 40 TB/s; bad arguments are refused
+    plan = nv.Plan(2, point_set("std", 2))
+    n = 16 << 20
+    src = torch.ones(n, dtype=torch.uint8, device="cuda")
+    dst = torch.empty(n, dtype=torch.uint8, device="cuda")
+    for kind in range(7):
+        ms = plan.probe_fabric(kind, src, dst, iters=5, ctas=148, depth=4)
+        moved = n * 5 * (2 if kind in (4, 6) else 1)
+        assert 0.2 < moved / (ms * 1e-3) / 1e12 < 40.0, (kind, ms)
+    assert plan.device_status() == 0
+    for bad in (dict(kind=7), dict(depth=0), dict(depth=13), dict(iters=0), dict(ctas=0)):
+        args = dict(kind=0, iters=1, ctas=8, depth=1)
+        args.update(bad)
+        with pytest.raises(nv.NovaError):
+            plan.probe_fabric(args.pop("kind"), src, dst, **args)
+    with pytest.raises(nv.NovaError):
+        plan.probe_fabric(0, src[:1000], dst[:1000])          # not a multiple of 16 KiB
