@@ -38,7 +38,9 @@ extern "C" {
  * projective (1:0) (Section 2.4, "Symbolic Verification"). */
 typedef struct { int64_t num, den; } nova_rat;
 
-/* Arithmetic mode.  NOVA_FP32: x, g, y and every intermediate are float.
+/* Arithmetic mode.  NOVA_FP32: x, g, y and the stored intermediates (U, V, M) are float; every
+ * stored element is one rounding of a sum carried in double (with float sums the F(8,3) tile
+ * would not reach a relative error of 1e-4 even on well-conditioned points); accuracy path.
  * NOVA_FP16_F32ACC: x, g, y are IEEE half; transforms are evaluated in float
  * and rounded once to half; the transformed-domain product accumulates in
  * float (Section 5.1 "FP16 Setup"; Appendix "Float16 Precision Analysis"). */
@@ -206,7 +208,8 @@ size_t nova_conv2d_min_workspace_bytes(const nova_plan* plan, int N, int H, int 
  * x_dev [N,H,W,C], y_dev [N,H,W,K] in the storage type, 16-byte aligned;
  * U_dev from nova_filter_transform with the same plan, K and C.
  * workspace_dev: 256-byte aligned scratch of workspace_bytes; contents are
- * undefined afterwards; calls sharing a workspace must be stream-ordered.
+ * undefined afterwards (the kernels tell the L2 to drop its lines unwritten once
+ * they have been read); calls sharing a workspace must be stream-ordered.
  */
 int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
                     int N, int H, int W, int C, int K,
