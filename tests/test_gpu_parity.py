@@ -524,6 +524,19 @@ def test_cfg5_vgg16_stack_f8_nova_two_images():
         assert e_gpu <= 2.0 * e_emu
 
 
+def test_cfg5_first_two_layers_tile_by_tile():
+    """The two 224 x 224 layers of the stack (C = 8 with the CUDA-core input transform, then C = K = 64)
+    on one image, each judged on its own like any single layer: against the direct convolution, and
+    tile by tile against the emulation (the stack test above can only judge the final features)."""
+    x, weights = make_vgg_inputs(1)
+    pts = point_set("nova", 8)
+    y, _, _ = gpu_conv(x, weights[0], 8, pts, nv.FP16_F32ACC)
+    check_fp16(y, x, weights[0], 8, pts)
+    a = conv.winograd_conv_emulated(x, weights[0], 8, pts, "fp16", apply_relu=True)     # layer 2's input
+    y, _, _ = gpu_conv(a, weights[1], 8, pts, nv.FP16_F32ACC)
+    check_fp16(y, a, weights[1], 8, pts)
+
+
 # ---------------------------------------------------------------- diagonal rescaling (D_A D_G D_B = I)
 def _pow2_scales(m, pts):
     from oracle import toom_cook as tc
