@@ -47,6 +47,7 @@ struct nova_plan {
   int* status_dev;                        // device status word (null without a device)
   int device;                             // device that owns status_dev
   int sm_count;                           // multiprocessors of that device
+  int l2_bytes;                           // size of its L2
 };
 
 namespace nova {

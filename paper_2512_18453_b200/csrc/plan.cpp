@@ -434,6 +434,7 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
         pl->status_dev = w;
         pl->device = dev;
         cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&pl->l2_bytes, cudaDevAttrL2CacheSize, dev);
       }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
       if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
