@@ -259,6 +259,47 @@ def run_fabric(args):
     print(json.dumps({"fabric": rows}))
 
 
+def run_wait_profile(args):
+    """Where the warps of the transformed-domain product kernel spend their time: 20 calls of the
+    workload with the wait-profiling variant of that kernel, the counters of the last one printed
+    as shares of each warp role's total.  A measurement aid; its step time is not a bench value."""
+    import torch
+    import paper_2512_18453_b200 as nv
+    from synth import point_set, make_conv_inputs
+    torch.cuda.set_device(0)
+    c = workload(args.workload)
+    plan = nv.Plan(c.m, point_set(args.points, c.m), nv.FP16_F32ACC)
+    x_np, g_np = make_conv_inputs(c.N, c.H, c.W, c.C, c.K, c.dtype, c.relu_inputs, c.he_weights, c.seed)
+    x, g = torch.from_numpy(x_np).cuda(), torch.from_numpy(g_np).cuda()
+    U = plan.filter_transform(g)
+    y = torch.empty(c.N, c.H, c.W, c.K, dtype=torch.float16, device="cuda")
+    ws = torch.empty(plan.workspace_bytes(c.N, c.H, c.W, c.C, c.K), dtype=torch.uint8, device="cuda")
+    out = {}
+    for name, flags in (("plain", 0), ("profiled", nv.PROFILE_WAITS)):
+        for _ in range(5):
+            plan.conv2d(x, U, y=y, workspace=ws, flags=flags)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(20):
+            plan.conv2d(x, U, y=y, workspace=ws, flags=flags)
+        e1.record()
+        torch.cuda.synchronize()
+        out["us_per_step_" + name] = e0.elapsed_time(e1) / 20 * 1e3
+    w = plan.wait_profile()
+    assert plan.device_status() == 0
+    out["workload"] = c.name
+    out["cycles_per_cta"] = w
+    out["shares"] = {
+        "producer_waiting_for_a_free_stage": w["producer_wait_stage"] / max(w["producer_total"], 1.0),
+        "mma_waiting_for_operands": w["mma_wait_operands"] / max(w["mma_total"], 1.0),
+        "mma_waiting_for_a_free_accumulator": w["mma_wait_accumulator"] / max(w["mma_total"], 1.0),
+        "epilogue_waiting_for_an_accumulator": w["epilogue_wait_accumulator"] / max(w["epilogue_total"], 1.0),
+        "epilogue_storing": 1.0 - w["epilogue_wait_accumulator"] / max(w["epilogue_total"], 1.0),
+    }
+    print(json.dumps({"wait_profile": out}))
+
+
 def rank_seed(base_seed, rank):
     """Each rank draws its own batch (weak scaling): the seed is offset by the rank."""
     return base_seed + 100 * rank
@@ -812,6 +853,8 @@ def main():
     ap.add_argument("--launch", default="graph", choices=["graph", "direct"])
     ap.add_argument("--fabric", action="store_true",
                     help="measure the SM <-> L2 / HBM rates by access kind (nova_probe_fabric) and print them")
+    ap.add_argument("--wait-profile", action="store_true",
+                    help="print where the product kernel's warps wait (NOVA_PROFILE_WAITS; not a bench value)")
     ap.add_argument("--images", type=int, default=0, help="override the batch size (profiling aid)")
     ap.add_argument("--accuracy", action="store_true",
                     help="report rel-L2 per point set (and per rescaled variant) even with --no-cpu-baseline")
@@ -831,6 +874,8 @@ def main():
         run_reference(args)
     elif args.fabric:
         run_fabric(args)
+    elif args.wait_profile:
+        run_wait_profile(args)
     elif args.workload == "cfg5":
         run_vgg(args)
     elif args.int8:

@@ -55,6 +55,9 @@ enum {
   NOVA_RELU = 1,            /* y = (v < 0) ? 0 : v after the output transform */
   NOVA_GEMM_SIMT = 1 << 8,  /* force the CUDA-core product kernel (fp16 mode; testing) */
   NOVA_GEMM_TCGEN05 = 2 << 8, /* force the tcgen05 tensor-core product kernel */
+  NOVA_PROFILE_WAITS = 1 << 13, /* measurement aid: the tensor-core product kernel (half mode, K > 128) runs in a
+                                   variant that sums the cycles its warps spend waiting; read them with
+                                   nova_plan_wait_profile.  A few per cent slower; results unchanged */
   NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
                                    where the tensor-core formulation applies, the output transform
                                    without TMA staging (testing) */
@@ -349,6 +352,19 @@ int nova_selftest_wait_timeout(const nova_plan* plan, unsigned limit_ms, unsigne
  */
 int nova_probe_fabric(const nova_plan* plan, int kind, const void* src_dev, void* dst_dev, size_t bytes,
                       int iters, int ctas, int depth, float* ms_host, nova_stream stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): where the transformed-domain product kernel of the
+ * last nova_conv2d_fwd call with NOVA_PROFILE_WAITS spent its time.  cycles_host receives 9 doubles,
+ * SM clock cycles averaged over the CTAs that ran:
+ *   [0] TMA producer warp waiting for a free ring stage      [1] its total
+ *   [2] MMA warp waiting for a free TMEM accumulator         [3] MMA warp waiting for operands in the ring
+ *   [4] MMA warp total                                       [5] an epilogue warp waiting for a finished accumulator
+ *   [6] that epilogue warp's total (the rest of it is spent storing M)
+ *   [7] work items per CTA                                   [8] number of CTAs
+ * Synchronises `stream`.  The counters are the plan's: not thread-safe against a concurrent profiled call.
+ */
+int nova_plan_wait_profile(const nova_plan* plan, double* cycles_host, nova_stream stream);
 
 /* 2x2 max pooling, stride 2, NHWC, H and W even, C % 8 == 0 (used between the
  * blocks of a VGG-style stack; not part of the paper's method).  `mode`

@@ -11,6 +11,7 @@ RELU = 1
 GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
 TRANSFORM_SIMT = 1 << 10
+PROFILE_WAITS = 1 << 13
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
@@ -20,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "nova_status_string", "nova_conv2d_fwd_static", "nova_plan_frequency_order", "nova_last_cuda_error",
     "nova_plan_create_scaled", "nova_plan_create_f64", "nova_snap_to_rational", "nova_verify_decomposition",
     "nova_plan_get_matrices_rational", "nova_plan_kappa_matrices", "nova_symmetric_search",
-    "nova_selftest_wait_timeout", "nova_probe_fabric",
+    "nova_selftest_wait_timeout", "nova_probe_fabric", "nova_plan_wait_profile",
     "nova_filter_transform_int8_bytes", "nova_filter_transform_int8", "nova_conv2d_int8_workspace_bytes",
     "nova_conv2d_fwd_int8", "nova_conv2d_fwd_int8_timed",
 )
@@ -80,6 +81,8 @@ def lib():
     L.nova_plan_get_device_tables.restype = i
     L.nova_plan_frequency_order.argtypes = [vp, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.nova_plan_frequency_order.restype = i
+    L.nova_plan_wait_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
+    L.nova_plan_wait_profile.restype = i
     L.nova_probe_fabric.argtypes = [vp, i, vp, vp, sz, i, i, i, fp, vp]
     L.nova_probe_fabric.restype = i
     L.nova_last_cuda_error.argtypes = []
@@ -264,6 +267,14 @@ class Plan:
         sym = ctypes.c_int()
         _check(lib().nova_plan_frequency_order(self._h, perm, ctypes.byref(sym)), "nova_plan_frequency_order")
         return list(perm), bool(sym.value)
+
+    def wait_profile(self):
+        """nova_plan_wait_profile: dict of mean SM cycles per CTA of the last product kernel run with PROFILE_WAITS."""
+        out = (ctypes.c_double * 9)()
+        _check(lib().nova_plan_wait_profile(self._h, out, _stream()), "nova_plan_wait_profile")
+        names = ("producer_wait_stage", "producer_total", "mma_wait_accumulator", "mma_wait_operands", "mma_total",
+                 "epilogue_wait_accumulator", "epilogue_total", "items_per_cta", "ctas")
+        return dict(zip(names, list(out)))
 
     def probe_fabric(self, kind, src, dst, iters=10, ctas=148, depth=8):
         """nova_probe_fabric on two uint8 CUDA tensors of equal size; returns milliseconds for `iters` passes."""

@@ -149,7 +149,8 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
                 : launch_input_transform(p, g, x, Vb, p0, pc, c.pc_pad, stream))
       return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 1], s);
-    const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream)
+    const int e = tc ? launch_gemm_tcgen05(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, p->status_dev, stream,
+                                           (flags & NOVA_PROFILE_WAITS) ? p->prof_dev : nullptr)
                      : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
@@ -459,6 +460,32 @@ extern "C" int nova_selftest_wait_timeout(const nova_plan* p, unsigned limit_ms,
                         cudaStreamSynchronize(s) != cudaSuccess))
     st = NOVA_ERR_CUDA;
   cudaFree(w);
+  return st;
+}
+
+extern "C" int nova_plan_wait_profile(const nova_plan* p, double* cycles_host, nova_stream stream) {
+  if (!p || !cycles_host) return NOVA_ERR_INVALID_ARG;
+  if (!p->prof_dev || p->sm_count <= 0) return NOVA_ERR_CUDA;
+  if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int n = p->sm_count;
+  unsigned long long* h = new unsigned long long[(size_t)n * 8];
+  int st = NOVA_OK;
+  if (cudaMemcpyAsync(h, p->prof_dev, sizeof(unsigned long long) * n * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    st = NOVA_ERR_CUDA;
+  if (st == NOVA_OK) {
+    int ctas = 0;                                      // CTAs that ran: those with a non-zero item count
+    for (int k = 0; k < 8; ++k) cycles_host[k] = 0.0;
+    for (int i = 0; i < n; ++i) {
+      if (h[(size_t)i * 8 + 7] == 0) continue;
+      ++ctas;
+      for (int k = 0; k < 8; ++k) cycles_host[k] += (double)h[(size_t)i * 8 + k];
+    }
+    for (int k = 0; k < 8; ++k) cycles_host[k] = ctas ? cycles_host[k] / ctas : 0.0;
+    cycles_host[8] = (double)ctas;
+  }
+  delete[] h;
   return st;
 }
 

@@ -44,11 +44,21 @@ struct SmemLayout {
   static constexpr int kTotal = kBarrierOffset + 256 + 1024;     // barriers + alignment slack
 };
 
-template <int BLOCK_N, bool I8>
+// Measurement aid: sums of clock64() spent in (or around) the waits of one warp.  With ON = false
+// every member is empty and the kernel is the production one.
+template <bool ON>
+struct WaitClock {
+  long long sum = 0, t0 = 0;
+  __device__ __forceinline__ void start() { if constexpr (ON) t0 = clock64(); }
+  __device__ __forceinline__ void stop() { if constexpr (ON) sum += clock64() - t0; }
+};
+
+template <int BLOCK_N, bool I8, bool PROF = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmU,
                     float* __restrict__ Mo, int nfreq, int pc, int pc_pad, int C, int K,
-                    int* __restrict__ status, const uint8_t* __restrict__ Vdrop, int f_major, int keep_pct) {
+                    int* __restrict__ status, const uint8_t* __restrict__ Vdrop, int f_major, int keep_pct,
+                    unsigned long long* __restrict__ prof) {
   using L = SmemLayout<BLOCK_N>;
   constexpr int BLOCK_K = I8 ? kRowBytes : kRowBytes / 2;   // elements of K per stage
   constexpr uint32_t kTmemCols = 2 * BLOCK_N;       // two accumulators; 128, 256 or 512
@@ -107,12 +117,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 
   if (warp == 0) {
     // ---------------- TMA producer
+    WaitClock<PROF> w_empty, total;
+    total.start();
     uint32_t stage = 0, phase = 0;
     for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
       int pb, f, kb;
       item_of(local, pb, f, kb);
       for (int ks = 0; ks < num_ks; ++ks) {
+        w_empty.start();
         if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
+        w_empty.stop();
         if (lane == 0) {
           uint8_t* sa = smem + stage * L::kStageBytes;
           uint8_t* sb = sa + L::kABytes;
@@ -124,19 +138,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
+    if constexpr (PROF) {
+      total.stop();
+      if (lane == 0) { prof[blockIdx.x * 8 + 0] = w_empty.sum; prof[blockIdx.x * 8 + 1] = total.sum; }
+    }
   } else if (warp == 1) {
     // ---------------- MMA issuer
     constexpr uint32_t idesc = I8 ? umma_idesc_i8(BLOCK_M, BLOCK_N) : umma_idesc_f16(BLOCK_M, BLOCK_N);
+    WaitClock<PROF> w_acc, w_ops, total;
+    total.start();
     uint32_t stage = 0, phase = 0;
     for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+      w_acc.start();
       if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) { timed_out = true; break; }
+      w_acc.stop();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tmem_d = tmem_base + acc * BLOCK_N;
       int item_pb, item_f, item_kb;
       item_of(local, item_pb, item_f, item_kb);
       for (int ks = 0; ks < num_ks; ++ks) {
+        w_ops.start();
         if (!mbar_wait_warp(&full_bar[stage], phase, abort_flag)) { timed_out = true; break; }
+        w_ops.stop();
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (lane == 0) {
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
@@ -170,6 +194,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
+    if constexpr (PROF) {
+      total.stop();
+      if (lane == 0) {
+        prof[blockIdx.x * 8 + 2] = w_acc.sum; prof[blockIdx.x * 8 + 3] = w_ops.sum; prof[blockIdx.x * 8 + 4] = total.sum;
+        prof[blockIdx.x * 8 + 7] = n_local;
+      }
+    }
   } else {
     // ---------------- epilogue (warps 2..9); a warp may only read TMEM lanes 32*(warp%4)..+31.
     // Rows >= pc of the last row block are zeros (the TMA loads of V fill them) and land in the
@@ -178,11 +209,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int half = (warp - 2) >> 2;                    // which half of the BLOCK_N columns
     constexpr int HALF_N = BLOCK_N / 2;
     const int k4 = K >> 2;
+    WaitClock<PROF> w_full, total;
+    total.start();
     for (uint32_t local = 0; local < n_local && !timed_out; ++local) {
       int pb, f, kb;
       item_of(local, pb, f, kb);
       const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+      w_full.start();
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
+      w_full.stop();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       // M is larger than the L2 on the layers that matter, and the output transform reads the row
       // blocks written last (the lowest) first: the share of row blocks that can still be resident
@@ -210,6 +245,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+    }
+    if constexpr (PROF) {
+      total.stop();
+      if (warp == 2 && lane == 0) { prof[blockIdx.x * 8 + 5] = w_full.sum; prof[blockIdx.x * 8 + 6] = total.sum; }
     }
   }
 
@@ -243,7 +282,7 @@ bool make_map_3d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void
 
 template <int BLOCK_N, bool I8>
 int launch_n(int sms, int l2_bytes, const void* V, const void* U, float* M, int nfreq, int pc, int pc_pad, int C, int K,
-             int* status, cudaStream_t stream) {
+             int* status, cudaStream_t stream, unsigned long long* prof = nullptr) {
   using L = SmemLayout<BLOCK_N>;
   if (cudaError_t e = allow_dynamic_smem(gemm_tcgen05_kernel<BLOCK_N, I8>, L::kTotal); e != cudaSuccess) return (int)e;
   CUtensorMap tmV, tmU;
@@ -270,17 +309,28 @@ int launch_n(int sms, int l2_bytes, const void* V, const void* U, float* M, int 
   if (keep_pct > 100) keep_pct = 100;
   // V may be dropped from the L2 after its last read when the pieces read are whole 128-byte lines
   const bool drop = ((size_t)C * esize) % kRowBytes == 0 && (reinterpret_cast<uintptr_t>(V) % kRowBytes) == 0;
+  const uint8_t* vdrop = drop ? (const uint8_t*)V : (const uint8_t*)nullptr;
+  // the wait-profiling variant exists for the half product with 256-wide filter blocks only
+  if constexpr (BLOCK_N == 256 && !I8) {
+    if (prof) {
+      if (cudaError_t e = allow_dynamic_smem(gemm_tcgen05_kernel<BLOCK_N, I8, true>, L::kTotal); e != cudaSuccess) return (int)e;
+      // CTAs beyond this launch's grid must read as "did not run"
+      if (cudaError_t e = cudaMemsetAsync(prof, 0, sizeof(unsigned long long) * 8 * sms, stream); e != cudaSuccess) return (int)e;
+      return (int)launch_overlapped(gemm_tcgen05_kernel<BLOCK_N, I8, true>, grid, kThreads, L::kTotal, stream, tmV, tmU, M,
+                                    nfreq, pc, pc_pad, C, K, status, vdrop, f_major ? 1 : 0, keep_pct, prof);
+    }
+  }
   return (int)launch_overlapped(gemm_tcgen05_kernel<BLOCK_N, I8>, grid, kThreads, L::kTotal, stream, tmV, tmU, M, nfreq,
-                                pc, pc_pad, C, K, status, drop ? (const uint8_t*)V : (const uint8_t*)nullptr, f_major ? 1 : 0, keep_pct);
+                                pc, pc_pad, C, K, status, vdrop, f_major ? 1 : 0, keep_pct, (unsigned long long*)nullptr);
 }
 
 }  // namespace
 
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M, int nfreq, int pc,
-                        int pc_pad, int C, int K, int* status_dev, void* stream) {
+                        int pc_pad, int C, int K, int* status_dev, void* stream, unsigned long long* prof) {
   cudaStream_t s = (cudaStream_t)stream;
   const int sms = plan->sm_count;
-  if (K > 128) return launch_n<256, false>(sms, plan->l2_bytes, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
+  if (K > 128) return launch_n<256, false>(sms, plan->l2_bytes, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s, prof);
   if (K > 64) return launch_n<128, false>(sms, plan->l2_bytes, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
   return launch_n<64, false>(sms, plan->l2_bytes, V, U, M, nfreq, pc, pc_pad, C, K, status_dev, s);
 }

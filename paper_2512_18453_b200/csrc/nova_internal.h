@@ -48,6 +48,7 @@ struct nova_plan {
   int device;                             // device that owns status_dev
   int sm_count;                           // multiprocessors of that device
   int l2_bytes;                           // size of its L2
+  unsigned long long* prof_dev;           // 8 wait counters per multiprocessor (NOVA_PROFILE_WAITS; may be null)
 };
 
 namespace nova {
@@ -101,8 +102,10 @@ int launch_output_transform_f32(const nova_plan* plan, const Geom& g, const void
                                 int pc_pad, int relu, void* stream);
 int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float* M,
                      int nfreq, int pc, int pc_pad, int C, int K, void* stream);
+// prof non-null (K > 128, half operands): the wait-profiling variant writes 8 counters per CTA there
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M,
-                        int nfreq, int pc, int pc_pad, int C, int K, int* status_dev, void* stream);
+                        int nfreq, int pc, int pc_pad, int C, int K, int* status_dev, void* stream,
+                        unsigned long long* prof = nullptr);
 int launch_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode, void* stream);
 
 }  // namespace nova

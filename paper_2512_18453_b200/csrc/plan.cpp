@@ -436,6 +436,14 @@ int create_impl(int m, int r, const nova_rat* points, int n, const nova_rat* sca
         cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev);
         cudaDeviceGetAttribute(&pl->l2_bytes, cudaDevAttrL2CacheSize, dev);
       }
+      if (pl->status_dev && pl->sm_count > 0) {
+        unsigned long long* pd = nullptr;
+        const size_t nb = (size_t)pl->sm_count * 8 * sizeof(unsigned long long);
+        if (cudaMalloc((void**)&pd, nb) == cudaSuccess) {
+          cudaMemset(pd, 0, nb);
+          pl->prof_dev = pd;
+        }
+      }
       // Kronecker table of the tensor-core input transform (half mode, half-rounded tables).
       if (pl->status_dev && mode == NOVA_FP16_F32ACC && coef == NOVA_COEF_ROUND_TO_MODE) {
         std::vector<unsigned short> img(nova::kron_table_halves(n));
@@ -613,6 +621,7 @@ extern "C" void nova_plan_destroy(nova_plan* plan) {
   if (!plan) return;
   if (plan->status_dev) cudaFree(plan->status_dev);
   if (plan->kron_dev) cudaFree(plan->kron_dev);
+  if (plan->prof_dev) cudaFree(plan->prof_dev);
   delete plan;
 }
 

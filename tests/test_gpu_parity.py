@@ -915,3 +915,26 @@ def test_fabric_probe_runs_every_kind_and_reports_plausible_rates():
             plan.probe_fabric(args.pop("kind"), src, dst, **args)
     with pytest.raises(nv.NovaError):
         plan.probe_fabric(0, src[:1000], dst[:1000])          # not a multiple of 16 KiB
+
+
+def test_wait_profiling_variant_gives_the_same_bits_and_consistent_counters():
+    # the measurement aid NOVA_PROFILE_WAITS: the product kernel's profiled variant writes the same y, and
+    # its counters are consistent (waits within totals, every CTA ran, items add up to pairs x filter blocks)
+    m, N, H, W, C, K = 6, 8, 56, 56, 256, 256
+    x_np, g_np = make_conv_inputs(N, H, W, C, K, "fp16", True, True, 77)
+    plan = nv.Plan(m, point_set("nova", m))
+    x, g = torch.from_numpy(x_np).cuda(), torch.from_numpy(g_np).cuda()
+    U = plan.filter_transform(g)
+    y0 = plan.conv2d(x, U)
+    y1 = plan.conv2d(x, U, flags=nv.PROFILE_WAITS)
+    w = plan.wait_profile()
+    assert plan.device_status() == 0
+    assert torch.equal(y0.view(torch.int16), y1.view(torch.int16))
+    assert 0 <= w["producer_wait_stage"] <= w["producer_total"]
+    assert 0 <= w["mma_wait_accumulator"] + w["mma_wait_operands"] <= w["mma_total"]
+    assert 0 <= w["epilogue_wait_accumulator"] <= w["epilogue_total"]
+    assert w["epilogue_total"] > 0 and w["mma_total"] > 0
+    tiles = N * ((H + m - 1) // m) * ((W + m - 1) // m)
+    pairs = (m + 2) ** 2 * ((tiles + 127) // 128)
+    assert w["ctas"] == min(pairs, torch.cuda.get_device_properties(0).multi_processor_count)
+    assert abs(w["items_per_cta"] * w["ctas"] - pairs * ((K + 255) // 256)) < 0.5
