@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnova.so")
-SOURCES = ["plan.cpp", "transforms.cu", "gemm_simt.cu", "fp32_path.cu", "gemm_tcgen05.cu", "input_transform_tc.cu", "output_transform_tma.cu", "fabric_probe.cu", "conv.cu"]
+SOURCES = ["plan.cpp", "transforms.cu", "gemm_simt.cu", "fp32_path.cu", "gemm_tcgen05.cu", "input_transform_tc.cu", "output_transform_tma.cu", "fabric_probe.cu", "fused_small_c.cu", "conv.cu"]
 
 
 def _nvcc():

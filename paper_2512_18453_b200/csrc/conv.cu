@@ -62,6 +62,13 @@ bool on_plan_device(const nova_plan* p) {
   return p->device >= 0 && cudaGetDevice(&dev) == cudaSuccess && dev == p->device;
 }
 
+// The one-kernel path for 8 input channels runs unless a flag asks for a particular kernel of the
+// three-kernel path.
+bool use_fused_small_c(const nova_plan* p, const Geom& g, int flags) {
+  const int forcing = NOVA_GEMM_SIMT | NOVA_GEMM_TCGEN05 | NOVA_TRANSFORM_SIMT | NOVA_PROFILE_WAITS;
+  return (flags & forcing) == 0 && fused_small_c_applies(p, g);
+}
+
 bool use_tcgen05(const nova_plan* p, int flags) {
   if (p->mode == NOVA_FP32) return false;
   return (flags & NOVA_GEMM_SIMT) == 0;
@@ -107,12 +114,12 @@ extern "C" size_t nova_conv2d_workspace_bytes(const nova_plan* p, int N, int H, 
 
 extern "C" int nova_conv2d_launch_count(const nova_plan* p, int N, int H, int W, int C, int K,
                                         size_t workspace_bytes, int flags) {
-  (void)flags;
   if (!p || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   Geom g = make_geom(p, N, H, W, C, K);
   Chunking c;
   if (!choose_chunking(p, g, workspace_bytes, &c)) return NOVA_ERR_WORKSPACE;
+  if (use_fused_small_c(p, g, flags)) return 1;
   return 3 * c.chunks;
 }
 
@@ -132,6 +139,13 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   Geom g = make_geom(p, N, H, W, C, K);
   Chunking c;
   if (!choose_chunking(p, g, ws_bytes, &c)) return NOVA_ERR_WORKSPACE;
+  if (use_fused_small_c(p, g, flags)) {
+    // steps 2-4 in one kernel, V and M kept on the SM: the workspace is not touched
+    if (ev) cudaEventRecord(ev[0], (cudaStream_t)stream);
+    if (launch_fused_small_c(p, g, x, U, y, (flags & NOVA_RELU) ? 1 : 0, stream)) return NOVA_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[1], (cudaStream_t)stream);
+    return NOVA_OK;
+  }
   const bool tc = use_tcgen05(p, flags);
   if (tc && !p->status_dev) return NOVA_ERR_CUDA;
   char* Vb = static_cast<char*>(ws);
@@ -178,6 +192,18 @@ extern "C" int nova_conv2d_fwd_timed(const nova_plan* p, const void* x, const vo
   if (!kernel_ms) return NOVA_ERR_INVALID_ARG;
   const int launches = nova_conv2d_launch_count(p, N, H, W, C, K, ws_bytes, flags);
   if (launches < 0) return launches;
+  if (launches == 1) {               // the one-kernel path: its time is reported as the product's
+    cudaEvent_t e2[2];
+    cudaEventCreate(&e2[0]);
+    cudaEventCreate(&e2[1]);
+    int st1 = conv2d_fwd_impl(p, x, U, y, N, H, W, C, K, ws, ws_bytes, flags, stream, e2);
+    if (st1 == NOVA_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st1 = NOVA_ERR_CUDA;
+    kernel_ms[0] = kernel_ms[1] = kernel_ms[2] = 0.f;
+    if (st1 == NOVA_OK) cudaEventElapsedTime(&kernel_ms[1], e2[0], e2[1]);
+    cudaEventDestroy(e2[0]);
+    cudaEventDestroy(e2[1]);
+    return st1;
+  }
   const int chunks = launches / 3;
   cudaEvent_t* ev = new cudaEvent_t[4 * chunks];
   for (int i = 0; i < 4 * chunks; ++i) cudaEventCreate(&ev[i]);

@@ -1,0 +1,297 @@
+// Section 2.1 steps 2-4 in ONE kernel for layers with 8 input channels (half mode, 3-tap filters):
+// V = B^T d B, M[f] = V[f] U[f]^T and Y = A^T M A for a group of 8 tiles at a time, with V and M
+// never leaving the SM.  The first layer of an image network is of this kind (3 colour channels
+// padded to 8).  There the three-kernel path is bound by its intermediate tensors alone - the
+// n*n*K floats of M per tile are 160 times the bytes of the tile's input patch - while the product
+// itself is tiny (8 channels), so it fits the register-level tensor-core instruction: one
+// mma.sync m16n8k8 per frequency gives M[f] for 8 tiles x 8 filters, the two results a thread
+// holds are the same tile's two adjacent filters, i.e. one packed-fp32 operand of the output
+// transform, whose n*n inputs per (tile, filter) are consumed row by row and never all alive.
+// (The TMEM-accumulator route of the large-C product kernel cannot do this: n*n frequencies x 8
+// filters already exceed an SM's 512 accumulator columns.)
+//
+// One CTA = 256 threads = 8 warps; the CTA keeps the transformed filters of its 64-filter block in
+// shared memory for its whole life and walks groups of 8 consecutive tiles:
+//   TMA      one n x n x 8-channel box per tile straight from x (out-of-range pixels read as 0:
+//            halo and ragged tiles), double buffered, issued one group ahead
+//   pass 1   B^T along the patch's rows index a, float, to shared memory       (tile, column, channel pair)
+//   pass 2   B^T along the columns index b, rounded once to half: V            (tile, row, channel pair)
+//   product  warp w: filters 8w..8w+7; per row xi of frequencies n mma.sync, then A^T along nu
+//            and the accumulation of Y = sum_xi A^T[.][xi] z_xi, all in registers (packed fp32)
+//   store    Y rounded to half into a shared-memory image of the 8 tiles x 64 filters, then
+//            16-byte streaming stores, 128 contiguous bytes per pixel
+// Rounding points are those of the three-kernel path: tables as the plan holds them, V evaluated
+// in float and rounded once to half, products of halves summed in float, Y evaluated in float and
+// rounded once to half.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "nova_internal.h"
+#include "output_math.cuh"
+#include "sm100.cuh"
+#include "tma_host.h"
+
+namespace nova {
+namespace {
+using namespace sm100;
+using namespace xf;
+
+constexpr int kThreads = 256;
+constexpr int kGroupTiles = 8;     // rows 0..7 of the m16n8k8 product (rows 8..15 are fed zeros)
+constexpr int kFilterBlock = 64;   // 8 warps x 8 filters
+
+template <int M>
+struct SmallCLayout {
+  static constexpr int N = M + 2;
+  static constexpr int kPatchBytes = N * N * 16;                        // one tile: [a][b][8 halves]
+  static constexpr int kPatchStride = (kPatchBytes + 127) & ~127;       // TMA destinations: 128-byte aligned
+  static constexpr int kUBytes = N * kFilterBlock * 4 * N * 4;          // [xi][filter][channel pair][nu] half2
+  static constexpr int kVBytes = N * kGroupTiles * 4 * N * 4;           // [xi][tile][channel pair][nu] half2
+  static constexpr int kTTile = N * N * 4 * 8 + 32;                     // [xi][b][channel pair] float2 (+32: banks)
+  static constexpr int kTBytes = kGroupTiles * kTTile;
+  static constexpr int kYTile = M * M * 128 + 16;                       // [i][j][64 filters] half (+16: banks)
+  static constexpr int kYBytes = kGroupTiles * kYTile;
+  static constexpr int kScratch = kTBytes > kYBytes ? kTBytes : kYBytes;   // T and the image of y share
+  static constexpr int kOffU = 0;
+  static constexpr int kOffPatch = kOffU + kUBytes;
+  static constexpr int kOffV = kOffPatch + 2 * kGroupTiles * kPatchStride;
+  static constexpr int kOffScratch = kOffV + kVBytes;
+  static constexpr int kOffBar = (kOffScratch + kScratch + 15) & ~15;
+  static constexpr int kTotal = kOffBar + 64 + 16 * kGroupTiles + 128;  // barriers, tile records, alignment slack
+};
+
+struct TileRec {          // where a tile's outputs go; rows = 0 for a tile past the end
+  long long ybase;        // element offset of pixel (0, 0), filter 0 of the tile
+  int rows, cols;
+};
+
+template <int OFF>
+__device__ __forceinline__ uint2 lds_v2(uint32_t saddr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(saddr), "n"(OFF));
+  return v;
+}
+// D[0..7][0..7] = A[0..7][0..7] * B[0..7][0..7] (halves, float sums) on the warp's tensor-core
+// path; rows 8..15 of A are zero and their results are dropped.  A thread (g = lane / 4, t = lane
+// % 4) passes A[g][2t, 2t+1] and B[2t, 2t+1][g] and receives D[g][2t, 2t+1].
+__device__ __forceinline__ float2 mma_8x8x8(uint32_t a, uint32_t b) {
+  float d0, d1, d2, d3;
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%7, %7, %7, %7};"
+               : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+               : "r"(a), "r"(0u), "r"(b), "f"(0.f));
+  (void)d2;
+  (void)d3;
+  return make_float2(d0, d1);
+}
+
+// z_xi[j] = sum_nu A^T[j][nu] * M[xi][nu] with M[xi][nu] made on the spot from the thread's
+// operands of V and U in shared memory.
+template <int M, bool SYM>
+struct ProductRows {
+  static constexpr int N = M + 2;
+  using L = SmallCLayout<M>;
+  const Coefs& cf;
+  uint32_t va, ub;          // shared addresses of this thread's words of V and U at xi = 0, nu = 0
+  template <int XI>
+  __device__ __forceinline__ void row(float2 (&z)[M]) const {
+    float2 in[N];
+#pragma unroll
+    for (int h = 0; h < N / 2; ++h) {
+      const uint2 a = lds_v2<XI * (L::kVBytes / N) + 0>(va + h * 8);
+      const uint2 b = lds_v2<XI * (L::kUBytes / N) + 0>(ub + h * 8);
+      in[2 * h] = mma_8x8x8(a.x, b.x);
+      in[2 * h + 1] = mma_8x8x8(a.y, b.y);
+    }
+    at_apply<M, SYM, float2, N>(cf, in, z);
+  }
+};
+
+template <int M, bool SYM>
+__global__ void __launch_bounds__(kThreads, 1)
+fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ CUtensorMap tmX,
+                     const uint32_t* __restrict__ U, __half* __restrict__ y, int H, int W, int K, int Th, int Tw,
+                     long long P, int num_kb, int relu, int* __restrict__ status) {
+  using L = SmallCLayout<M>;
+  constexpr int N = L::N;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+  uint32_t* Us = reinterpret_cast<uint32_t*>(smem + L::kOffU);
+  uint8_t* patch = smem + L::kOffPatch;
+  uint8_t* Vs = smem + L::kOffV;
+  uint8_t* scratch = smem + L::kOffScratch;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBar);          // [2]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(full + 2);
+  TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [8]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kb = blockIdx.x % num_kb;                       // this CTA's block of 64 filters
+  const int cta = blockIdx.x / num_kb, ctas = gridDim.x / num_kb;
+  const long long groups = (P + kGroupTiles - 1) / kGroupTiles;
+
+  if (tid == 0) {
+    mbar_init(&full[0], 1);
+    mbar_init(&full[1], 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                               // x and U may come from the preceding kernels
+
+  // the boxes of group `grp` into patch buffer `buf`; tiles past the end are not fetched
+  auto fetch = [&](long long grp, int buf) {
+    const long long p0 = grp * kGroupTiles;
+    const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
+    mbar_expect_tx(&full[buf], (uint32_t)live * L::kPatchBytes);
+    for (int tl = 0; tl < live; ++tl) {
+      const long long p = p0 + tl;
+      const int tw = (int)(p % Tw), th = (int)((p / Tw) % Th), img = (int)(p / ((long long)Tw * Th));
+      tma_load_4d(patch + (buf * kGroupTiles + tl) * L::kPatchStride, &tmX, &full[buf], 0, M * tw - 1, M * th - 1, img);
+    }
+  };
+  if (tid == 0 && cta < groups) fetch(cta, 0);
+
+  // U[f][K][8] (internal frequency order) -> Us[xi][filter][channel pair][nu]; filters >= K read as 0
+  for (int i = tid; i < N * N * kFilterBlock * 4; i += kThreads) {
+    const int t = i & 3, kl = (i >> 2) & (kFilterBlock - 1), f = i >> 8;
+    const int k = kb * kFilterBlock + kl;
+    const uint32_t v = k < K ? U[((size_t)f * K + k) * 4 + t] : 0u;
+    Us[(((f / N) * kFilterBlock + kl) * 4 + t) * N + (f % N)] = v;
+  }
+
+  const int g = lane >> 2, t = lane & 3;
+  const uint32_t va0 = smem_u32(Vs) + (uint32_t)((g * 4 + t) * N * 4);
+  const uint32_t ub0 = smem_u32(Us) + (uint32_t)((((warp * 8 + g) * 4) + t) * N * 4);
+  const float lo = relu ? 0.f : -__int_as_float(0x7f800000);
+  bool timed_out = false;
+
+  uint32_t it = 0;
+  for (long long grp = cta; grp < groups; grp += ctas, ++it) {
+    const int buf = it & 1;
+    // ---- patches of this group; output records; the next group's fetch
+    if (!mbar_wait(&full[buf], (it >> 1) & 1, abort_flag)) *abort_flag = 1;
+    if (tid < kGroupTiles) {
+      const long long p = grp * kGroupTiles + tid;
+      TileRec r = {0, 0, 0};
+      if (p < P) {
+        const int tw = (int)(p % Tw), th = (int)((p / Tw) % Th);
+        const long long img = p / ((long long)Tw * Th);
+        r.ybase = ((img * H + (long long)M * th) * W + (long long)M * tw) * K + (long long)kb * kFilterBlock;
+        r.rows = min(M, H - M * th);
+        r.cols = min(M, W - M * tw);
+      }
+      rec[tid] = r;
+    }
+    __syncthreads();               // also: every thread is done with the previous group's scratch and V
+    if (*abort_flag) { timed_out = true; break; }
+    if (tid == 0 && grp + ctas < groups) fetch(grp + ctas, buf ^ 1);   // that buffer was last read two syncs ago
+
+    // ---- pass 1: T[tile][xi][b][cp] = sum_a B^T[xi][a] d[a][b]
+    for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
+      const int cp = item & 3, b = (item >> 2) % N, tl = item / (4 * N);
+      const uint8_t* src = patch + (buf * kGroupTiles + tl) * L::kPatchStride + b * 16 + cp * 4;
+      float2 d[N], o[N];
+#pragma unroll
+      for (int a = 0; a < N; ++a) d[a] = __half22float2(*reinterpret_cast<const __half2*>(src + a * N * 16));
+      bt_all_rows<N, SYM>(cf, d, o);
+      float2* dst = reinterpret_cast<float2*>(scratch + tl * L::kTTile) + b * 4 + cp;
+#pragma unroll
+      for (int xi = 0; xi < N; ++xi) dst[xi * N * 4] = o[xi];
+    }
+    __syncthreads();
+    // ---- pass 2: V[xi][nu] = sum_b T[xi][b] B^T[nu][b], rounded to half
+    for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
+      const int cp = item & 3, tl = (item >> 2) & (kGroupTiles - 1), xi = item >> 5;
+      const float2* src = reinterpret_cast<const float2*>(scratch + tl * L::kTTile) + xi * N * 4 + cp;
+      float2 d[N], o[N];
+#pragma unroll
+      for (int b = 0; b < N; ++b) d[b] = src[b * 4];
+      bt_all_rows<N, SYM>(cf, d, o);
+      uint32_t* dst = reinterpret_cast<uint32_t*>(Vs) + ((xi * kGroupTiles + tl) * 4 + cp) * N;
+#pragma unroll
+      for (int nu = 0; nu < N; nu += 2) {
+        const __half2 h0 = __floats2half2_rn(o[nu].x, o[nu].y), h1 = __floats2half2_rn(o[nu + 1].x, o[nu + 1].y);
+        *reinterpret_cast<uint2*>(dst + nu) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      }
+    }
+    __syncthreads();
+    // ---- product and output transform of (tile g, filters 8 warp + 2t, +1)
+    float2 Y[M][M];
+    const ProductRows<M, SYM> rows{cf, va0, ub0};
+    accumulate_rows<M, SYM, float2, N>(cf, rows, Y);
+    // ---- image of y in shared memory (pass 2's readers of the scratch are past the last sync)
+    {
+      uint8_t* dst = scratch + g * L::kYTile + warp * 16 + t * 4;
+#pragma unroll
+      for (int i = 0; i < M; ++i)
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+          const float2 v = vmax_lo(Y[i][j], lo);
+          *reinterpret_cast<__half2*>(dst + (i * M + j) * 128) = __floats2half2_rn(v.x, v.y);
+        }
+    }
+    __syncthreads();
+    // ---- 16-byte pieces: 8 per pixel
+#pragma unroll 4
+    for (int c = tid; c < kGroupTiles * M * M * 8; c += kThreads) {
+      const int q = c & 7, pix = (c >> 3) % (M * M), tl = c / (8 * M * M);
+      const int i = pix / M, j = pix % M;
+      const TileRec r = rec[tl];
+      if (i < r.rows && j < r.cols && kb * kFilterBlock + q * 8 < K) {
+        const uint4 v = *reinterpret_cast<const uint4*>(scratch + tl * L::kYTile + pix * 128 + q * 16);
+        __stcs(reinterpret_cast<uint4*>(y + r.ybase + ((long long)i * W + j) * K + q * 8), v);
+      }
+    }
+  }
+  if (timed_out && tid == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+}
+
+template <int M, bool SYM>
+int go(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, int relu, cudaStream_t stream) {
+  using L = SmallCLayout<M>;
+  EncodeTiledFn enc = tensor_map_encoder();
+  if (!enc) return (int)cudaErrorUnknown;
+  CUtensorMap tmX;
+  cuuint64_t dims[4] = {8, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+  cuuint64_t strides[3] = {16, (cuuint64_t)g.W * 16, (cuuint64_t)g.H * g.W * 16};
+  cuuint32_t box[4] = {8, (cuuint32_t)L::N, (cuuint32_t)L::N, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  if (enc(&tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return (int)cudaErrorUnknown;
+  if (cudaError_t e = allow_dynamic_smem(fused_small_c_kernel<M, SYM>, L::kTotal); e != cudaSuccess) return (int)e;
+  const int num_kb = (g.K + kFilterBlock - 1) / kFilterBlock;
+  const long long groups = (g.P + kGroupTiles - 1) / kGroupTiles;
+  long long per_kb = plan->sm_count / num_kb;
+  if (per_kb < 1) per_kb = 1;
+  if (per_kb > groups) per_kb = groups;
+  return (int)launch_overlapped(fused_small_c_kernel<M, SYM>, (int)(per_kb * num_kb), kThreads, L::kTotal, stream,
+                                plan->kcoefs, tmX, (const uint32_t*)U, (__half*)y, g.H, g.W, g.K, g.Th, g.Tw, g.P, num_kb,
+                                relu, plan->status_dev);
+}
+
+}  // namespace
+
+// x, U and y are 16-byte aligned and K is a multiple of 8 on every path that reaches the launcher.
+bool fused_small_c_applies(const nova_plan* plan, const Geom& g) {
+  return plan->mode == NOVA_FP16_F32ACC && plan->r == 3 && g.C == 8 && plan->status_dev != nullptr;
+}
+
+int launch_fused_small_c(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, int relu,
+                         void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+#define NOVA_SMALLC(MV)                                                       \
+  return plan->symmetric ? go<MV, true>(plan, g, x, U, y, relu, s) : go<MV, false>(plan, g, x, U, y, relu, s)
+  switch (plan->m) {
+    case 2: NOVA_SMALLC(2);
+    case 4: NOVA_SMALLC(4);
+    case 6: NOVA_SMALLC(6);
+    case 8: NOVA_SMALLC(8);
+  }
+#undef NOVA_SMALLC
+  return (int)cudaErrorInvalidValue;
+}
+
+}  // namespace nova

@@ -106,6 +106,10 @@ int launch_gemm_simt(const nova_plan* plan, const void* V, const void* U, float*
 int launch_gemm_tcgen05(const nova_plan* plan, const void* V, const void* U, float* M,
                         int nfreq, int pc, int pc_pad, int C, int K, int* status_dev, void* stream,
                         unsigned long long* prof = nullptr);
+// Input transform, product and output transform in one kernel for C = 8 (half mode, 3-tap filters)
+bool fused_small_c_applies(const nova_plan* plan, const Geom& g);
+int launch_fused_small_c(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, int relu,
+                         void* stream);
 int launch_maxpool2x2(const void* x, void* y, int N, int H, int W, int C, int mode, void* stream);
 
 }  // namespace nova

@@ -25,6 +25,66 @@ __device__ __forceinline__ float2 dequant(float2 bits, float2 s) {
   return make_float2(__fmul_rn(__int2float_rn(__float_as_int(bits.x)), s.x), __fmul_rn(__int2float_rn(__float_as_int(bits.y)), s.y));
 }
 
+// Y[i][j] = sum_xi A^T[i][xi] * z_xi[j], where `rows.template row<XI>(z)` delivers z_xi[j] =
+// sum_nu A^T[j][nu] * M[xi][nu] for its (tile, filters).  The row index is a template parameter so
+// that whatever the provider loads is addressed by immediates.
+template <int M, bool SYM, typename V, int N, typename Rows>
+struct RowAccumulator {
+  const Coefs& cf;
+  const Rows& rows;
+  // dense: Y[i][j] += A^T[i][xi] * z_xi[j] for every xi
+  template <int XI>
+  __device__ __forceinline__ void dense_from(V (&Y)[M][M]) const {
+    if constexpr (XI < N) {
+      V z[M];
+      rows.template row<XI>(z);
+#pragma unroll
+      for (int i = 0; i < M; ++i)
+#pragma unroll
+        for (int j = 0; j < M; ++j) Y[i][j] = (XI == 0) ? vmul(cf.AT[i][0], z[j]) : vfma(cf.AT[i][XI], z[j], Y[i][j]);
+      dense_from<XI + 1>(Y);
+    }
+  }
+  // symmetric: rows +a / -a (Q, Q+1) share |coefficients|: even output rows take the sum of
+  // the two row results, odd output rows the difference
+  template <int Q>
+  __device__ __forceinline__ void pairs_from(V (&Y)[M][M]) const {
+    if constexpr (Q < N - 1) {
+      V zp[M], zm[M];
+      rows.template row<Q>(zp);
+      rows.template row<Q + 1>(zm);
+#pragma unroll
+      for (int j = 0; j < M; ++j) {
+        const V s = vadd(zp[j], zm[j]), d = vsub(zp[j], zm[j]);
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+          Y[i][j] = (Q == 1) ? vmul(cf.AT[i][1], (i & 1) ? d : s) : vfma(cf.AT[i][Q], (i & 1) ? d : s, Y[i][j]);
+      }
+      pairs_from<Q + 2>(Y);
+    }
+  }
+  __device__ __forceinline__ void run(V (&Y)[M][M]) const {
+    if constexpr (!SYM) {
+      dense_from<0>(Y);
+    } else {
+      pairs_from<1>(Y);
+      // A^T column 0 is e_0 and column n-1 is e_{m-1}
+      V z0[M], zi[M];
+      rows.template row<0>(z0);
+      rows.template row<N - 1>(zi);
+#pragma unroll
+      for (int j = 0; j < M; ++j) {
+        Y[0][j] = vadd(Y[0][j], z0[j]);
+        Y[M - 1][j] = vadd(Y[M - 1][j], zi[j]);
+      }
+    }
+  }
+};
+template <int M, bool SYM, typename V, int N, typename Rows>
+__device__ __forceinline__ void accumulate_rows(const Coefs& cf, const Rows& rows, V (&Y)[M][M]) {
+  RowAccumulator<M, SYM, V, N, Rows>{cf, rows}.run(Y);
+}
+
 // QUANT: the stage holds the int32 sums of the int8 pipeline; every value is converted to float
 // and multiplied by qscale (this thread's filters' s_U[k] * s_V) as it is loaded.
 template <int M, bool SYM, int VEC = 1, bool QUANT = false, int R = 3>
@@ -54,53 +114,7 @@ struct OutputTile {
     fill<XI, 0>(in);
     at_apply<M, SYM, V, N>(cf, in, z);
   }
-  // dense: Y[i][j] += A^T[i][xi] * z_xi[j] for every xi
-  template <int XI>
-  __device__ __forceinline__ void dense_from(V (&Y)[M][M]) const {
-    if constexpr (XI < N) {
-      V z[M];
-      row<XI>(z);
-#pragma unroll
-      for (int i = 0; i < M; ++i)
-#pragma unroll
-        for (int j = 0; j < M; ++j) Y[i][j] = (XI == 0) ? vmul(cf.AT[i][0], z[j]) : vfma(cf.AT[i][XI], z[j], Y[i][j]);
-      dense_from<XI + 1>(Y);
-    }
-  }
-  // symmetric: rows +a / -a (Q, Q+1) share |coefficients|: even output rows take the sum of
-  // the two row results, odd output rows the difference
-  template <int Q>
-  __device__ __forceinline__ void pairs_from(V (&Y)[M][M]) const {
-    if constexpr (Q < N - 1) {
-      V zp[M], zm[M];
-      row<Q>(zp);
-      row<Q + 1>(zm);
-#pragma unroll
-      for (int j = 0; j < M; ++j) {
-        const V s = vadd(zp[j], zm[j]), d = vsub(zp[j], zm[j]);
-#pragma unroll
-        for (int i = 0; i < M; ++i)
-          Y[i][j] = (Q == 1) ? vmul(cf.AT[i][1], (i & 1) ? d : s) : vfma(cf.AT[i][Q], (i & 1) ? d : s, Y[i][j]);
-      }
-      pairs_from<Q + 2>(Y);
-    }
-  }
-  __device__ __forceinline__ void run(V (&Y)[M][M]) const {
-    if constexpr (!SYM) {
-      dense_from<0>(Y);
-    } else {
-      pairs_from<1>(Y);
-      // A^T column 0 is e_0 and column n-1 is e_{m-1}
-      V z0[M], zi[M];
-      row<0>(z0);
-      row<N - 1>(zi);
-#pragma unroll
-      for (int j = 0; j < M; ++j) {
-        Y[0][j] = vadd(Y[0][j], z0[j]);
-        Y[M - 1][j] = vadd(Y[M - 1][j], zi[j]);
-      }
-    }
-  }
+  __device__ __forceinline__ void run(V (&Y)[M][M]) const { accumulate_rows<M, SYM, V, N>(cf, *this, Y); }
 };
 
 // Streaming stores of y (written once, not read again by this library): evict-first in the caches,

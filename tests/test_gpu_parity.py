@@ -938,3 +938,46 @@ def test_wait_profiling_variant_gives_the_same_bits_and_consistent_counters():
     pairs = (m + 2) ** 2 * ((tiles + 127) // 128)
     assert w["ctas"] == min(pairs, torch.cuda.get_device_properties(0).multi_processor_count)
     assert abs(w["items_per_cta"] * w["ctas"] - pairs * ((K + 255) // 256)) < 0.5
+
+
+# ---------------------------------------------------------------- 8 input channels: steps 2-4 in one kernel
+@pytest.mark.parametrize("kind,m", [("std", 2), ("std", 4), ("nova", 4), ("nova", 6), ("asym", 6), ("nova", 8),
+                                    ("asym", 8), ("shuf", 8)])
+@pytest.mark.parametrize("shape,relu", [((2, 20, 19, 8, 64), False), ((1, 37, 29, 8, 72), True),
+                                        ((3, 9, 50, 8, 136), False), ((1, 3, 5, 8, 8), True)])
+def test_eight_channel_layers_run_in_one_kernel_and_match_the_emulation(kind, m, shape, relu):
+    # C = 8 in half mode takes the one-kernel path (V and M stay on the SM); a flag that names a kernel of the
+    # three-kernel path switches it off.  Both are judged against the emulation, whole and tile by tile, and
+    # against each other; the cases cover filter blocks with a ragged tail (K = 72, 136), tile groups with a
+    # ragged tail (tiles not a multiple of 8), ragged tiles and images smaller than a tile.
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", relu, True, seed=300 + m)
+    pts = point_set(kind, m)
+    flags = nv.RELU if relu else 0
+    y, _, plan = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, flags=flags)
+    y3, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, flags=flags | nv.GEMM_TCGEN05)
+    wsb = plan.workspace_bytes(N, H, W, C, K)
+    assert plan.launch_count(N, H, W, C, K, wsb, flags) == 1
+    assert plan.launch_count(N, H, W, C, K, wsb, flags | nv.GEMM_TCGEN05) == 3
+    y1 = conv.direct_conv_fp64(x, g)
+    ye = conv.winograd_conv_emulated(x, g, m, pts, "fp16")
+    if relu:
+        y1, ye = np.maximum(y1, 0.0), np.maximum(ye, 0.0)
+    for out in (y, y3):
+        assert np.isfinite(out.astype(np.float32)).all()
+        whole, tile = closeness(out, ye, y1, m)
+        assert whole <= EMU_CLOSE and tile <= EMU_CLOSE_TILE, (whole, tile)
+    whole, tile = closeness(y, y3, y1, m)
+    assert whole <= EMU_CLOSE and tile <= EMU_CLOSE_TILE, (whole, tile)
+
+
+def test_one_kernel_path_passes_nan_and_inf_through_relu_like_the_three_kernel_path():
+    m, N, H, W, C, K = 4, 1, 12, 12, 8, 64
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", False, True, seed=311)
+    x[0, 5, 5, 2] = np.nan
+    pts = point_set("nova", m)
+    y, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, flags=nv.RELU)
+    y3, _, _ = gpu_conv(x, g, m, pts, nv.FP16_F32ACC, flags=nv.RELU | nv.GEMM_TCGEN05)
+    assert np.array_equal(np.isnan(y), np.isnan(y3))
+    assert np.isnan(y[0, 4:8, 4:8, :]).all()          # the tile that holds the pixel
+    assert (y[~np.isnan(y)] >= 0).all()
