@@ -13,13 +13,14 @@
 // One CTA = 256 threads = 8 warps; the CTA keeps the transformed filters of its 64-filter block in
 // shared memory for its whole life and walks groups of 8 consecutive tiles:
 //   TMA      one n x n x 8-channel box per tile straight from x (out-of-range pixels read as 0:
-//            halo and ragged tiles), double buffered, issued one group ahead
+//            halo and ragged tiles), issued for the next group as soon as pass 1 has read this one's
 //   pass 1   B^T along the patch's rows index a, float, to shared memory       (tile, column, channel pair)
 //   pass 2   B^T along the columns index b, rounded once to half: V            (tile, row, channel pair)
 //   product  warp w: filters 8w..8w+7; per row xi of frequencies n mma.sync, then A^T along nu
 //            and the accumulation of Y = sum_xi A^T[.][xi] z_xi, all in registers (packed fp32)
-//   store    Y rounded to half into a shared-memory image of the 8 tiles x 64 filters, then
-//            16-byte streaming stores, 128 contiguous bytes per pixel
+//   store    Y rounded to half into a shared-memory image of the 8 tiles x 64 filters, then bulk
+//            asynchronous copies to y (a kilobyte per tile row when K = 64), which drain while
+//            the next group is computed
 // Rounding points are those of the three-kernel path: tables as the plan holds them, V evaluated
 // in float and rounded once to half, products of halves summed in float, Y evaluated in float and
 // rounded once to half.
@@ -51,13 +52,14 @@ struct SmallCLayout {
   static constexpr int kTBytes = kGroupTiles * kTTile;
   static constexpr int kYTile = M * M * 128 + 16;                       // [i][j][64 filters] half (+16: banks)
   static constexpr int kYBytes = kGroupTiles * kYTile;
-  static constexpr int kScratch = kTBytes > kYBytes ? kTBytes : kYBytes;   // T and the image of y share
   static constexpr int kOffU = 0;
   static constexpr int kOffPatch = kOffU + kUBytes;
-  static constexpr int kOffV = kOffPatch + 2 * kGroupTiles * kPatchStride;
-  static constexpr int kOffScratch = kOffV + kVBytes;
-  static constexpr int kOffBar = (kOffScratch + kScratch + 15) & ~15;
-  static constexpr int kTotal = kOffBar + 64 + 16 * kGroupTiles + 128;  // barriers, tile records, alignment slack
+  static constexpr int kOffV = kOffPatch + kGroupTiles * kPatchStride;
+  static constexpr int kOffT = kOffV + kVBytes;
+  static constexpr int kOffY = kOffT + kTBytes;
+  static constexpr int kOffBar = (kOffY + kYBytes + 15) & ~15;
+  static constexpr int kTotal = kOffBar + 64 + 2 * 16 * kGroupTiles + 128;  // barrier, two sets of tile records, alignment slack
+  static_assert(kTotal <= 227 * 1024, "shared memory of one CTA");
 };
 
 struct TileRec {          // where a tile's outputs go; rows = 0 for a tile past the end
@@ -65,6 +67,10 @@ struct TileRec {          // where a tile's outputs go; rows = 0 for a tile past
   int rows, cols;
 };
 
+__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes)
+               : "memory");
+}
 template <int OFF>
 __device__ __forceinline__ uint2 lds_v2(uint32_t saddr) {
   uint2 v;
@@ -118,10 +124,11 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   uint32_t* Us = reinterpret_cast<uint32_t*>(smem + L::kOffU);
   uint8_t* patch = smem + L::kOffPatch;
   uint8_t* Vs = smem + L::kOffV;
-  uint8_t* scratch = smem + L::kOffScratch;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBar);          // [2]
+  uint8_t* Ts = smem + L::kOffT;
+  uint8_t* Ys = smem + L::kOffY;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBar);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(full + 2);
-  TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [8]
+  TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [2][8]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kb = blockIdx.x % num_kb;                       // this CTA's block of 64 filters
@@ -129,8 +136,7 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   const long long groups = (P + kGroupTiles - 1) / kGroupTiles;
 
   if (tid == 0) {
-    mbar_init(&full[0], 1);
-    mbar_init(&full[1], 1);
+    mbar_init(full, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -138,71 +144,73 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   pdl_launch_dependents();
   pdl_wait();                                               // x and U may come from the preceding kernels
 
-  // the boxes of group `grp` into patch buffer `buf`; tiles past the end are not fetched
-  auto fetch = [&](long long grp, int buf) {
+  // Lanes 0..7 of warp 0, one tile each: the tile's box into the patch buffer and its output record
+  // into record set `set`.  Tiles past the end are not fetched and get an empty record.
+  auto fetch = [&](long long grp, int set) {
     const long long p0 = grp * kGroupTiles;
-    const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
-    mbar_expect_tx(&full[buf], (uint32_t)live * L::kPatchBytes);
-    for (int tl = 0; tl < live; ++tl) {
-      const long long p = p0 + tl;
-      const int tw = (int)(p % Tw), th = (int)((p / Tw) % Th), img = (int)(p / ((long long)Tw * Th));
-      tma_load_4d(patch + (buf * kGroupTiles + tl) * L::kPatchStride, &tmX, &full[buf], 0, M * tw - 1, M * th - 1, img);
+    if (lane == 0) {
+      const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
+      mbar_expect_tx(full, (uint32_t)live * L::kPatchBytes);
     }
+    TileRec r = {0, 0, 0};
+    if (p0 + lane < P) {
+      const uint32_t p = (uint32_t)(p0 + lane);             // the launcher keeps P below 2^31
+      const uint32_t tw = p % (uint32_t)Tw, q = p / (uint32_t)Tw, th = q % (uint32_t)Th, img = q / (uint32_t)Th;
+      tma_load_4d(patch + lane * L::kPatchStride, &tmX, full, 0, (int)(M * tw) - 1, (int)(M * th) - 1, (int)img);
+      r.ybase = (((long long)img * H + M * th) * W + M * tw) * K + (long long)kb * kFilterBlock;
+      r.rows = min(M, H - (int)(M * th));
+      r.cols = min(M, W - (int)(M * tw));
+    }
+    rec[set * kGroupTiles + lane] = r;
   };
-  if (tid == 0 && cta < groups) fetch(cta, 0);
+  if (warp == 0 && lane < kGroupTiles && cta < groups) fetch(cta, 0);
 
-  // U[f][K][8] (internal frequency order) -> Us[xi][filter][channel pair][nu]; filters >= K read as 0
-  for (int i = tid; i < N * N * kFilterBlock * 4; i += kThreads) {
-    const int t = i & 3, kl = (i >> 2) & (kFilterBlock - 1), f = i >> 8;
-    const int k = kb * kFilterBlock + kl;
-    const uint32_t v = k < K ? U[((size_t)f * K + k) * 4 + t] : 0u;
-    Us[(((f / N) * kFilterBlock + kl) * 4 + t) * N + (f % N)] = v;
+  // U[f][K][8] (internal frequency order) -> Us[xi][filter][channel pair][nu]; filters >= K read as 0.
+  // A thread owns one (filter, channel pair): n loads in flight, then n contiguous words stored.
+  {
+    const int t = tid & 3, kl = tid >> 2, k = kb * kFilterBlock + kl;
+    const uint32_t* src = U + ((size_t)(k < K ? k : 0) * 4 + t);
+    uint32_t* dst = Us + (kl * 4 + t) * N;
+#pragma unroll 2
+    for (int xi = 0; xi < N; ++xi) {
+      uint32_t v[N];
+#pragma unroll
+      for (int nu = 0; nu < N; ++nu) v[nu] = k < K ? __ldg(src + (size_t)(xi * N + nu) * K * 4) : 0u;
+#pragma unroll
+      for (int nu = 0; nu < N; nu += 2) *reinterpret_cast<uint2*>(dst + xi * kFilterBlock * 4 * N + nu) = make_uint2(v[nu], v[nu + 1]);
+    }
   }
 
   const int g = lane >> 2, t = lane & 3;
   const uint32_t va0 = smem_u32(Vs) + (uint32_t)((g * 4 + t) * N * 4);
   const uint32_t ub0 = smem_u32(Us) + (uint32_t)((((warp * 8 + g) * 4) + t) * N * 4);
-  const float lo = relu ? 0.f : -__int_as_float(0x7f800000);
+  const __half2 lo2 = relu ? __half2half2(__ushort_as_half(0)) : __half2half2(__ushort_as_half(0xfc00));   // 0 or -inf
+  const int k_here = min(kFilterBlock, K - kb * kFilterBlock);      // filters of this block that exist
   bool timed_out = false;
 
   uint32_t it = 0;
   for (long long grp = cta; grp < groups; grp += ctas, ++it) {
-    const int buf = it & 1;
-    // ---- patches of this group; output records; the next group's fetch
-    if (!mbar_wait(&full[buf], (it >> 1) & 1, abort_flag)) *abort_flag = 1;
-    if (tid < kGroupTiles) {
-      const long long p = grp * kGroupTiles + tid;
-      TileRec r = {0, 0, 0};
-      if (p < P) {
-        const int tw = (int)(p % Tw), th = (int)((p / Tw) % Th);
-        const long long img = p / ((long long)Tw * Th);
-        r.ybase = ((img * H + (long long)M * th) * W + (long long)M * tw) * K + (long long)kb * kFilterBlock;
-        r.rows = min(M, H - M * th);
-        r.cols = min(M, W - M * tw);
-      }
-      rec[tid] = r;
-    }
-    __syncthreads();               // also: every thread is done with the previous group's scratch and V
-    if (*abort_flag) { timed_out = true; break; }
-    if (tid == 0 && grp + ctas < groups) fetch(grp + ctas, buf ^ 1);   // that buffer was last read two syncs ago
-
+    if (!mbar_wait(full, it & 1, abort_flag)) *abort_flag = 1;
     // ---- pass 1: T[tile][xi][b][cp] = sum_a B^T[xi][a] d[a][b]
     for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
       const int cp = item & 3, b = (item >> 2) % N, tl = item / (4 * N);
-      const uint8_t* src = patch + (buf * kGroupTiles + tl) * L::kPatchStride + b * 16 + cp * 4;
+      const uint8_t* src = patch + tl * L::kPatchStride + b * 16 + cp * 4;
       float2 d[N], o[N];
 #pragma unroll
       for (int a = 0; a < N; ++a) d[a] = __half22float2(*reinterpret_cast<const __half2*>(src + a * N * 16));
       bt_all_rows<N, SYM>(cf, d, o);
-      float2* dst = reinterpret_cast<float2*>(scratch + tl * L::kTTile) + b * 4 + cp;
+      float2* dst = reinterpret_cast<float2*>(Ts + tl * L::kTTile) + b * 4 + cp;
 #pragma unroll
       for (int xi = 0; xi < N; ++xi) dst[xi * N * 4] = o[xi];
     }
-    __syncthreads();
+    bulk_wait_read<0>();           // this thread's stores of the previous group have left the image of y
+    __syncthreads();               // the patch buffer is free; the previous group's V and image of y are too
+    if (*abort_flag) { timed_out = true; break; }
+    if (warp == 0 && lane < kGroupTiles && grp + ctas < groups) fetch(grp + ctas, (it + 1) & 1);
     // ---- pass 2: V[xi][nu] = sum_b T[xi][b] B^T[nu][b], rounded to half
     for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
       const int cp = item & 3, tl = (item >> 2) & (kGroupTiles - 1), xi = item >> 5;
-      const float2* src = reinterpret_cast<const float2*>(scratch + tl * L::kTTile) + xi * N * 4 + cp;
+      const float2* src = reinterpret_cast<const float2*>(Ts + tl * L::kTTile) + xi * N * 4 + cp;
       float2 d[N], o[N];
 #pragma unroll
       for (int b = 0; b < N; ++b) d[b] = src[b * 4];
@@ -220,30 +228,35 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
     float2 Y[M][M];
     const ProductRows<M, SYM> rows{cf, va0, ub0};
     accumulate_rows<M, SYM, float2, N>(cf, rows, Y);
-    // ---- image of y in shared memory (pass 2's readers of the scratch are past the last sync)
+    // ---- image of y in shared memory: rounded to half, then the ReLU (NaN and +inf pass)
     {
-      uint8_t* dst = scratch + g * L::kYTile + warp * 16 + t * 4;
+      uint8_t* dst = Ys + g * L::kYTile + warp * 16 + t * 4;
 #pragma unroll
       for (int i = 0; i < M; ++i)
 #pragma unroll
-        for (int j = 0; j < M; ++j) {
-          const float2 v = vmax_lo(Y[i][j], lo);
-          *reinterpret_cast<__half2*>(dst + (i * M + j) * 128) = __floats2half2_rn(v.x, v.y);
-        }
+        for (int j = 0; j < M; ++j)
+          *reinterpret_cast<__half2*>(dst + (i * M + j) * 128) = __hmax2_nan(__floats2half2_rn(Y[i][j].x, Y[i][j].y), lo2);
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk copies below read these writes
     __syncthreads();
-    // ---- 16-byte pieces: 8 per pixel
-#pragma unroll 4
-    for (int c = tid; c < kGroupTiles * M * M * 8; c += kThreads) {
-      const int q = c & 7, pix = (c >> 3) % (M * M), tl = c / (8 * M * M);
-      const int i = pix / M, j = pix % M;
-      const TileRec r = rec[tl];
-      if (i < r.rows && j < r.cols && kb * kFilterBlock + q * 8 < K) {
-        const uint4 v = *reinterpret_cast<const uint4*>(scratch + tl * L::kYTile + pix * 128 + q * 16);
-        __stcs(reinterpret_cast<uint4*>(y + r.ybase + ((long long)i * W + j) * K + q * 8), v);
+    // ---- one thread per (tile, output row): bulk copies shared -> global, asynchronous.  A full-width
+    // row of a 64-filter layer is one contiguous kilobyte; otherwise one copy per pixel.
+    if (tid < kGroupTiles * M) {
+      const int tl = tid / M, i = tid % M;
+      const TileRec r = rec[(it & 1) * kGroupTiles + tl];
+      if (i < r.rows) {
+        __half* dst = y + r.ybase + (long long)i * W * K;
+        const uint8_t* src = Ys + tl * L::kYTile + i * M * 128;
+        if (K == kFilterBlock && r.cols == M) {
+          bulk_s2g(dst, src, M * 128);
+        } else {
+          for (int j = 0; j < r.cols; ++j) bulk_s2g(dst + (long long)j * K, src + j * 128, (uint32_t)k_here * 2);
+        }
+        bulk_commit();
       }
     }
   }
+  bulk_wait_read<0>();             // shared memory stays valid until the last copies have read it
   if (timed_out && tid == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
 }
 
@@ -267,6 +280,7 @@ int go(const nova_plan* plan, const Geom& g, const void* x, const void* U, void*
   long long per_kb = plan->sm_count / num_kb;
   if (per_kb < 1) per_kb = 1;
   if (per_kb > groups) per_kb = groups;
+  if (g.P >= ((long long)1 << 31) - kGroupTiles) return (int)cudaErrorInvalidValue;   // tile indices are 32-bit in the kernel
   return (int)launch_overlapped(fused_small_c_kernel<M, SYM>, (int)(per_kb * num_kb), kThreads, L::kTotal, stream,
                                 plan->kcoefs, tmX, (const uint32_t*)U, (__half*)y, g.H, g.W, g.K, g.Th, g.Tw, g.P, num_kb,
                                 relu, plan->status_dev);
