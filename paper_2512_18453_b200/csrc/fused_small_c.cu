@@ -37,9 +37,19 @@ namespace {
 using namespace sm100;
 using namespace xf;
 
-constexpr int kThreads = 256;
+constexpr int kProductWarps = 8;   // two warpgroups
+constexpr int kHelperWarps = 4;    // one warpgroup
+constexpr int kStoreWarps = 2;     // helper warps that issue the copies of y: 64 threads, one per (tile, output row)
+constexpr int kThreads = (kProductWarps + kHelperWarps) * 32;
 constexpr int kGroupTiles = 8;     // rows 0..7 of the m16n8k8 product (rows 8..15 are fed zeros)
-constexpr int kFilterBlock = 64;   // 8 warps x 8 filters
+constexpr int kFilterBlock = 64;   // 8 product warps x 8 filters
+// Registers per thread after the role split.  The CTA is alone on its SM (shared memory), so the
+// register file holds 256 x 216 + 128 x 72 = 64 512 <= 65 536 whatever the kernel was launched with.
+constexpr int kProductRegs = 216;
+constexpr int kHelperRegs = 72;
+
+// barrier of the helper warps only
+__device__ __forceinline__ void helper_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kHelperWarps * 32) : "memory"); }
 
 template <int M>
 struct SmallCLayout {
@@ -58,7 +68,7 @@ struct SmallCLayout {
   static constexpr int kOffT = kOffV + kVBytes;
   static constexpr int kOffY = kOffT + kTBytes;
   static constexpr int kOffBar = (kOffY + kYBytes + 15) & ~15;
-  static constexpr int kTotal = kOffBar + 64 + 2 * 16 * kGroupTiles + 128;  // barrier, two sets of tile records, alignment slack
+  static constexpr int kTotal = kOffBar + 64 + 4 * 16 * kGroupTiles + 128;  // barriers, four sets of tile records, alignment slack
   static_assert(kTotal <= 227 * 1024, "shared memory of one CTA");
 };
 
@@ -126,9 +136,14 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   uint8_t* Vs = smem + L::kOffV;
   uint8_t* Ts = smem + L::kOffT;
   uint8_t* Ys = smem + L::kOffY;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBar);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(full + 2);
-  TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [2][8]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kOffBar);
+  uint64_t* patch_full = bars;       // the group's boxes have landed                     (TMA)
+  uint64_t* v_full = bars + 1;       // V of the group is in shared memory                (helper warps)
+  uint64_t* v_free = bars + 2;       // the product warps have read V for the last time   (product warps)
+  uint64_t* y_full = bars + 3;       // the image of y is complete                        (product warps)
+  uint64_t* y_free = bars + 4;       // the copies to global memory have read the image   (storing warps)
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 5);
+  TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [4][8]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kb = blockIdx.x % num_kb;                       // this CTA's block of 64 filters
@@ -136,7 +151,11 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   const long long groups = (P + kGroupTiles - 1) / kGroupTiles;
 
   if (tid == 0) {
-    mbar_init(full, 1);
+    mbar_init(patch_full, 1);
+    mbar_init(v_full, kHelperWarps);
+    mbar_init(v_free, kProductWarps);
+    mbar_init(y_full, kProductWarps);
+    mbar_init(y_free, kStoreWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -144,120 +163,155 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   pdl_launch_dependents();
   pdl_wait();                                               // x and U may come from the preceding kernels
 
-  // Lanes 0..7 of warp 0, one tile each: the tile's box into the patch buffer and its output record
-  // into record set `set`.  Tiles past the end are not fetched and get an empty record.
-  auto fetch = [&](long long grp, int set) {
-    const long long p0 = grp * kGroupTiles;
-    if (lane == 0) {
-      const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
-      mbar_expect_tx(full, (uint32_t)live * L::kPatchBytes);
-    }
-    TileRec r = {0, 0, 0};
-    if (p0 + lane < P) {
-      const uint32_t p = (uint32_t)(p0 + lane);             // the launcher keeps P below 2^31
-      const uint32_t tw = p % (uint32_t)Tw, q = p / (uint32_t)Tw, th = q % (uint32_t)Th, img = q / (uint32_t)Th;
-      tma_load_4d(patch + lane * L::kPatchStride, &tmX, full, 0, (int)(M * tw) - 1, (int)(M * th) - 1, (int)img);
-      r.ybase = (((long long)img * H + M * th) * W + M * tw) * K + (long long)kb * kFilterBlock;
-      r.rows = min(M, H - (int)(M * th));
-      r.cols = min(M, W - (int)(M * tw));
-    }
-    rec[set * kGroupTiles + lane] = r;
-  };
-  if (warp == 0 && lane < kGroupTiles && cta < groups) fetch(cta, 0);
-
-  // U[f][K][8] (internal frequency order) -> Us[xi][filter][channel pair][nu]; filters >= K read as 0.
-  // A thread owns one (filter, channel pair): n loads in flight, then n contiguous words stored.
-  {
-    const int t = tid & 3, kl = tid >> 2, k = kb * kFilterBlock + kl;
-    const uint32_t* src = U + ((size_t)(k < K ? k : 0) * 4 + t);
-    uint32_t* dst = Us + (kl * 4 + t) * N;
-#pragma unroll 2
-    for (int xi = 0; xi < N; ++xi) {
-      uint32_t v[N];
-#pragma unroll
-      for (int nu = 0; nu < N; ++nu) v[nu] = k < K ? __ldg(src + (size_t)(xi * N + nu) * K * 4) : 0u;
-#pragma unroll
-      for (int nu = 0; nu < N; nu += 2) *reinterpret_cast<uint2*>(dst + xi * kFilterBlock * 4 * N + nu) = make_uint2(v[nu], v[nu + 1]);
-    }
-  }
-
-  const int g = lane >> 2, t = lane & 3;
-  const uint32_t va0 = smem_u32(Vs) + (uint32_t)((g * 4 + t) * N * 4);
-  const uint32_t ub0 = smem_u32(Us) + (uint32_t)((((warp * 8 + g) * 4) + t) * N * 4);
-  const __half2 lo2 = relu ? __half2half2(__ushort_as_half(0)) : __half2half2(__ushort_as_half(0xfc00));   // 0 or -inf
-  const int k_here = min(kFilterBlock, K - kb * kFilterBlock);      // filters of this block that exist
-  bool timed_out = false;
-
-  uint32_t it = 0;
-  for (long long grp = cta; grp < groups; grp += ctas, ++it) {
-    if (!mbar_wait(full, it & 1, abort_flag)) *abort_flag = 1;
-    // ---- pass 1: T[tile][xi][b][cp] = sum_a B^T[xi][a] d[a][b]
-    for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
-      const int cp = item & 3, b = (item >> 2) % N, tl = item / (4 * N);
-      const uint8_t* src = patch + tl * L::kPatchStride + b * 16 + cp * 4;
-      float2 d[N], o[N];
-#pragma unroll
-      for (int a = 0; a < N; ++a) d[a] = __half22float2(*reinterpret_cast<const __half2*>(src + a * N * 16));
-      bt_all_rows<N, SYM>(cf, d, o);
-      float2* dst = reinterpret_cast<float2*>(Ts + tl * L::kTTile) + b * 4 + cp;
-#pragma unroll
-      for (int xi = 0; xi < N; ++xi) dst[xi * N * 4] = o[xi];
-    }
-    bulk_wait_read<0>();           // this thread's stores of the previous group have left the image of y
-    __syncthreads();               // the patch buffer is free; the previous group's V and image of y are too
-    if (*abort_flag) { timed_out = true; break; }
-    if (warp == 0 && lane < kGroupTiles && grp + ctas < groups) fetch(grp + ctas, (it + 1) & 1);
-    // ---- pass 2: V[xi][nu] = sum_b T[xi][b] B^T[nu][b], rounded to half
-    for (int item = tid; item < kGroupTiles * N * 4; item += kThreads) {
-      const int cp = item & 3, tl = (item >> 2) & (kGroupTiles - 1), xi = item >> 5;
-      const float2* src = reinterpret_cast<const float2*>(Ts + tl * L::kTTile) + xi * N * 4 + cp;
-      float2 d[N], o[N];
-#pragma unroll
-      for (int b = 0; b < N; ++b) d[b] = src[b * 4];
-      bt_all_rows<N, SYM>(cf, d, o);
-      uint32_t* dst = reinterpret_cast<uint32_t*>(Vs) + ((xi * kGroupTiles + tl) * 4 + cp) * N;
-#pragma unroll
-      for (int nu = 0; nu < N; nu += 2) {
-        const __half2 h0 = __floats2half2_rn(o[nu].x, o[nu].y), h1 = __floats2half2_rn(o[nu + 1].x, o[nu + 1].y);
-        *reinterpret_cast<uint2*>(dst + nu) =
-            make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-      }
-    }
-    __syncthreads();
-    // ---- product and output transform of (tile g, filters 8 warp + 2t, +1)
-    float2 Y[M][M];
-    const ProductRows<M, SYM> rows{cf, va0, ub0};
-    accumulate_rows<M, SYM, float2, N>(cf, rows, Y);
-    // ---- image of y in shared memory: rounded to half, then the ReLU (NaN and +inf pass)
+  if (warp < kProductWarps) {
+    // ================= product warps: M[f] = V[f] U[f]^T by mma.sync, Y = A^T M A, image of y
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kProductRegs));
+    // U[f][K][8] (internal frequency order) -> Us[xi][filter][channel pair][nu]; filters >= K read as 0.
+    // A thread owns one (filter, channel pair) - of its own warp's 8 filters: n loads in flight, then
+    // n contiguous words stored, and only the warp itself reads them back.
     {
+      const int t = tid & 3, kl = tid >> 2, k = kb * kFilterBlock + kl;
+      const uint32_t* src = U + ((size_t)(k < K ? k : 0) * 4 + t);
+      uint32_t* dst = Us + (kl * 4 + t) * N;
+#pragma unroll 2
+      for (int xi = 0; xi < N; ++xi) {
+        uint32_t v[N];
+#pragma unroll
+        for (int nu = 0; nu < N; ++nu) v[nu] = k < K ? __ldg(src + (size_t)(xi * N + nu) * K * 4) : 0u;
+#pragma unroll
+        for (int nu = 0; nu < N; nu += 2)
+          *reinterpret_cast<uint2*>(dst + xi * kFilterBlock * 4 * N + nu) = make_uint2(v[nu], v[nu + 1]);
+      }
+      __syncwarp();
+    }
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t va0 = smem_u32(Vs) + (uint32_t)((g * 4 + t) * N * 4);
+    const uint32_t ub0 = smem_u32(Us) + (uint32_t)((((warp * 8 + g) * 4) + t) * N * 4);
+    const __half2 lo2 = relu ? __half2half2(__ushort_as_half(0)) : __half2half2(__ushort_as_half(0xfc00));   // 0 or -inf
+    uint32_t it = 0;
+    for (long long grp = cta; grp < groups; grp += ctas, ++it) {
+      if (!mbar_poll(v_full, it & 1, abort_flag)) { *abort_flag = 1; break; }
+      float2 Y[M][M];
+      const ProductRows<M, SYM> rows{cf, va0, ub0};
+      accumulate_rows<M, SYM, float2, N>(cf, rows, Y);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(v_free);
+      // the copies of the previous group must have read the image before it is overwritten
+      if (!mbar_wait(y_free, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; break; }
+      // rounded to half, then the ReLU (NaN and +inf pass)
       uint8_t* dst = Ys + g * L::kYTile + warp * 16 + t * 4;
 #pragma unroll
       for (int i = 0; i < M; ++i)
 #pragma unroll
         for (int j = 0; j < M; ++j)
           *reinterpret_cast<__half2*>(dst + (i * M + j) * 128) = __hmax2_nan(__floats2half2_rn(Y[i][j].x, Y[i][j].y), lo2);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk copies read these writes
+      __syncwarp();
+      if (lane == 0) mbar_arrive(y_full);
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk copies below read these writes
-    __syncthreads();
-    // ---- one thread per (tile, output row): bulk copies shared -> global, asynchronous.  A full-width
-    // row of a 64-filter layer is one contiguous kilobyte; otherwise one copy per pixel.
-    if (tid < kGroupTiles * M) {
-      const int tl = tid / M, i = tid % M;
-      const TileRec r = rec[(it & 1) * kGroupTiles + tl];
-      if (i < r.rows) {
-        __half* dst = y + r.ybase + (long long)i * W * K;
-        const uint8_t* src = Ys + tl * L::kYTile + i * M * 128;
-        if (K == kFilterBlock && r.cols == M) {
-          bulk_s2g(dst, src, M * 128);
-        } else {
-          for (int j = 0; j < r.cols; ++j) bulk_s2g(dst + (long long)j * K, src + j * 128, (uint32_t)k_here * 2);
-        }
-        bulk_commit();
+  } else {
+    // ================= helper warps: boxes of x by TMA, V = B^T d B, copies of the image of y to global memory
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
+    const int ht = tid - kProductWarps * 32;                 // 0 .. 127
+    const int k_here = min(kFilterBlock, K - kb * kFilterBlock);      // filters of this block that exist
+    // Lanes 0..7 of the first helper warp, one tile each: the tile's box into the patch buffer and its
+    // output record into record set `set`.  Tiles past the end are not fetched and get an empty record.
+    auto fetch = [&](long long grp, int set) {
+      const long long p0 = grp * kGroupTiles;
+      if (lane == 0) {
+        const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
+        mbar_expect_tx(patch_full, (uint32_t)live * L::kPatchBytes);
       }
+      TileRec r = {0, 0, 0};
+      if (p0 + lane < P) {
+        const uint32_t p = (uint32_t)(p0 + lane);             // the launcher keeps P below 2^31
+        const uint32_t tw = p % (uint32_t)Tw, q = p / (uint32_t)Tw, th = q % (uint32_t)Th, img = q / (uint32_t)Th;
+        tma_load_4d(patch + lane * L::kPatchStride, &tmX, patch_full, 0, (int)(M * tw) - 1, (int)(M * th) - 1, (int)img);
+        r.ybase = (((long long)img * H + M * th) * W + M * tw) * K + (long long)kb * kFilterBlock;
+        r.rows = min(M, H - (int)(M * th));
+        r.cols = min(M, W - (int)(M * tw));
+      }
+      rec[set * kGroupTiles + lane] = r;
+    };
+    // The last kStoreWarps helper warps, one thread per (tile, output row) of group number `n` of this
+    // CTA: bulk copies shared -> global.  A full-width row of a 64-filter layer is one contiguous
+    // kilobyte; otherwise one copy per pixel.  store_release, a good thousand cycles later, finds the
+    // copies' reads of the image complete and hands the image back to the product warps.
+    const int st = ht - (kHelperWarps - kStoreWarps) * 32;     // >= 0 in a storing warp
+    auto store_issue = [&](uint32_t n) {
+      if (st < 0) return;
+      const bool ok = mbar_wait(y_full, n & 1, abort_flag);
+      if (!ok) *abort_flag = 1;
+      if (ok && st < kGroupTiles * M) {
+        const int tl = st / M, i = st % M;
+        const TileRec r = rec[(n & 3) * kGroupTiles + tl];
+        if (i < r.rows) {
+          __half* dst = y + r.ybase + (long long)i * W * K;
+          const uint8_t* src = Ys + tl * L::kYTile + i * M * 128;
+          if (K == kFilterBlock && r.cols == M) {
+            bulk_s2g(dst, src, M * 128);
+          } else {
+            for (int j = 0; j < r.cols; ++j) bulk_s2g(dst + (long long)j * K, src + j * 128, (uint32_t)k_here * 2);
+          }
+          bulk_commit();
+        }
+      }
+    };
+    auto store_release = [&]() {
+      if (st < 0) return;
+      bulk_wait_read<0>();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(y_free);
+    };
+    if (warp == kProductWarps && lane < kGroupTiles && cta < groups) fetch(cta, 0);
+    uint32_t it = 0;
+    for (long long grp = cta; grp < groups; grp += ctas, ++it) {
+      if (!mbar_wait(patch_full, it & 1, abort_flag)) *abort_flag = 1;
+      // ---- pass 1: T[tile][xi][b][cp] = sum_a B^T[xi][a] d[a][b]
+      for (int item = ht; item < kGroupTiles * N * 4; item += kHelperWarps * 32) {
+        const int cp = item & 3, b = (item >> 2) % N, tl = item / (4 * N);
+        const uint8_t* src = patch + tl * L::kPatchStride + b * 16 + cp * 4;
+        float2 d[N], o[N];
+#pragma unroll
+        for (int a = 0; a < N; ++a) d[a] = __half22float2(*reinterpret_cast<const __half2*>(src + a * N * 16));
+        bt_all_rows<N, SYM>(cf, d, o);
+        float2* dst = reinterpret_cast<float2*>(Ts + tl * L::kTTile) + b * 4 + cp;
+#pragma unroll
+        for (int xi = 0; xi < N; ++xi) dst[xi * N * 4] = o[xi];
+      }
+      helper_sync();                 // T is complete and the patch buffer is free
+      if (*abort_flag) break;        // uniform: every helper reads the flag after the same barrier
+      if (warp == kProductWarps && lane < kGroupTiles && grp + ctas < groups) fetch(grp + ctas, (it + 1) & 3);
+      if (it > 1) store_release();   // the copies of group it - 2, issued one iteration ago
+      if (!mbar_poll(v_free, (it & 1) ^ 1, abort_flag)) *abort_flag = 1;   // on the critical path
+      // ---- pass 2: V[xi][nu] = sum_b T[xi][b] B^T[nu][b], rounded to half
+      for (int item = ht; item < kGroupTiles * N * 4; item += kHelperWarps * 32) {
+        const int cp = item & 3, tl = (item >> 2) & (kGroupTiles - 1), xi = item >> 5;
+        const float2* src = reinterpret_cast<const float2*>(Ts + tl * L::kTTile) + xi * N * 4 + cp;
+        float2 d[N], o[N];
+#pragma unroll
+        for (int b = 0; b < N; ++b) d[b] = src[b * 4];
+        bt_all_rows<N, SYM>(cf, d, o);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(Vs) + ((xi * kGroupTiles + tl) * 4 + cp) * N;
+#pragma unroll
+        for (int nu = 0; nu < N; nu += 2) {
+          const __half2 h0 = __floats2half2_rn(o[nu].x, o[nu].y), h1 = __floats2half2_rn(o[nu + 1].x, o[nu + 1].y);
+          *reinterpret_cast<uint2*>(dst + nu) =
+              make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(v_full);
+      if (it > 0) store_issue(it - 1);
+      helper_sync();                 // T may be overwritten
     }
+    if (!*abort_flag) {
+      if (it > 1) store_release();
+      if (it > 0) { store_issue(it - 1); store_release(); }
+    }
+    bulk_wait_read<0>();
   }
-  bulk_wait_read<0>();             // shared memory stays valid until the last copies have read it
-  if (timed_out && tid == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
+  if (*abort_flag && lane == 0) atomicExch(status, NOVA_ERR_DEVICE_TIMEOUT);
 }
 
 template <int M, bool SYM>
