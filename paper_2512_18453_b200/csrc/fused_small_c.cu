@@ -39,7 +39,7 @@ using namespace xf;
 
 constexpr int kProductWarps = 8;   // two warpgroups
 constexpr int kHelperWarps = 4;    // one warpgroup
-constexpr int kStoreWarps = 2;     // helper warps that issue the copies of y: 64 threads, one per (tile, output row)
+constexpr int kStoreLanes = 16;    // lanes per helper warp that issue the copies of y: 64 threads, one per (tile, output row)
 constexpr int kThreads = (kProductWarps + kHelperWarps) * 32;
 constexpr int kGroupTiles = 8;     // rows 0..7 of the m16n8k8 product (rows 8..15 are fed zeros)
 constexpr int kFilterBlock = 64;   // 8 product warps x 8 filters
@@ -87,18 +87,18 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t saddr) {
   asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(saddr), "n"(OFF));
   return v;
 }
+#pragma nv_diag_suppress 550
 // D[0..7][0..7] = A[0..7][0..7] * B[0..7][0..7] (halves, float sums) on the warp's tensor-core
 // path; rows 8..15 of A are zero and their results are dropped.  A thread (g = lane / 4, t = lane
 // % 4) passes A[g][2t, 2t+1] and B[2t, 2t+1][g] and receives D[g][2t, 2t+1].
 __device__ __forceinline__ float2 mma_8x8x8(uint32_t a, uint32_t b) {
-  float d0, d1, d2, d3;
+  float d0, d1, d2, d3;                 // d2, d3: rows 8..15, unused
   asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%7, %7, %7, %7};"
                : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
                : "r"(a), "r"(0u), "r"(b), "f"(0.f));
-  (void)d2;
-  (void)d3;
   return make_float2(d0, d1);
 }
+#pragma nv_diag_default 550
 
 // z_xi[j] = sum_nu A^T[j][nu] * M[xi][nu] with M[xi][nu] made on the spot from the thread's
 // operands of V and U in shared memory.
@@ -155,7 +155,7 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
     mbar_init(v_full, kHelperWarps);
     mbar_init(v_free, kProductWarps);
     mbar_init(y_full, kProductWarps);
-    mbar_init(y_free, kStoreWarps);
+    mbar_init(y_free, kHelperWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -214,32 +214,37 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
     const int ht = tid - kProductWarps * 32;                 // 0 .. 127
     const int k_here = min(kFilterBlock, K - kb * kFilterBlock);      // filters of this block that exist
-    // Lanes 0..7 of the first helper warp, one tile each: the tile's box into the patch buffer and its
-    // output record into record set `set`.  Tiles past the end are not fetched and get an empty record.
+    // Lanes 0 and 1 of every helper warp, one tile each (tile 2 hw + lane of the group): the tile's box
+    // into the patch buffer and its output record into record set `set`.  Tiles past the end are not
+    // fetched and get an empty record.  (Eight lanes of one warp took 1 500 cycles over it, on the
+    // critical path of that warp.)
+    const int hw = warp - kProductWarps;
     auto fetch = [&](long long grp, int set) {
+      if (lane >= kGroupTiles / kHelperWarps) return;
+      const int tl = hw * (kGroupTiles / kHelperWarps) + lane;
       const long long p0 = grp * kGroupTiles;
-      if (lane == 0) {
+      if (tl == 0) {
         const int live = (int)((P - p0) < kGroupTiles ? (P - p0) : kGroupTiles);
         mbar_expect_tx(patch_full, (uint32_t)live * L::kPatchBytes);
       }
       TileRec r = {0, 0, 0};
-      if (p0 + lane < P) {
-        const uint32_t p = (uint32_t)(p0 + lane);             // the launcher keeps P below 2^31
+      if (p0 + tl < P) {
+        const uint32_t p = (uint32_t)(p0 + tl);               // the launcher keeps P below 2^31
         const uint32_t tw = p % (uint32_t)Tw, q = p / (uint32_t)Tw, th = q % (uint32_t)Th, img = q / (uint32_t)Th;
-        tma_load_4d(patch + lane * L::kPatchStride, &tmX, patch_full, 0, (int)(M * tw) - 1, (int)(M * th) - 1, (int)img);
+        tma_load_4d(patch + tl * L::kPatchStride, &tmX, patch_full, 0, (int)(M * tw) - 1, (int)(M * th) - 1, (int)img);
         r.ybase = (((long long)img * H + M * th) * W + M * tw) * K + (long long)kb * kFilterBlock;
         r.rows = min(M, H - (int)(M * th));
         r.cols = min(M, W - (int)(M * tw));
       }
-      rec[set * kGroupTiles + lane] = r;
+      rec[set * kGroupTiles + tl] = r;
     };
-    // The last kStoreWarps helper warps, one thread per (tile, output row) of group number `n` of this
-    // CTA: bulk copies shared -> global.  A full-width row of a 64-filter layer is one contiguous
-    // kilobyte; otherwise one copy per pixel.  store_release, a good thousand cycles later, finds the
-    // copies' reads of the image complete and hands the image back to the product warps.
-    const int st = ht - (kHelperWarps - kStoreWarps) * 32;     // >= 0 in a storing warp
+    // The first kStoreLanes lanes of every helper warp, one thread per (tile, output row) of group
+    // number `n` of this CTA: bulk copies shared -> global.  A full-width row of a 64-filter layer is
+    // one contiguous kilobyte; otherwise one copy per pixel.  (A warp issues such copies lane after
+    // lane, some 85 cycles each: hence four warps.)  store_release, a good thousand cycles later, finds
+    // the copies' reads of the image complete and hands the image back to the product warps.
+    const int st = lane < kStoreLanes ? hw * kStoreLanes + lane : kGroupTiles * M;
     auto store_issue = [&](uint32_t n) {
-      if (st < 0) return;
       const bool ok = mbar_wait(y_full, n & 1, abort_flag);
       if (!ok) *abort_flag = 1;
       if (ok && st < kGroupTiles * M) {
@@ -258,12 +263,11 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
       }
     };
     auto store_release = [&]() {
-      if (st < 0) return;
       bulk_wait_read<0>();
       __syncwarp();
       if (lane == 0) mbar_arrive(y_free);
     };
-    if (warp == kProductWarps && lane < kGroupTiles && cta < groups) fetch(cta, 0);
+    if (cta < groups) fetch(cta, 0);
     uint32_t it = 0;
     for (long long grp = cta; grp < groups; grp += ctas, ++it) {
       if (!mbar_wait(patch_full, it & 1, abort_flag)) *abort_flag = 1;
@@ -281,7 +285,7 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
       }
       helper_sync();                 // T is complete and the patch buffer is free
       if (*abort_flag) break;        // uniform: every helper reads the flag after the same barrier
-      if (warp == kProductWarps && lane < kGroupTiles && grp + ctas < groups) fetch(grp + ctas, (it + 1) & 3);
+      if (grp + ctas < groups) fetch(grp + ctas, (it + 1) & 3);
       if (it > 1) store_release();   // the copies of group it - 2, issued one iteration ago
       if (!mbar_poll(v_free, (it & 1) ^ 1, abort_flag)) *abort_flag = 1;   // on the critical path
       // ---- pass 2: V[xi][nu] = sum_b T[xi][b] B^T[nu][b], rounded to half
