@@ -213,6 +213,10 @@ size_t nova_conv2d_min_workspace_bytes(const nova_plan* plan, int N, int H, int 
  * workspace_dev: 256-byte aligned scratch of workspace_bytes; contents are
  * undefined afterwards (the kernels tell the L2 to drop its lines unwritten once
  * they have been read); calls sharing a workspace must be stream-ordered.
+ * With C = 8 (NOVA_FP16_F32ACC, 3-tap filters, none of NOVA_GEMM_SIMT, NOVA_GEMM_TCGEN05,
+ * NOVA_TRANSFORM_SIMT, NOVA_PROFILE_WAITS) the three steps run in ONE kernel that keeps V and M
+ * on the SM: same arithmetic and rounding points, one launch, workspace checked but not touched.
+ * Needs fewer than 2^31 tiles (NOVA_ERR_CUDA otherwise).
  */
 int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
                     int N, int H, int W, int C, int K,
@@ -222,7 +226,8 @@ int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev,
  * Measurement aid: the same work as nova_conv2d_fwd with CUDA events recorded
  * on `stream` around each kernel; synchronises the stream and writes the summed
  * device time in milliseconds of the three kernel classes to kernel_ms_host[0..2]
- * (input transform, transformed-domain product, output transform).
+ * (input transform, transformed-domain product, output transform); the one-kernel
+ * path of C = 8 reports its time as the product's and 0 for the transforms.
  */
 int nova_conv2d_fwd_timed(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
                           int N, int H, int W, int C, int K,
