@@ -215,8 +215,8 @@ size_t nova_conv2d_min_workspace_bytes(const nova_plan* plan, int N, int H, int 
  * they have been read); calls sharing a workspace must be stream-ordered.
  * With C = 8 (NOVA_FP16_F32ACC, 3-tap filters, none of NOVA_GEMM_SIMT, NOVA_GEMM_TCGEN05,
  * NOVA_TRANSFORM_SIMT, NOVA_PROFILE_WAITS) the three steps run in ONE kernel that keeps V and M
- * on the SM: same arithmetic and rounding points, one launch, workspace checked but not touched.
- * Needs fewer than 2^31 tiles (NOVA_ERR_CUDA otherwise).
+ * on the SM: same arithmetic and rounding points, one launch, workspace checked but not touched
+ * (problems of 2^31 tiles or more stay on the three-kernel path).
  */
 int nova_conv2d_fwd(const nova_plan* plan, const void* x_dev, const void* U_dev, void* y_dev,
                     int N, int H, int W, int C, int K,

@@ -338,7 +338,6 @@ int go(const nova_plan* plan, const Geom& g, const void* x, const void* U, void*
   long long per_kb = plan->sm_count / num_kb;
   if (per_kb < 1) per_kb = 1;
   if (per_kb > groups) per_kb = groups;
-  if (g.P >= ((long long)1 << 31) - kGroupTiles) return (int)cudaErrorInvalidValue;   // tile indices are 32-bit in the kernel
   return (int)launch_overlapped(fused_small_c_kernel<M, SYM>, (int)(per_kb * num_kb), kThreads, L::kTotal, stream,
                                 plan->kcoefs, tmX, (const uint32_t*)U, (__half*)y, g.H, g.W, g.K, g.Th, g.Tw, g.P, num_kb,
                                 relu, plan->status_dev);
@@ -347,8 +346,10 @@ int go(const nova_plan* plan, const Geom& g, const void* x, const void* U, void*
 }  // namespace
 
 // x, U and y are 16-byte aligned and K is a multiple of 8 on every path that reaches the launcher.
+// Tile indices are 32-bit in the kernel: larger problems stay on the three-kernel path.
 bool fused_small_c_applies(const nova_plan* plan, const Geom& g) {
-  return plan->mode == NOVA_FP16_F32ACC && plan->r == 3 && g.C == 8 && plan->status_dev != nullptr;
+  return plan->mode == NOVA_FP16_F32ACC && plan->r == 3 && g.C == 8 && plan->status_dev != nullptr &&
+         g.P < ((long long)1 << 31) - kGroupTiles;
 }
 
 int launch_fused_small_c(const nova_plan* plan, const Geom& g, const void* x, const void* U, void* y, int relu,
