@@ -10,17 +10,22 @@
 // (The TMEM-accumulator route of the large-C product kernel cannot do this: n*n frequencies x 8
 // filters already exceed an SM's 512 accumulator columns.)
 //
-// One CTA = 256 threads = 8 warps; the CTA keeps the transformed filters of its 64-filter block in
-// shared memory for its whole life and walks groups of 8 consecutive tiles:
-//   TMA      one n x n x 8-channel box per tile straight from x (out-of-range pixels read as 0:
-//            halo and ragged tiles), issued for the next group as soon as pass 1 has read this one's
-//   pass 1   B^T along the patch's rows index a, float, to shared memory       (tile, column, channel pair)
-//   pass 2   B^T along the columns index b, rounded once to half: V            (tile, row, channel pair)
-//   product  warp w: filters 8w..8w+7; per row xi of frequencies n mma.sync, then A^T along nu
-//            and the accumulation of Y = sum_xi A^T[.][xi] z_xi, all in registers (packed fp32)
-//   store    Y rounded to half into a shared-memory image of the 8 tiles x 64 filters, then bulk
-//            asynchronous copies to y (a kilobyte per tile row when K = 64), which drain while
-//            the next group is computed
+// One CTA per SM, 12 warps in two roles with their own register budgets (setmaxnreg); the CTA
+// keeps the transformed filters of its 64-filter block in shared memory for its whole life and
+// walks groups of 8 consecutive tiles:
+//   helper warps (4)   TMA: one n x n x 8-channel box per tile straight from x (out-of-range pixels
+//                      read as 0: halo and ragged tiles), issued for the next group as soon as
+//                      pass 1 has read this one's;
+//                      pass 1: B^T along the patch's rows index a, float, to shared memory;
+//                      pass 2: B^T along the columns index b, rounded once to half: V (as soon as
+//                      the product warps have released the V buffer);
+//                      bulk asynchronous copies of the finished image of y to global memory (a
+//                      kilobyte per tile row when K = 64), which drain while the next group is computed
+//   product warps (8)  warp w owns filters 8w..8w+7: per row xi of frequencies n mma.sync, then
+//                      A^T along nu and the accumulation of Y = sum_xi A^T[.][xi] z_xi, all in
+//                      registers (packed fp32); Y rounded to half (and ReLU) into a shared-memory
+//                      image of the 8 tiles x 64 filters
+// The roles meet at mbarriers (V full / free, image full / free), every wait bounded.
 // Rounding points are those of the three-kernel path: tables as the plan holds them, V evaluated
 // in float and rounded once to half, products of halves summed in float, Y evaluated in float and
 // rounded once to half.
