@@ -800,20 +800,21 @@ def run_vgg(args):
     ms = e0.elapsed_time(e1) / steps
     clocks = sampler.stop()
     status = plan.device_status()
-    # per-layer durations (events around each convolution, direct launches, one extra pass)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in shapes]
+    # per-layer durations: the layer's call five times back to back between two events (direct launches;
+    # the activations of the last step are still in the buffers, so every layer sees its real input)
+    reps = 5
+    layers_ms = []
     a = x
     for i, (h, ci, co, pool) in enumerate(shapes):
-        evs[i][0].record()
+        e0l, e1l = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         plan.conv2d(a, Us[i], y=ys[i], workspace=ws, flags=flags)
-        evs[i][1].record()
-        a = ys[i]
-        if pool:
-            nv.binding._check(L.nova_maxpool2x2(a.data_ptr(), ps[i].data_ptr(), N, h, h, co, nv.FP16_F32ACC,
-                                                nv.binding._stream()), "nova_maxpool2x2")
-            a = ps[i]
-    torch.cuda.synchronize()
-    layers_ms = ["%dx%d C%d K%d: %.3f" % (h, h, ci, co, e[0].elapsed_time(e[1])) for (h, ci, co, _), e in zip(shapes, evs)]
+        e0l.record()
+        for _ in range(reps):
+            plan.conv2d(a, Us[i], y=ys[i], workspace=ws, flags=flags)
+        e1l.record()
+        torch.cuda.synchronize()
+        layers_ms.append("%dx%d C%d K%d: %.3f" % (h, h, ci, co, e0l.elapsed_time(e1l) / reps))
+        a = ps[i] if pool else ys[i]
     direct = sum(2.0 * N * h * h * co * ci_true * 9 for (h, _, co, _), (ci_true, _, _) in zip(shapes, VGG16_LAYERS))
     launches = sum(plan.launch_count(N, h, h, ci, co, ws_bytes, flags) for (h, ci, co, _) in shapes) + 5
     # accuracy on the first two images (images are independent), untimed
