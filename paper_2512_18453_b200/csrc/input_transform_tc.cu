@@ -10,12 +10,14 @@
 // accumulation of exact products of the rounded coefficients with the inputs, i.e. the
 // same quantity the CUDA-core transform evaluates, in a different summation order.
 //
-// One work unit = (tile p, block of 128 channels):
-// The units of a CTA (a contiguous range) are numbered i = 0, 1, ..; unit i uses ring stage
+// One work unit = two (tile, block of 64 channels) pairs, one per half of the 128 TMEM lanes; the
+// pairs are numbered tile-major, so a unit is a tile's two neighbouring channel blocks when C is a
+// multiple of 128 and two neighbouring tiles when C = 64 (no lane computes on zero fill).
+// The units of a CTA are numbered i = 0, 1, ..; unit i uses ring stage
 // i % kStages and TMEM accumulator i % kNumAcc.  Issuing a TMA box or a small MMA costs the
 // issuing thread a few hundred cycles, so every role is spread over several warps:
 //   warps 0-3   TMA producers, unit i by warp i%4: the n x n x 64-channel patch boxes of the
-//               unit (two boxes, one per 64 channels) straight from x [N,H,W,C]; rows/columns
+//               unit (two boxes, one per pair) straight from x [N,H,W,C]; rows/columns
 //               outside the image and channels >= C are zero-filled by the TMA unit (the pad-1
 //               halo and ragged tiles cost nothing).  A box lands as n*n rows of 128 bytes with
 //               the 128-byte swizzle, which is the MN-major operand layout of tcgen05.mma
@@ -113,11 +115,15 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int CB = (C + 127) / 128;
-  // Unit i of this CTA is unit blockIdx.x + i * gridDim.x of the chunk: the chunk's tiles are
-  // transformed in ascending order chip-wide, so that the rows of V written last - the ones
-  // still in L2 when the product kernel starts - are the highest tiles.
-  const unsigned num_units = (unsigned)pc * (unsigned)CB;
+  // A unit is two (tile, 64-channel block) pairs, one per half of the 128 TMEM lanes; the pairs are
+  // numbered tile-major, so a unit is one tile's two consecutive channel blocks when C is a multiple
+  // of 128 and two consecutive tiles when C = 64.  Unit i of this CTA is unit blockIdx.x + i *
+  // gridDim.x of the chunk: the chunk's tiles are transformed in ascending order chip-wide, so that
+  // the rows of V written last - the ones still in L2 when the product kernel starts - are the
+  // highest tiles.
+  const unsigned CB64 = (unsigned)(C + 63) / 64;
+  const unsigned num_sub = (unsigned)pc * CB64;
+  const unsigned num_units = (num_sub + 1) / 2;
   const uint32_t n_local = num_units > blockIdx.x ? (num_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
 
   if (threadIdx.x == 0) {
@@ -158,17 +164,20 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
     // ---------------- TMA producers
     for (uint32_t local = warp; local < n_local && !timed_out; local += kProdWarps) {
       const unsigned u = blockIdx.x + local * gridDim.x;
-      const int cblk = (int)(u % (unsigned)CB);
-      const unsigned p = (unsigned)p0 + u / (unsigned)CB;
-      const int tw = (int)(p % (unsigned)Tw), th = (int)((p / (unsigned)Tw) % (unsigned)Th);
-      const int img = (int)(p / ((unsigned)Tw * (unsigned)Th));
       const uint32_t stage = local % kStages, phase = (local / kStages) & 1;
       if (!mbar_wait_warp(&empty_bar[stage], phase ^ 1, abort_flag)) { timed_out = true; break; }
       if (lane == 0) {
         uint8_t* dst = ring + (size_t)stage * Cfg::kStageBytes;
-        mbar_expect_tx(&full_bar[stage], 2 * Cfg::NF * 128);
-        tma_load_4d(dst, &tmX, &full_bar[stage], cblk * 128, M * tw - Cfg::PAD, M * th - Cfg::PAD, img);
-        tma_load_4d(dst + Cfg::kHalfBytes, &tmX, &full_bar[stage], cblk * 128 + 64, M * tw - Cfg::PAD, M * th - Cfg::PAD, img);
+        const int halves = 2 * u + 1 < num_sub ? 2 : 1;      // the last unit of an odd count has one half
+        mbar_expect_tx(&full_bar[stage], halves * Cfg::NF * 128);
+        for (int h = 0; h < halves; ++h) {
+          const unsigned sidx = 2 * u + h;
+          const int cb = (int)(sidx % CB64);
+          const unsigned p = (unsigned)p0 + sidx / CB64;
+          const int tw = (int)(p % (unsigned)Tw), th = (int)((p / (unsigned)Tw) % (unsigned)Th);
+          const int img = (int)(p / ((unsigned)Tw * (unsigned)Th));
+          tma_load_4d(dst + h * Cfg::kHalfBytes, &tmX, &full_bar[stage], cb * 64, M * tw - Cfg::PAD, M * th - Cfg::PAD, img);
+        }
       }
       __syncwarp();
     }
@@ -214,9 +223,11 @@ const uint64_t ad0 = umma_desc_mn_sw128(sa, Cfg::kHalfBytes);
     }
     for (uint32_t local = group; local < n_local && !timed_out; local += kEpiGroups) {
       const unsigned u = blockIdx.x + local * gridDim.x;
-      const int cblk = (int)(u % (unsigned)CB), pl = (int)(u / (unsigned)CB);
+      const unsigned sidx = 2 * u + (quad >> 1);            // this lane quadrant's (tile, channel block) pair
+      const int pl = (int)(sidx / CB64);
       const uint32_t acc = local % kNumAcc, acc_phase = (local / kNumAcc) & 1;
-      const int c = cblk * 128 + quad * 32 + lane;
+      // a pair past the end (odd count) has c >= C: nothing of it is stored or reduced
+      const int c = sidx < num_sub ? (int)(sidx % CB64) * 64 + (quad & 1) * 32 + lane : C;
       if (!mbar_wait_warp(&tmem_full[acc], acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols;
@@ -321,7 +332,7 @@ int launch_m(const nova_plan* plan, const Geom& g, const void* x, void* V, long 
       return (int)cudaErrorUnknown;
   }
   const int sms = plan->sm_count;
-  const long long units = (long long)pc * ((g.C + 127) / 128);
+  const long long units = ((long long)pc * ((g.C + 63) / 64) + 1) / 2;   // two (tile, 64-channel block) pairs each
   const int grid = (int)(units < sms ? units : sms);
   return (int)launch_overlapped(input_transform_tc_kernel<M, QMODE, R>, grid, kTcThreads, Cfg::kTotal, stream, tmX, tmK,
                                 V, g.C, g.Th, g.Tw, p0, pc, pc_pad, plan->status_dev, qslot);
