@@ -6,6 +6,6 @@ only; every step of the computation runs in the library's CUDA kernels.
 """
 from .binding import (  # noqa: F401
     NovaError, Plan, lib, status_string, maxpool2x2, snap_to_rational, verify_decomposition, symmetric_search,
-    FP32, FP16_F32ACC, COEF_ROUND_TO_MODE, COEF_FP32, RELU, GEMM_SIMT, GEMM_TCGEN05, TRANSFORM_SIMT, PROFILE_WAITS,
+    FP32, FP16_F32ACC, COEF_ROUND_TO_MODE, COEF_FP32, RELU, GEMM_SIMT, GEMM_TCGEN05, TRANSFORM_SIMT, PROFILE_WAITS, POOL2X2,
     EXPORTED_SYMBOLS, STATIC_SCRATCH_BYTES, QUANT_PER_TENSOR, QUANT_PER_CHANNEL, QUANT_GIVEN,
 )

@@ -12,6 +12,7 @@ GEMM_SIMT = 1 << 8
 GEMM_TCGEN05 = 2 << 8
 TRANSFORM_SIMT = 1 << 10
 PROFILE_WAITS = 1 << 13
+POOL2X2 = 1 << 14
 
 EXPORTED_SYMBOLS = (
     "nova_plan_create", "nova_plan_destroy", "nova_plan_get_matrices", "nova_plan_get_device_tables",
@@ -318,7 +319,7 @@ class Plan:
         N, H, W, C = x.shape
         K = U.shape[1]
         if y is None:
-            y = torch.empty(N, H, W, K, dtype=x.dtype, device=x.device)
+            y = torch.empty((N, H // 2, W // 2, K) if flags & POOL2X2 else (N, H, W, K), dtype=x.dtype, device=x.device)
         if workspace is None:
             workspace = torch.empty(self.workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device=x.device)
         _check(lib().nova_conv2d_fwd(self._h, x.data_ptr(), U.data_ptr(), y.data_ptr(), N, H, W, C, K,

@@ -65,7 +65,7 @@ bool on_plan_device(const nova_plan* p) {
 // The one-kernel path for 8 input channels runs unless a flag asks for a particular kernel of the
 // three-kernel path.
 bool use_fused_small_c(const nova_plan* p, const Geom& g, int flags) {
-  const int forcing = NOVA_GEMM_SIMT | NOVA_GEMM_TCGEN05 | NOVA_TRANSFORM_SIMT | NOVA_PROFILE_WAITS;
+  const int forcing = NOVA_GEMM_SIMT | NOVA_GEMM_TCGEN05 | NOVA_TRANSFORM_SIMT | NOVA_PROFILE_WAITS | NOVA_POOL2X2;
   return (flags & forcing) == 0 && fused_small_c_applies(p, g);
 }
 
@@ -136,6 +136,10 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
   if ((flags & NOVA_GEMM_TCGEN05) && p->mode == NOVA_FP32) return NOVA_ERR_UNSUPPORTED;
   if (p->device < 0) return NOVA_ERR_CUDA;
   if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
+  if (flags & NOVA_POOL2X2) {        // the pooled epilogue lives in the TMA-staged half-mode output transform
+    if ((H | W) & 1) return NOVA_ERR_INVALID_ARG;
+    if (p->mode != NOVA_FP16_F32ACC || !p->status_dev || (flags & NOVA_TRANSFORM_SIMT)) return NOVA_ERR_UNSUPPORTED;
+  }
   Geom g = make_geom(p, N, H, W, C, K);
   Chunking c;
   if (!choose_chunking(p, g, ws_bytes, &c)) return NOVA_ERR_WORKSPACE;
@@ -168,7 +172,7 @@ int conv2d_fwd_impl(const nova_plan* p, const void* x, const void* U, void* y, i
                      : launch_gemm_simt(p, Vb, U, Mb, nfreq, pc, c.pc_pad, C, K, stream);
     if (e) return NOVA_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4 * ci + 2], s);
-    const int relu = (flags & NOVA_RELU) ? 1 : 0;
+    const int relu = ((flags & NOVA_RELU) ? 1 : 0) | ((flags & NOVA_POOL2X2) ? 2 : 0);   // bit 1: pooled store
     if (f32 ? launch_output_transform_f32(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
         : (p->status_dev && !(flags & NOVA_TRANSFORM_SIMT))
             ? launch_output_transform_tma(p, g, Mb, y, p0, pc, c.pc_pad, relu, stream)
@@ -260,6 +264,7 @@ extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, cons
                                     int N, int H, int W, int C, int K, void* x_stage, void* y_stage,
                                     void* ws, size_t ws_bytes, int flags, nova_stream stream) {
   if (!p || !x_host || !y_host || !x_stage || !y_stage || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
+  if (flags & NOVA_POOL2X2) return NOVA_ERR_UNSUPPORTED;      // the staging of y is sized for the unpooled output
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t x_img = (size_t)H * W * C * elt_bytes(p->mode);
@@ -360,6 +365,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
       !(scale_V >= 0.f))
     return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
+  if (flags & NOVA_POOL2X2) return NOVA_ERR_UNSUPPORTED;
   if (!p->status_dev) return NOVA_ERR_CUDA;
   if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
   const Geom g = make_geom(p, N, H, W, C, K);

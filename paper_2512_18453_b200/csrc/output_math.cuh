@@ -163,5 +163,41 @@ __device__ __forceinline__ void store_tile(const V (&Y)[M][M], T* dst, size_t ro
   }
 }
 
+// max with NaN propagation (either operand NaN -> NaN; +0 > -0), as the pooling kernel's half max
+__device__ __forceinline__ float max_nan_f32(float a, float b) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ float vmax_nan(float a, float b) { return max_nan_f32(a, b); }
+__device__ __forceinline__ float2 vmax_nan(float2 a, float2 b) {
+  return make_float2(max_nan_f32(a.x, b.x), max_nan_f32(a.y, b.y));
+}
+
+// The same for the 2 x 2 / 2 max-pooled output: the largest of each 2 x 2 window of the tile goes to
+// dst + (pi * Wo + pj) * K, with dst, row_stride (= Wo * K), rows and cols those of the POOLED
+// tensor (H and W are even and m is even, so a window never straddles tiles or the image edge).
+// Max, ReLU and rounding are all monotone, so the result equals pooling the stored outputs.
+template <int M, typename T, typename V>
+__device__ __forceinline__ void store_tile_pooled(const V (&Y)[M][M], T* dst, size_t row_stride, int K, int rows,
+                                                  int cols, int relu) {
+  static_assert(M % 2 == 0, "pooling windows must not straddle tiles");
+  const float lo = relu ? 0.f : -__int_as_float(0x7f800000);
+#pragma unroll
+  for (int pi = 0; pi < M / 2; ++pi) {
+    if (pi < rows) {
+      T* p = dst;
+#pragma unroll
+      for (int pj = 0; pj < M / 2; ++pj) {
+        if (pj < cols)
+          vstore_cs(p, vmax_lo(vmax_nan(vmax_nan(Y[2 * pi][2 * pj], Y[2 * pi][2 * pj + 1]),
+                                        vmax_nan(Y[2 * pi + 1][2 * pj], Y[2 * pi + 1][2 * pj + 1])), lo));
+        p += K;
+      }
+    }
+    dst += row_stride;
+  }
+}
+
 }  // namespace xf
 }  // namespace nova

@@ -45,6 +45,7 @@ struct OtCfg {
 };
 
 // QUANT: M holds the int32 sums of the int8 pipeline; scale_U[k] * *scale_V dequantises filter k.
+// relu: bit 0 = ReLU, bit 1 = the 2 x 2 max-pooled store (y is then [N, H/2, W/2, K]).
 template <int M, typename T, bool SYM, int VEC, bool QUANT, int R = 3>
 __global__ void __launch_bounds__(kOtThreads, 1)
 output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ Coefs cf,
@@ -138,8 +139,14 @@ output_transform_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __gri
         const unsigned tw = p % (unsigned)Tw, q2 = p / (unsigned)Tw;
         const unsigned th = q2 % (unsigned)Th, img = q2 / (unsigned)Th;
         const int h0 = M * (int)th, w0 = M * (int)tw;
-        T* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
-        store_tile<M, T>(Y, dst, (size_t)W * K, K, H - h0, W - w0, relu);
+        if (relu & 2) {              // 2 x 2 / 2 max-pool before the store: y is [N, H/2, W/2, K]
+          const int Ho = H >> 1, Wo = W >> 1, ho = h0 >> 1, wo = w0 >> 1;
+          T* dst = y + (((size_t)img * Ho + ho) * Wo + wo) * K + k;
+          store_tile_pooled<M, T>(Y, dst, (size_t)Wo * K, K, Ho - ho, Wo - wo, relu & 1);
+        } else {
+          T* dst = y + (((size_t)img * H + h0) * W + w0) * K + k;
+          store_tile<M, T>(Y, dst, (size_t)W * K, K, H - h0, W - w0, relu & 1);
+        }
       }
     }
   }

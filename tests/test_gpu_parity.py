@@ -481,11 +481,14 @@ def test_cfg4_f8_full_size(kind):
     assert abs(plan.kappa() / want - 1) < 1e-3
 
 
-def _gpu_vgg(x, weights, m, pts, n_layers=None):
+def _gpu_vgg(x, weights, m, pts, n_layers=None, fused_pool=False):
     plan = nv.Plan(m, pts)
     a = torch.from_numpy(x).cuda()
     for gw, (_, _, pool) in list(zip(weights, VGG16_LAYERS))[:n_layers]:
         U = plan.filter_transform(torch.from_numpy(gw).cuda())
+        if pool and fused_pool:
+            a = plan.conv2d(a, U, flags=nv.RELU | nv.POOL2X2)
+            continue
         a = plan.conv2d(a, U, flags=nv.RELU)
         if pool:
             a = nv.maxpool2x2(a, nv.FP16_F32ACC)
@@ -981,3 +984,67 @@ def test_one_kernel_path_passes_nan_and_inf_through_relu_like_the_three_kernel_p
     assert np.array_equal(np.isnan(y), np.isnan(y3))
     assert np.isnan(y[0, 4:8, 4:8, :]).all()          # the tile that holds the pixel
     assert (y[~np.isnan(y)] >= 0).all()
+
+
+# ---------------------------------------------------------------- max-pool fused into the output transform
+@pytest.mark.parametrize("kind,m", [("std", 2), ("nova", 4), ("nova", 6), ("asym", 6), ("nova", 8), ("shuf", 8)])
+@pytest.mark.parametrize("shape,relu", [((2, 20, 18, 16, 24), True), ((1, 38, 30, 64, 72), False), ((3, 8, 50, 8, 64), True),
+                                        ((1, 2, 6, 8, 8), True)])
+def test_pooled_output_equals_pooling_the_unpooled_output(kind, m, shape, relu):
+    # NOVA_POOL2X2: the output transform stores the 2 x 2 / 2 max-pooled (ReLU'd) tile.  Bit for bit the
+    # pooling kernel applied to the unpooled output of the same call, and within the emulation's bounds of the
+    # pooled emulation; ragged tiles, images smaller than a tile, a ragged filter group and C = 8 (which then
+    # takes the three-kernel path) are among the cases.
+    N, H, W, C, K = shape
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=400 + m)
+    pts = point_set(kind, m)
+    plan = nv.Plan(m, pts)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    U = plan.filter_transform(gd)
+    fl = nv.RELU if relu else 0
+    y_full = plan.conv2d(xd, U, flags=fl | nv.GEMM_TCGEN05)
+    want = nv.maxpool2x2(y_full, nv.FP16_F32ACC)
+    got = torch.full((N, H // 2, W // 2, K), float("nan"), dtype=torch.float16, device="cuda")
+    plan.conv2d(xd, U, y=got, flags=fl | nv.POOL2X2)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert got.shape == want.shape
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    ye = conv.winograd_conv_emulated(x, g, m, pts, "fp16", apply_relu=relu)
+    y1 = conv.direct_conv_fp64(x, g)
+    if relu:
+        y1 = np.maximum(y1, 0.0)
+    pe, p1 = conv.maxpool2x2(ye.astype(np.float64)), conv.maxpool2x2(y1)
+    e_emu = conv.rel_l2(pe, p1)
+    if np.isfinite(e_emu) and e_emu < 1.0:
+        assert conv.rel_l2(got.cpu().numpy(), p1) <= 2.0 * e_emu + 1e-4
+        assert conv.rel_l2(got.cpu().numpy(), pe) <= EMU_CLOSE * e_emu + 1e-4
+
+
+def test_pooled_output_keeps_nan_and_rejects_what_it_does_not_support():
+    m, N, H, W, C, K = 4, 1, 12, 12, 16, 16
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", False, True, seed=411)
+    x[0, 5, 5, 2] = np.nan
+    plan = nv.Plan(m, point_set("nova", m))
+    xd = torch.from_numpy(x).cuda()
+    U = plan.filter_transform(torch.from_numpy(g).cuda())
+    got = plan.conv2d(xd, U, flags=nv.RELU | nv.POOL2X2).cpu().numpy()
+    want = nv.maxpool2x2(plan.conv2d(xd, U, flags=nv.RELU), nv.FP16_F32ACC).cpu().numpy()
+    assert np.array_equal(got, want, equal_nan=True) and np.isnan(got[0, 2:4, 2:4, :]).all()
+    with pytest.raises(nv.NovaError):                       # odd height
+        plan.conv2d(xd[:, :11].contiguous(), U, flags=nv.POOL2X2)
+    with pytest.raises(nv.NovaError):                       # the plain output transform has no pooled store
+        plan.conv2d(xd, U, flags=nv.POOL2X2 | nv.TRANSFORM_SIMT)
+    p32 = nv.Plan(m, point_set("nova", m), nv.FP32)
+    x32 = torch.from_numpy(x.astype(np.float32)).cuda()
+    U32 = p32.filter_transform(torch.from_numpy(g.astype(np.float32)).cuda())
+    with pytest.raises(nv.NovaError):                       # fp32 mode
+        p32.conv2d(x32, U32, flags=nv.POOL2X2)
+
+
+def test_vgg_stack_with_fused_pooling_gives_the_same_bits():
+    x, weights = make_vgg_inputs(2, HW=64)
+    pts = point_set("nova", 8)
+    a = _gpu_vgg(x, weights, 8, pts)
+    b = _gpu_vgg(x, weights, 8, pts, fused_pool=True)
+    assert a.shape == b.shape and np.array_equal(a.view(np.int16), b.view(np.int16))
