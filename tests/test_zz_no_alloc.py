@@ -43,7 +43,8 @@ def test_static_scratch_matches_workspace_entry_point_on_two_calls_in_a_row():
         pytest.fail("needs a CUDA device; there is no CPU fallback")
     # two different problems back to back: the second one finds the first one's
     # data in the shared scratch (different tile count, channel count and tile size)
-    for m, shape, seed in ((6, (3, 40, 44, 72, 136), 901), (4, (2, 50, 50, 64, 64), 902)):
+    # the third has 8 input channels: the one-kernel path, which touches no scratch at all
+    for m, shape, seed in ((6, (3, 40, 44, 72, 136), 901), (4, (2, 50, 50, 64, 64), 902), (8, (2, 30, 26, 8, 72), 903)):
         a, b, (x, g, plan, _, _, _) = _both_ways(m, shape, seed)
         assert np.isfinite(a.astype(np.float32)).all()
         # same kernels, same chunking: the same bits (within the tolerance of the other tests, which is 0 here)
