@@ -520,6 +520,9 @@ def test_cfg5_vgg16_stack_f8_nova_two_images():
     pts = point_set("nova", 8)
     y = _gpu_vgg(x, weights, 8, pts)
     assert y.shape == (2, 7, 7, 512)
+    # the configuration the bench times fuses the five max-pools into the output transforms: same bits
+    yf = _gpu_vgg(x, weights, 8, pts, fused_pool=True)
+    assert np.array_equal(y.view(np.int16), yf.view(np.int16))
     ref = conv.vgg_stack_fp64(x, weights, VGG16_LAYERS)
     emu = conv.vgg_stack_emulated(x, weights, VGG16_LAYERS, 8, pts)
     e_gpu, e_emu = conv.rel_l2(y, ref), conv.rel_l2(emu, ref)
@@ -530,7 +533,7 @@ def test_cfg5_vgg16_stack_f8_nova_two_images():
 
 
 def test_cfg5_first_two_layers_tile_by_tile():
-    """The two 224 x 224 layers of the stack (C = 8 with the CUDA-core input transform, then C = K = 64)
+    """The two 224 x 224 layers of the stack (C = 8 in the one-kernel path, then C = K = 64)
     on one image, each judged on its own like any single layer: against the direct convolution, and
     tile by tile against the emulation (the stack test above can only judge the final features)."""
     x, weights = make_vgg_inputs(1)
