@@ -61,7 +61,9 @@ enum {
   NOVA_POOL2X2 = 1 << 14,   /* 2 x 2 max-pool, stride 2, fused into the output transform (after the ReLU if
                                both are given): y_dev is [N, H/2, W/2, K]; the result equals nova_maxpool2x2
                                of the unpooled output.  H and W even; NOVA_FP16_F32ACC with the default
-                               (TMA-staged) output transform only, NOVA_ERR_UNSUPPORTED otherwise */
+                               (TMA-staged) output transform only, NOVA_ERR_UNSUPPORTED otherwise; also
+                               accepted by nova_conv2d_fwd_static, _host (y_host and y_stage pooled) and
+                               the INT8 entry points */
   NOVA_TRANSFORM_SIMT = 1 << 10 /* plain transform kernels: the input transform on CUDA cores even
                                    where the tensor-core formulation applies, the output transform
                                    without TMA staging (testing) */

@@ -386,7 +386,7 @@ class Plan:
         K = Uq.shape[1]
         assert x.is_cuda and x.is_contiguous() and x.dtype == torch.float16 and Uq.dtype == torch.int8
         if y is None:
-            y = torch.empty((N, H, W, K), dtype=torch.float16, device=x.device)
+            y = torch.empty((N, H // 2, W // 2, K) if flags & POOL2X2 else (N, H, W, K), dtype=torch.float16, device=x.device)
         if workspace is None:
             workspace = torch.empty(self.int8_workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device=x.device)
         args = (self._h, x.data_ptr(), Uq.data_ptr(), scale_U.data_ptr(), float(scale_V), y.data_ptr(),

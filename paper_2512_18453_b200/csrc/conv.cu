@@ -264,11 +264,11 @@ extern "C" int nova_conv2d_fwd_host(const nova_plan* p, const void* x_host, cons
                                     int N, int H, int W, int C, int K, void* x_stage, void* y_stage,
                                     void* ws, size_t ws_bytes, int flags, nova_stream stream) {
   if (!p || !x_host || !y_host || !x_stage || !y_stage || !shape_ok(N, H, W, C, K)) return NOVA_ERR_INVALID_ARG;
-  if (flags & NOVA_POOL2X2) return NOVA_ERR_UNSUPPORTED;      // the staging of y is sized for the unpooled output
   if (!device_plan(p)) return NOVA_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t x_img = (size_t)H * W * C * elt_bytes(p->mode);
-  const size_t y_img = (size_t)H * W * K * elt_bytes(p->mode);
+  const bool pooled = (flags & NOVA_POOL2X2) != 0;          // y_host and y_stage then hold [N, H/2, W/2, K]
+  const size_t y_img = (size_t)(pooled ? H / 2 : H) * (pooled ? W / 2 : W) * K * elt_bytes(p->mode);
   std::lock_guard<std::mutex> lock(g_pipe_mu);
   HostPipe* hp = host_pipe();
   if (!hp) return NOVA_ERR_CUDA;
@@ -365,7 +365,7 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
       !(scale_V >= 0.f))
     return p && (p->mode != NOVA_FP16_F32ACC || !device_plan(p)) ? NOVA_ERR_UNSUPPORTED : NOVA_ERR_INVALID_ARG;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign)) return NOVA_ERR_WORKSPACE;
-  if (flags & NOVA_POOL2X2) return NOVA_ERR_UNSUPPORTED;
+  if ((flags & NOVA_POOL2X2) && ((H | W) & 1)) return NOVA_ERR_INVALID_ARG;
   if (!p->status_dev) return NOVA_ERR_CUDA;
   if (!on_plan_device(p)) return NOVA_ERR_INVALID_ARG;
   const Geom g = make_geom(p, N, H, W, C, K);
@@ -401,7 +401,8 @@ int conv2d_int8_impl(const nova_plan* p, const void* x, const void* Uq, const fl
                                  : launch_gemm_tcgen05_i8(p, Vq, Uq, Mb, nfreq, pc, l.pad, C, K, p->status_dev, stream);
   if (ev) cudaEventRecord(ev[2], s);
   if (!e)
-    e = launch_output_transform_tma(p, g, Mb, y, 0, pc, l.pad, (flags & NOVA_RELU) ? 1 : 0, stream, scale_U, slot);
+    e = launch_output_transform_tma(p, g, Mb, y, 0, pc, l.pad,
+                                    ((flags & NOVA_RELU) ? 1 : 0) | ((flags & NOVA_POOL2X2) ? 2 : 0), stream, scale_U, slot);
   if (ev) cudaEventRecord(ev[3], s);
   if (e) g_last_cuda_error = e;
   return e ? NOVA_ERR_CUDA : NOVA_OK;

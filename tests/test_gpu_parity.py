@@ -1053,3 +1053,30 @@ def test_vgg_stack_with_fused_pooling_gives_the_same_bits():
     a = _gpu_vgg(x, weights, 8, pts)
     b = _gpu_vgg(x, weights, 8, pts, fused_pool=True)
     assert a.shape == b.shape and np.array_equal(a.view(np.int16), b.view(np.int16))
+
+
+def test_pooled_output_through_the_int8_and_host_entry_points():
+    m, N, H, W, C, K = 4, 3, 20, 24, 64, 80
+    x, g = make_conv_inputs(N, H, W, C, K, "fp16", True, True, seed=421)
+    pts = point_set("nova", m)
+    plan = nv.Plan(m, pts, nv.FP16_F32ACC, nv.COEF_FP32)
+    xd, gd = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+    # INT8 pipeline: same quantised product, pooled or not
+    Uq, sU = plan.filter_transform_int8(gd)
+    full = plan.conv2d_int8(xd, Uq, sU, flags=nv.RELU)
+    got = plan.conv2d_int8(xd, Uq, sU, flags=nv.RELU | nv.POOL2X2)
+    want = nv.maxpool2x2(full, nv.FP16_F32ACC)
+    assert got.shape == want.shape and torch.equal(got.view(torch.int16), want.view(torch.int16))
+    # host buffers in and out
+    plan16 = nv.Plan(m, pts)
+    U = plan16.filter_transform(gd)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.full((N, H // 2, W // 2, K), float("nan"), dtype=torch.float16).pin_memory()
+    xs = torch.empty(N, H, W, C, dtype=torch.float16, device="cuda")
+    ys = torch.empty(N, H // 2, W // 2, K, dtype=torch.float16, device="cuda")
+    ws = torch.empty(plan16.workspace_bytes(N, H, W, C, K), dtype=torch.uint8, device="cuda")
+    plan16.conv2d_host(xh, U, yh, xs, ys, ws, flags=nv.RELU | nv.POOL2X2)
+    torch.cuda.synchronize()
+    want16 = nv.maxpool2x2(plan16.conv2d(xd, U, flags=nv.RELU), nv.FP16_F32ACC).cpu()
+    assert torch.equal(yh.view(torch.int16), want16.view(torch.int16))
+    assert plan.device_status() == 0 and plan16.device_status() == 0
