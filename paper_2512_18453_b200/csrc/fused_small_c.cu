@@ -148,6 +148,7 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
   uint64_t* y_full = bars + 3;       // the image of y is complete                        (product warps)
   uint64_t* y_free = bars + 4;       // the copies to global memory have read the image   (storing warps)
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 5);
+  volatile int* helper_stop = abort_flag + 1;
   TileRec* rec = reinterpret_cast<TileRec*>(smem + L::kOffBar + 64);         // [4][8]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -162,6 +163,7 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
     mbar_init(y_full, kProductWarps);
     mbar_init(y_free, kHelperWarps);
     *abort_flag = 0;
+    *helper_stop = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -288,8 +290,12 @@ fused_small_c_kernel(const __grid_constant__ Coefs cf, const __grid_constant__ C
 #pragma unroll
         for (int xi = 0; xi < N; ++xi) dst[xi * N * 4] = o[xi];
       }
+      // One thread samples the abort flag before the barrier and every helper reads that sample
+      // after it: the helpers leave the loop together or not at all (a flag read by each thread
+      // for itself could change between two reads and strand the others at the next barrier).
+      if (ht == 0) *helper_stop = *abort_flag;
       helper_sync();                 // T is complete and the patch buffer is free
-      if (*abort_flag) break;        // uniform: every helper reads the flag after the same barrier
+      if (*helper_stop) break;
       if (grp + ctas < groups) fetch(grp + ctas, (it + 1) & 3);
       if (it > 1) store_release();   // the copies of group it - 2, issued one iteration ago
       if (!mbar_poll(v_free, (it & 1) ^ 1, abort_flag)) *abort_flag = 1;   // on the critical path
