@@ -220,3 +220,25 @@ def test_symmetric_search_through_the_abi_finds_the_discovered_sets():
     with pytest.raises(nv.NovaError) as e:                       # too many combinations to enumerate
         nv.symmetric_search(9, 30, 5)
     assert e.value.status == -7
+
+
+def test_binding_constants_agree_with_the_header():
+    # the flag, mode and error values of the binding are those include/nova.h declares (parsed from the
+    # header's enums; catches a constant changed on one side only)
+    text = open(os.path.join(os.path.dirname(__file__), "..", "include", "nova.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+
+    def header_value(name):
+        m = re.search(r"\b%s\s*=\s*([^,}\n]+)" % name, text)
+        assert m, name
+        return int(eval(m.group(1).strip(), {"__builtins__": {}}, {}))
+    pairs = {"NOVA_RELU": nv.RELU, "NOVA_GEMM_SIMT": nv.GEMM_SIMT, "NOVA_GEMM_TCGEN05": nv.GEMM_TCGEN05,
+             "NOVA_TRANSFORM_SIMT": nv.TRANSFORM_SIMT, "NOVA_PROFILE_WAITS": nv.PROFILE_WAITS,
+             "NOVA_POOL2X2": nv.POOL2X2, "NOVA_FP32": nv.FP32, "NOVA_FP16_F32ACC": nv.FP16_F32ACC,
+             "NOVA_COEF_ROUND_TO_MODE": nv.COEF_ROUND_TO_MODE, "NOVA_COEF_FP32": nv.COEF_FP32}
+    for name, value in pairs.items():
+        assert header_value(name) == value, name
+    flags = [nv.RELU, nv.GEMM_SIMT, nv.GEMM_TCGEN05, nv.TRANSFORM_SIMT, nv.PROFILE_WAITS, nv.POOL2X2]
+    assert len(set(flags)) == len(flags) and all(a & b == 0 for i, a in enumerate(flags) for b in flags[i + 1:])
+    m = re.search(r"#define\s+NOVA_STATIC_SCRATCH_BYTES\s+\(\(size_t\)(\d+)\s*<<\s*(\d+)\)", text)
+    assert m and (int(m.group(1)) << int(m.group(2))) == nv.STATIC_SCRATCH_BYTES
